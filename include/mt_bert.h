@@ -1,0 +1,205 @@
+/*
+ * mt_bert.h - C ABI of the merged multi-task BERT forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The paper (Section 3.3, Fig. 1(c)) merges several single-task student models - each made of
+ * x frozen bottom layers of one pre-trained BERT encoder plus y task-specific transformer layers,
+ * Table 2's "(x, y)" - into ONE computation graph whose frozen layers are evaluated once per
+ * request and shared by all tasks.  Every task reads the shared trunk after its own depth
+ * (Section 5.1), runs its own layers, and a request yields the output of every task (Section 5.2).
+ * This library is that serving-time graph: mt_create() builds the tree, mt_load_weights() loads
+ * the checkpoints into it, mt_forward() evaluates it.
+ *
+ * Conventions
+ *  - All device memory and all streams belong to the caller.  The library allocates only host
+ *    metadata.  Pointers named d_* are DEVICE pointers, everything else is a HOST pointer.
+ *  - cudaStream_t is passed as a plain `void*` (the value of the stream handle; NULL = default stream).
+ *  - Activations and weights are bf16, accumulation and statistics fp32, logits fp32.
+ *  - Every entry point returns an mt_status (0 = OK, negative = error); nothing throws, aborts or
+ *    traps.  mt_last_error_string() describes the most recent failure on that model.
+ *  - Encoder layer (the published post-LayerNorm BERT layer the paper builds on, Section 3):
+ *        u  = x + (softmax(QK^T/sqrt(64) over valid keys) V) Wo^T + bo ;  h1 = LN(u)
+ *        h2 = LN(h1 + GELU_erf(h1 W1^T + b1) W2^T + b2)
+ *    with Q,K,V = x W{q,k,v}^T + b, every W stored [out, in], LN with biased variance.
+ *  - There is no CPU fallback: without a CUDA device every compute entry point fails with MT_ERR_CUDA.
+ */
+#ifndef MT_BERT_H_
+#define MT_BERT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MT_OK = 0,
+  MT_ERR_INVALID_ARG = -1,   /* null pointer, bad index, empty task mask ...              */
+  MT_ERR_SHAPE = -2,         /* batch/seq beyond the limits given to mt_create             */
+  MT_ERR_NOT_BOUND = -3,     /* mt_bind_memory has not been called                         */
+  MT_ERR_NOT_LOADED = -4,    /* weights of the trunk or of an active task are not loaded   */
+  MT_ERR_BLOB_MISMATCH = -5, /* weight blob header/size disagrees with the configuration   */
+  MT_ERR_CUDA = -6,          /* a CUDA runtime/driver call failed                          */
+  MT_ERR_UNSUPPORTED = -7,   /* configuration outside what the kernels implement           */
+  MT_ERR_DEVICE_FLAG = -8    /* mt_poll_status: the device status word is non-zero         */
+} mt_status;
+
+/* Bits of the sticky device status word returned through mt_poll_status(). */
+#define MT_FLAG_BAD_TOKEN    0x1u  /* a token id was outside [0, vocab): clamped              */
+#define MT_FLAG_BAD_SEGMENT  0x2u  /* a segment id was outside [0, type_vocab): clamped       */
+#define MT_FLAG_BAD_LENGTH   0x4u  /* a length was outside [1, seq]: clamped                  */
+#define MT_FLAG_WAIT_TIMEOUT 0x8u  /* a pipeline wait inside a kernel gave up (results invalid) */
+
+/* Encoder shared by trunk and branches: the paper uses 12-layer uncased BERT-base (Section 3). */
+typedef struct {
+  int32_t vocab_size;    /* 30522 */
+  int32_t max_position;  /* 512: learned absolute positions */
+  int32_t type_vocab;    /* 2 */
+  int32_t hidden;        /* 768 or 1024; must be heads * 64 */
+  int32_t heads;         /* 12 or 16 */
+  int32_t ffn;           /* 3072 or 4096 */
+  int32_t trunk_layers;  /* number of frozen layers loaded (12 for BERT-base) */
+  float   ln_eps;        /* 1e-12 */
+  int32_t activation;    /* 0 = exact (erf) GELU; nothing else is implemented */
+} mt_trunk_config;
+
+/* One student model before merging, Table 2's (x, y): x = fork_depth frozen layers, y = branch_layers. */
+typedef struct {
+  int32_t fork_depth;     /* 0..trunk_layers; 0 forks off the embedding output */
+  int32_t branch_layers;  /* >= 0; 0 pools the trunk state directly            */
+  int32_t num_classes;    /* >= 1; 1 = regression head (raw output)            */
+} mt_task_config;
+
+typedef struct mt_model mt_model;
+
+/* ---- model merging (Section 3.3) ------------------------------------------------------------ */
+
+/* Builds the merged tree for n_tasks (1..64) students over one trunk.  No GPU work.
+ * max_batch*max_seq bounds every later mt_forward; max_seq <= max_position and <= 512.
+ * *out receives a heap object owned by the caller until mt_destroy().
+ * Errors: INVALID_ARG (nulls, depths out of range), UNSUPPORTED (hidden != heads*64, hidden/ffn not
+ * multiples of 256, activation != 0). */
+int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t n_tasks,
+              int32_t max_batch, int32_t max_seq, mt_model** out);
+void mt_destroy(mt_model* m);
+
+/* Sizes (bytes) of the two caller-provided device arenas.  The workspace size grows when the
+ * debug capture is enabled (mt_set_option "debug_capture") - query it after setting that option. */
+size_t mt_weights_bytes(const mt_model* m);
+size_t mt_workspace_bytes(const mt_model* m);
+
+/* Hands the library its two device arenas (both 256-byte aligned, at least the sizes above).
+ * The caller keeps ownership and must keep them alive while the model is used. */
+int mt_bind_memory(mt_model* m, void* d_weights, size_t weights_bytes, void* d_workspace, size_t workspace_bytes);
+
+/* Size and layout of the host weight blob: a 256-byte header followed by bf16 tensors, each padded
+ * to 256 bytes, in this order: word/position/type embedding tables, embedding LN gamma/beta; for
+ * every trunk layer: wq wk wv bq bk bv wo bo ln1_g ln1_b w1 b1 w2 b2 ln2_g ln2_b; then for every task
+ * its branch layers (same 16 tensors each), pool_w [H,H], pool_b, cls_w [C,H], cls_b.
+ * Header (little endian): u32 magic 'MTBW'=0x4D544257, u32 version=1, u32 kind (0 full, 1 one task),
+ * i32 hidden, heads, ffn, trunk_layers, vocab, max_position, type_vocab, n_tasks, task_index (-1 for
+ * full), fork_depth, branch_layers, num_classes (of that task; 0 for full), i32 reserved = 0,
+ * u64 payload_bytes (at byte 64). */
+size_t mt_blob_bytes(const mt_model* m);
+size_t mt_task_blob_bytes(const mt_model* m, int32_t task);
+
+/* "Load weights from multiple model checkpoints into one computation graph" (Section 3.3).
+ * Validates the header against the configuration, then copies the payload to the weights arena
+ * with cudaMemcpyAsync on `stream` (host_blob must stay valid until the stream reaches that point;
+ * pinned memory makes the copy asynchronous).  Errors: NOT_BOUND, BLOB_MISMATCH, CUDA. */
+int mt_load_weights(mt_model* m, const void* host_blob, size_t bytes, void* stream);
+
+/* Per-task update (Sections 1 and 5.1: a task is modified without affecting the others):
+ * replaces the branch layers, pooler and head of one task; nothing else in the arena is touched. */
+int mt_load_task_weights(mt_model* m, int32_t task, const void* host_blob, size_t bytes, void* stream);
+
+/* ---- the hot path ---------------------------------------------------------------------------- */
+
+/* Merged multi-task forward of one padded batch.
+ *   d_token_ids, d_segment_ids : int32 [batch, seq] row-major (device)
+ *   d_lengths                  : int32 [batch], valid tokens per sequence, 1..seq (device)
+ *   task_mask                  : bit t set = task t is evaluated; 0 is an error
+ *   d_logits                   : fp32 [batch, C_total] row-major (device), task t in columns
+ *                                [off_t, off_t + C_t), off_t = sum of C of the tasks before it;
+ *                                columns of tasks not in the mask are left untouched
+ * The shared trunk runs once, to the deepest fork among the active tasks only; each active task's
+ * branch starts from the trunk state at its fork depth; keys at positions >= length are excluded
+ * from every softmax; the pooler reads position 0.  Asynchronous: only enqueues kernels on `stream`,
+ * never synchronises, never allocates device memory.  The first call for a given
+ * (batch, seq, task_mask) builds and caches a launch plan on the host.
+ * Errors: INVALID_ARG, SHAPE, NOT_BOUND, NOT_LOADED, CUDA. */
+int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
+               const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
+               float* d_logits, void* stream);
+
+/* Same computation from HOST buffers: copies the three inputs to the workspace, runs mt_forward,
+ * copies the logits back to h_logits ([batch, C_total] fp32) and synchronises the stream.
+ * Pinned host buffers make the copies asynchronous with respect to the host. */
+int mt_forward_host(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids,
+                    const int32_t* h_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
+                    float* h_logits, void* stream);
+
+/* Synchronises `stream`, reads the sticky device status word into *flags (may be NULL) and clears
+ * it.  Returns MT_ERR_DEVICE_FLAG if it was non-zero. */
+int mt_poll_status(mt_model* m, void* stream, uint32_t* flags);
+
+/* ---- scheduler introspection (host only, no GPU needed) --------------------------------------- */
+
+/* The tree scheduler runs trunk layer w and every branch layer whose input is ready as one
+ * "wave" of grouped launches.  These report the plan for a task mask: the number of transformer
+ * layers executed (the paper's overhead measure, Section 4.1: shared depth + sum of task layers),
+ * the number of waves, and per wave the number of layers grouped in it (groups_per_wave may be NULL;
+ * otherwise room for trunk_layers + max branch_layers + 1 ints). */
+int mt_plan_summary(const mt_model* m, uint64_t task_mask, int32_t* n_layers, int32_t* n_waves,
+                    int32_t* trunk_depth, int32_t* groups_per_wave);
+/* Kernel launches one mt_forward enqueues for this mask (after its plan exists). */
+int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches);
+
+/* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
+ * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
+ * mt_workspace_bytes; set before mt_bind_memory). */
+int mt_set_option(mt_model* m, const char* key, int64_t value);
+
+/* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out.
+ * task = -1: trunk state after `layer` layers (0 = embedding output); task >= 0: state after branch
+ * layer `layer` (1-based) of that task.  Requires option debug_capture = 1. */
+int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out_bf16, void* stream);
+
+const char* mt_last_error_string(const mt_model* m);
+
+/* ---- the individual steps, callable on their own (used by the per-kernel parity tests) -------- */
+/* All pointers are device pointers; d_status may be NULL or point to one uint32 status word.      */
+
+/* Y[M,N] = epilogue(X[M,K] . W[N,K]^T + bias[N]) on tcgen05 tensor cores (bf16 in, fp32 accumulate).
+ * epilogue 0: +bias; 1: +bias then erf-GELU; 2: +bias +residual[M,N].  K % 64 == 0, N % 128 == 0,
+ * all pointers 16-byte aligned.  This is one linear map of the layer above. */
+int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
+                     void* d_y, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                     uint32_t* d_status, void* stream);
+
+/* ctx[B*S, heads*64] = softmax(QK^T/8 masked to keys < length) V per (sequence, head), from the
+ * packed projection qkv[B*S, 3*heads*64] = [Q | K | V].  Rows at positions >= length are written as 0. */
+int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx,
+                        int32_t batch, int32_t seq, int32_t heads, void* stream);
+
+/* y[rows, hidden] = LayerNorm(x) * gamma + beta (fp32 statistics, biased variance). hidden in {768, 1024}. */
+int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y,
+                        int32_t rows, int32_t hidden, float eps, void* stream);
+
+/* h0[B*S, hidden] = LayerNorm(word[tok] + pos[position] + type[seg]). */
+int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
+                    const void* d_word, const void* d_pos, const void* d_type,
+                    const void* d_gamma, const void* d_beta, void* d_h0,
+                    int32_t batch, int32_t seq, int32_t hidden, int32_t vocab, int32_t type_vocab,
+                    float eps, uint32_t* d_status, void* stream);
+
+/* logits[b, col0 + c] = cls_w[c,:] . tanh(pool_w . h[b*seq, :] + pool_b) + cls_b[c], c < num_classes. */
+int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void* d_pool_b,
+                          const void* d_cls_w, const void* d_cls_b, float* d_logits,
+                          int32_t batch, int32_t seq, int32_t hidden, int32_t num_classes,
+                          int32_t logits_stride, int32_t col0, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MT_BERT_H_ */

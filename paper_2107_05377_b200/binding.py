@@ -1,0 +1,259 @@
+"""ctypes binding of the C-ABI library (``include/mt_bert.h``), same names.
+
+Argument marshalling only: every step of the forward pass runs in the CUDA
+kernels of ``libmt_bert.so``.  PyTorch appears only as the owner of device
+memory and streams in the ``MTModel`` convenience wrapper.  There is no
+fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libmt_bert.so")
+
+MT_OK = 0
+ERRORS = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "NOT_BOUND", -4: "NOT_LOADED", -5: "BLOB_MISMATCH",
+          -6: "CUDA", -7: "UNSUPPORTED", -8: "DEVICE_FLAG"}
+FLAG_BAD_TOKEN, FLAG_BAD_SEGMENT, FLAG_BAD_LENGTH, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
+
+
+class TrunkConfig(C.Structure):
+    _fields_ = [("vocab_size", C.c_int32), ("max_position", C.c_int32), ("type_vocab", C.c_int32),
+                ("hidden", C.c_int32), ("heads", C.c_int32), ("ffn", C.c_int32), ("trunk_layers", C.c_int32),
+                ("ln_eps", C.c_float), ("activation", C.c_int32)]
+
+
+class TaskConfig(C.Structure):
+    _fields_ = [("fork_depth", C.c_int32), ("branch_layers", C.c_int32), ("num_classes", C.c_int32)]
+
+
+# name -> (restype, argtypes); the list is also what the symbol-export test checks.
+_P, _I32, _U64, _SZ = C.c_void_p, C.c_int32, C.c_uint64, C.c_size_t
+SIGNATURES = {
+    "mt_create": (C.c_int, [C.POINTER(TrunkConfig), C.POINTER(TaskConfig), _I32, _I32, _I32, C.POINTER(_P)]),
+    "mt_destroy": (None, [_P]),
+    "mt_weights_bytes": (_SZ, [_P]),
+    "mt_workspace_bytes": (_SZ, [_P]),
+    "mt_bind_memory": (C.c_int, [_P, _P, _SZ, _P, _SZ]),
+    "mt_blob_bytes": (_SZ, [_P]),
+    "mt_task_blob_bytes": (_SZ, [_P, _I32]),
+    "mt_load_weights": (C.c_int, [_P, _P, _SZ, _P]),
+    "mt_load_task_weights": (C.c_int, [_P, _I32, _P, _SZ, _P]),
+    "mt_forward": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
+    "mt_forward_host": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
+    "mt_poll_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
+    "mt_plan_summary": (C.c_int, [_P, _U64, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32)]),
+    "mt_plan_launches": (C.c_int, [_P, _U64, C.POINTER(_I32)]),
+    "mt_set_option": (C.c_int, [_P, C.c_char_p, C.c_int64]),
+    "mt_debug_copy_hidden": (C.c_int, [_P, _I32, _I32, _P, _P]),
+    "mt_last_error_string": (C.c_char_p, [_P]),
+    "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _P]),
+    "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
+    "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P, _P]),
+    "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
+}
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libmt_bert.so (built by ``python -m paper_2107_05377_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2107_05377_b200.build` "
+                               "(there is no fallback path)")
+        handle = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+class MTError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        super().__init__(f"{where}: {ERRORS.get(code, code)} {detail}".strip())
+        self.code = code
+
+
+def _check(code: int, where: str, model=None) -> None:
+    if code != MT_OK:
+        detail = lib().mt_last_error_string(model).decode() if model else ""
+        raise MTError(code, where, detail)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream=None) -> int:
+    import torch
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+# ---------------------------------------------------------------------------
+# single steps (device tensors in, device tensors out)
+# ---------------------------------------------------------------------------
+
+def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream=None) -> None:
+    M, K = x.shape
+    N = w.shape[0]
+    _check(lib().mt_kernel_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), M, N, K, epilogue,
+                                  _ptr(status), _stream(stream)), "mt_kernel_linear")
+
+
+def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None) -> None:
+    _check(lib().mt_kernel_attention(_ptr(qkv), _ptr(lengths), _ptr(ctx), batch, seq, heads, _stream(stream)),
+           "mt_kernel_attention")
+
+
+def mt_kernel_layernorm(x, gamma, beta, y, eps: float, stream=None) -> None:
+    rows, hidden = x.shape
+    _check(lib().mt_kernel_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), rows, hidden, eps, _stream(stream)),
+           "mt_kernel_layernorm")
+
+
+def mt_kernel_embed(token_ids, segment_ids, lengths, word, pos, type_, gamma, beta, h0, eps: float, status=None,
+                    stream=None) -> None:
+    batch, seq = token_ids.shape
+    _check(lib().mt_kernel_embed(_ptr(token_ids), _ptr(segment_ids), _ptr(lengths), _ptr(word), _ptr(pos), _ptr(type_),
+                                 _ptr(gamma), _ptr(beta), _ptr(h0), batch, seq, word.shape[1], word.shape[0],
+                                 type_.shape[0], eps, _ptr(status), _stream(stream)), "mt_kernel_embed")
+
+
+def mt_kernel_pooler_head(hidden, pool_w, pool_b, cls_w, cls_b, logits, batch: int, seq: int, col0: int = 0,
+                          stream=None) -> None:
+    _check(lib().mt_kernel_pooler_head(_ptr(hidden), _ptr(pool_w), _ptr(pool_b), _ptr(cls_w), _ptr(cls_b), _ptr(logits),
+                                       batch, seq, pool_w.shape[0], cls_w.shape[0], logits.shape[1], col0,
+                                       _stream(stream)), "mt_kernel_pooler_head")
+
+
+# ---------------------------------------------------------------------------
+# the model
+# ---------------------------------------------------------------------------
+
+class MTModel:
+    """mt_create + mt_bind_memory + mt_load_weights + mt_forward around torch-owned memory."""
+
+    def __init__(self, cfg, max_batch: int, max_seq: int, max_groups: Optional[int] = None,
+                 debug_capture: bool = False, device: str = "cuda:0", bind: bool = True):
+        self.cfg = cfg
+        self.max_batch, self.max_seq = max_batch, max_seq
+        self.handle = _P()
+        trunk = TrunkConfig(cfg.vocab_size, cfg.max_position, cfg.type_vocab, cfg.hidden, cfg.heads, cfg.ffn,
+                            cfg.trunk_layers, cfg.ln_eps, 0)
+        tasks = (TaskConfig * cfg.n_tasks)(*[TaskConfig(t.fork_depth, t.branch_layers, t.num_classes)
+                                             for t in cfg.tasks])
+        _check(lib().mt_create(C.byref(trunk), tasks, cfg.n_tasks, max_batch, max_seq, C.byref(self.handle)),
+               "mt_create")
+        if max_groups is not None:
+            self.set_option("max_groups", max_groups)
+        if debug_capture:
+            self.set_option("debug_capture", 1)
+        self.c_total = cfg.total_classes
+        self.weights = self.workspace = None
+        if bind:
+            self.bind(device)
+
+    # -- host-only ----------------------------------------------------------
+    def set_option(self, key: str, value: int) -> None:
+        _check(lib().mt_set_option(self.handle, key.encode(), value), "mt_set_option", self.handle)
+
+    def weights_bytes(self) -> int:
+        return lib().mt_weights_bytes(self.handle)
+
+    def workspace_bytes(self) -> int:
+        return lib().mt_workspace_bytes(self.handle)
+
+    def blob_bytes(self) -> int:
+        return lib().mt_blob_bytes(self.handle)
+
+    def task_blob_bytes(self, task: int) -> int:
+        return lib().mt_task_blob_bytes(self.handle, task)
+
+    def plan_summary(self, task_mask: int):
+        n_layers, n_waves, depth = _I32(), _I32(), _I32()
+        cap = self.cfg.trunk_layers + max(t.branch_layers for t in self.cfg.tasks) + 1
+        groups = (_I32 * cap)()
+        _check(lib().mt_plan_summary(self.handle, task_mask, C.byref(n_layers), C.byref(n_waves), C.byref(depth),
+                                     groups), "mt_plan_summary", self.handle)
+        return {"layers": n_layers.value, "waves": n_waves.value, "trunk_depth": depth.value,
+                "groups_per_wave": list(groups[:n_waves.value])}
+
+    def plan_launches(self, task_mask: int) -> int:
+        n = _I32()
+        _check(lib().mt_plan_launches(self.handle, task_mask, C.byref(n)), "mt_plan_launches", self.handle)
+        return n.value
+
+    # -- device -------------------------------------------------------------
+    def bind(self, device: str = "cuda:0") -> None:
+        import torch
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.weights = torch.empty(self.weights_bytes(), dtype=torch.uint8, device=self.device)
+        self.workspace = torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
+        _check(lib().mt_bind_memory(self.handle, self.weights.data_ptr(), self.weights.numel(),
+                                    self.workspace.data_ptr(), self.workspace.numel()), "mt_bind_memory", self.handle)
+
+    def load_weights(self, blob, stream=None) -> None:
+        """``blob``: numpy uint8 array or torch CPU uint8 tensor (pinned for an asynchronous copy)."""
+        import torch
+        t = blob if isinstance(blob, torch.Tensor) else torch.from_numpy(blob)
+        _check(lib().mt_load_weights(self.handle, t.data_ptr(), t.numel(), _stream(stream)), "mt_load_weights",
+               self.handle)
+        torch.cuda.current_stream().synchronize()
+
+    def load_task_weights(self, task: int, blob, stream=None) -> None:
+        import torch
+        t = blob if isinstance(blob, torch.Tensor) else torch.from_numpy(blob)
+        _check(lib().mt_load_task_weights(self.handle, task, t.data_ptr(), t.numel(), _stream(stream)),
+               "mt_load_task_weights", self.handle)
+        torch.cuda.current_stream().synchronize()
+
+    def full_mask(self) -> int:
+        return (1 << self.cfg.n_tasks) - 1
+
+    def forward(self, token_ids, segment_ids, lengths, logits, task_mask: Optional[int] = None, stream=None) -> None:
+        """Device int32 tensors in, fp32 ``logits`` [B, C_total] written in place.  Asynchronous."""
+        batch, seq = token_ids.shape
+        mask = self.full_mask() if task_mask is None else task_mask
+        _check(lib().mt_forward(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
+                                _ptr(logits), _stream(stream)), "mt_forward", self.handle)
+
+    def forward_host(self, token_ids, segment_ids, lengths, logits, task_mask: Optional[int] = None,
+                     stream=None) -> None:
+        """Host (ideally pinned) int32 tensors in, host fp32 ``logits`` out; returns after the copy back."""
+        batch, seq = token_ids.shape
+        mask = self.full_mask() if task_mask is None else task_mask
+        _check(lib().mt_forward_host(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
+                                     _ptr(logits), _stream(stream)), "mt_forward_host", self.handle)
+
+    def poll_status(self, stream=None) -> int:
+        flags = C.c_uint32(0)
+        rc = lib().mt_poll_status(self.handle, _stream(stream), C.byref(flags))
+        if rc not in (MT_OK, -8):
+            _check(rc, "mt_poll_status", self.handle)
+        return flags.value
+
+    def debug_hidden(self, task: int, layer: int, batch: int, seq: int):
+        import torch
+        out = torch.empty(batch * seq, self.cfg.hidden, dtype=torch.bfloat16, device=self.device)
+        _check(lib().mt_debug_copy_hidden(self.handle, task, layer, out.data_ptr(), _stream()), "mt_debug_copy_hidden",
+               self.handle)
+        return out
+
+    def close(self) -> None:
+        if self.handle:
+            lib().mt_destroy(self.handle)
+            self.handle = _P()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,253 @@
+// Fused masked self-attention of the encoder layer:
+//   ctx[i, head] = softmax_j( q_i . k_j / sqrt(64),  j < length ) . V        per (sequence, head)
+// from the packed projection qkv[B*S, 3H] = [Q | K | V].  Keys at positions >= length get weight
+// exactly 0 (their K/V rows are never read: zero-filled in shared memory), query rows >= length
+// are written as 0, so padded rows stay finite and deterministic whatever they contained.
+//
+// One CTA = 64 query rows of one (group, sequence, head); 4 warps x 16 rows.  Keys are visited in
+// tiles of 64 with an online softmax (running row maximum and sum in fp32, reduced across the four
+// lanes that share a row with warp shuffles).  Q, K, V tiles are staged in shared memory with
+// 16-byte cp.async copies into an XOR-swizzled layout and fed to the tensor cores through ldmatrix
+// (mma.sync m16n8k16, bf16 inputs, fp32 accumulate); the probabilities are rounded to bf16 for the
+// second product.  Several layers of one wave are the groups of a single launch.
+
+#include "mt_kernels.h"
+
+namespace mt {
+namespace {
+
+constexpr int kAttnThreads = 128;
+constexpr int kTileQ = 64;
+constexpr int kTileK = 64;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// 16-byte async copy; copies nothing and zero-fills when !valid.
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
+  const int bytes = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// A tile is 64 rows x 64 bf16 (128 bytes = eight 16-byte chunks per row); chunk c of row r lives at
+// chunk position c ^ (r & 7), which makes both the row-wise cp.async writes and the 8-row ldmatrix
+// reads free of bank conflicts.
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  return static_cast<uint32_t>(row * 128 + ((chunk ^ (row & 7)) << 4));
+}
+
+// Loads rows [row0, row0+64) x 64 columns starting at `col0` of a [*, ld] bf16 matrix; rows >= limit zero.
+__device__ __forceinline__ void load_tile(uint32_t smem_tile, const bf16* base, int ld, int row0, int limit, int tid) {
+#pragma unroll
+  for (int i = 0; i < (kTileK * 8) / kAttnThreads; ++i) {
+    const int idx = tid + i * kAttnThreads;
+    const int r = idx >> 3;
+    const int c = idx & 7;
+    const bool valid = (row0 + r) < limit;
+    const bf16* src = base + static_cast<size_t>(valid ? row0 + r : 0) * ld + c * 8;
+    cp_async_16(smem_tile + tile_off(r, c), src, valid);
+  }
+}
+
+__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams p) {
+  __shared__ __align__(128) uint8_t smem[3 * kTileQ * 128];
+  const uint32_t sQ = smem_u32(smem);
+  const uint32_t sK = sQ + kTileQ * 128;
+  const uint32_t sV = sK + kTileK * 128;
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int lane = tid & 31;
+  const int q0 = blockIdx.x * kTileQ;
+  const int head = blockIdx.y;
+  const int g = blockIdx.z / p.batch;
+  const int b = blockIdx.z - g * p.batch;
+  const int H = p.heads * kHeadDim;
+  const int ld = 3 * H;
+
+  int len = p.lengths[b];
+  len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
+
+  const bf16* qkv = p.qkv[g] + static_cast<size_t>(b) * p.seq * ld + head * kHeadDim;
+  bf16* ctx = p.ctx[g] + static_cast<size_t>(b) * p.seq * H + head * kHeadDim;
+  const int rows_here = min(kTileQ, p.seq - q0);
+
+  if (q0 >= len) {
+    // the whole query tile is padding: write zeros
+    for (int idx = tid; idx < rows_here * 8; idx += kAttnThreads) {
+      const int r = idx >> 3, c = idx & 7;
+      *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(q0 + r) * H + c * 8) = make_uint4(0, 0, 0, 0);
+    }
+    return;
+  }
+
+  load_tile(sQ, qkv, ld, q0, len, tid);
+  cp_async_commit();
+
+  float o[8][4];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+  uint32_t qf[4][4];
+  // scores are scaled by 1/sqrt(64) and moved to base 2 for exp2f
+  const float scale_log2 = 0.125f * 1.4426950408889634f;
+
+  const int n_key_tiles = (len + kTileK - 1) / kTileK;
+  for (int kt = 0; kt < n_key_tiles; ++kt) {
+    const int k0 = kt * kTileK;
+    if (kt > 0) __syncthreads();  // everyone is done reading the previous K/V tile
+    load_tile(sK, qkv + H, ld, k0, len, tid);
+    load_tile(sV, qkv + 2 * H, ld, k0, len, tid);
+    cp_async_commit();
+    cp_async_wait_all();
+    __syncthreads();
+
+    if (kt == 0) {
+      // Q fragments: 16 rows of this warp x 64 dims = four k-steps of 16
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        const int r = warp * 16 + (lane & 15);
+        const int c = ks * 2 + (lane >> 4);
+        ldmatrix_x4(sQ + tile_off(r, c), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+      }
+    }
+
+    // S = Q K^T : 16 x 64 per warp = eight n-tiles of 8 keys
+    float s[8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        // four 8x8 blocks of K rows (keys n*8..n*8+7), dims half*32 + {0,8,16,24}
+        uint32_t k0r, k1r, k2r, k3r;
+        const int r = n * 8 + (lane & 7);
+        const int c = half * 4 + (lane >> 3);
+        ldmatrix_x4(sK + tile_off(r, c), k0r, k1r, k2r, k3r);
+        mma_bf16_16816(s[n], qf[half * 2], k0r, k1r);
+        mma_bf16_16816(s[n], qf[half * 2 + 1], k2r, k3r);
+      }
+    }
+
+    // mask keys >= len, online softmax.  Thread holds rows (lane/4) and (lane/4 + 8);
+    // columns n*8 + 2*(lane%4) + {0,1}.
+    float m_new[2] = {m_run[0], m_run[1]};
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const int key = k0 + n * 8 + 2 * (lane & 3);
+      if (key >= len) { s[n][0] = -INFINITY; s[n][2] = -INFINITY; }
+      if (key + 1 >= len) { s[n][1] = -INFINITY; s[n][3] = -INFINITY; }
+      m_new[0] = fmaxf(m_new[0], fmaxf(s[n][0], s[n][1]));
+      m_new[1] = fmaxf(m_new[1], fmaxf(s[n][2], s[n][3]));
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      m_new[r] = fmaxf(m_new[r], __shfl_xor_sync(0xffffffffu, m_new[r], 1));
+      m_new[r] = fmaxf(m_new[r], __shfl_xor_sync(0xffffffffu, m_new[r], 2));
+    }
+    // key 0 of the first tile is always valid (len >= 1), so m_new is finite from the first tile on
+    float corr[2], sum[2] = {0.f, 0.f};
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      corr[r] = exp2f((m_run[r] - m_new[r]) * scale_log2);
+      m_run[r] = m_new[r];
+    }
+    uint32_t pf[4][4];  // probabilities as A fragments: four k-steps of 16 keys
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const float p0 = exp2f((s[n][0] - m_new[0]) * scale_log2);
+      const float p1 = exp2f((s[n][1] - m_new[0]) * scale_log2);
+      const float p2 = exp2f((s[n][2] - m_new[1]) * scale_log2);
+      const float p3 = exp2f((s[n][3] - m_new[1]) * scale_log2);
+      sum[0] += p0 + p1;
+      sum[1] += p2 + p3;
+      pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] * corr[r] + sum[r];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      o[n][0] *= corr[0]; o[n][1] *= corr[0];
+      o[n][2] *= corr[1]; o[n][3] *= corr[1];
+    }
+
+    // O += P V : k = keys (four steps of 16), n = 64 dims (eight n-tiles)
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        // V rows ks*16 .. +15, dims np*16 .. +15, transposed on load
+        uint32_t v0, v1, v2, v3;
+        const int r = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int c = np * 2 + (lane >> 4);
+        ldmatrix_x4_trans(sV + tile_off(r, c), v0, v1, v2, v3);
+        mma_bf16_16816(o[np * 2], pf[ks], v0, v1);
+        mma_bf16_16816(o[np * 2 + 1], pf[ks], v2, v3);
+      }
+    }
+  }
+
+  // row sums across the four lanes of a row, normalise, stage in this warp's rows of the Q tile
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+  }
+  const float inv0 = 1.f / l_run[0];
+  const float inv1 = 1.f / l_run[1];
+  __syncwarp();
+  uint8_t* sQg = smem;
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const int r0 = warp * 16 + (lane >> 2);
+    const int byte_in_chunk = (lane & 3) * 4;
+    *reinterpret_cast<uint32_t*>(sQg + tile_off(r0, n) + byte_in_chunk) = pack_bf16(o[n][0] * inv0, o[n][1] * inv0);
+    *reinterpret_cast<uint32_t*>(sQg + tile_off(r0 + 8, n) + byte_in_chunk) = pack_bf16(o[n][2] * inv1, o[n][3] * inv1);
+  }
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int idx = lane + i * 32;   // 16 rows x 8 chunks
+    const int r = warp * 16 + (idx >> 3);
+    const int c = idx & 7;
+    if (r < rows_here) {
+      uint4 val = *reinterpret_cast<const uint4*>(sQg + tile_off(r, c));
+      if (q0 + r >= len) val = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(q0 + r) * H + c * 8) = val;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1) return cudaErrorInvalidValue;
+  dim3 grid((p.seq + kTileQ - 1) / kTileQ, p.heads, p.batch * p.n_groups);
+  attention_kernel<<<grid, kAttnThreads, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace mt

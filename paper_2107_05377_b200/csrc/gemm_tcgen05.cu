@@ -1,0 +1,404 @@
+// Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   Y_g[M,N] = epilogue( X_g[M,K] . W_g[N,K]^T + bias_g )        g = 0 .. n_groups-1
+//
+// These are the linear maps of the encoder layer (QKV, attention output, FFN up, FFN down).
+// The layers that are ready in the same wave of the task tree (the trunk layer and the branch
+// layers of several tasks) are the groups of ONE launch, so their tiles fill the machine together.
+//
+// One persistent CTA per SM walks over the tiles (128 x BN) of all groups.  Warp roles:
+//   warp 0      : TMA producer - streams 128x64 X tiles and BNx64 W tiles (128-byte swizzle) into
+//                 a ring of shared-memory stages, signalling "full" mbarriers by transaction count
+//   warp 1      : allocates tensor memory; one thread issues tcgen05.mma (128 x BN x 16 per
+//                 instruction) with the accumulator in TMEM, and tcgen05.commit to release stages
+//   warps 2..   : epilogue - tcgen05.ld the fp32 accumulator (each warp its own 32-lane quarter),
+//                 add bias (+GELU or +residual), round once to bf16, 16-byte stores
+// The accumulator is double buffered in TMEM (2 x BN columns) so the epilogue of tile i overlaps
+// the MMAs of tile i+1.  Every output element is the sum over K in a fixed order inside a single
+// tile, so a result never depends on which other groups share the launch.
+//
+// Every mbarrier wait is bounded: after kWaitLimitNs the waiting thread raises the CTA's abort
+// flag, the status word gets kFlagWaitTimeout, all roles leave their loops, the producer drains
+// the copies it still has in flight, TMEM is freed and the CTA returns.
+
+#include "mt_kernels.h"
+
+namespace mt {
+namespace {
+
+constexpr int kNumEpilogueWarps = 8;
+constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s
+
+__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 256 ? 4 : 6; }
+__host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
+__host__ __device__ constexpr int gemm_b_bytes(int bn) { return bn * kGemmBlockK * 2; }
+__host__ __device__ constexpr int gemm_smem_bytes(int bn) {
+  // stages + barriers/bookkeeping + slack for manual 1024-byte alignment
+  return gemm_stages(bn) * (gemm_a_bytes() + gemm_b_bytes(bn)) + 256 + 1024;
+}
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false once the CTA is aborting (this thread's limit ran out, or another
+// role raised the flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xFFu) == 0xFFu) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] . B[smem]^T, 128 x N x 16, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier gets one arrival when all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives lane (quarter*32 + t).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16), stored
+// with the 128-byte swizzle exactly as TMA writes it: start address >> 4 in bits [0,14); leading
+// byte offset (unused for swizzled K-major) = 1 in [16,30); stride byte offset = 1024 B (eight
+// rows) >> 4 in [32,46); descriptor version 1 in [46,48); layout type 2 (128-byte swizzle) in [61,64).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
+  uint64_t d = static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: D fp32 (bits [4,6) = 1), A and B bf16 ([7,10) = [10,13) = 1),
+// both K-major (bits 15, 16 = 0), N >> 3 in [17,23), M >> 4 in [24,29).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+// ---- the kernel -------------------------------------------------------------------------------
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __grid_constant__ GemmParams p) {
+  constexpr int STAGES = gemm_stages(BN);
+  constexpr int A_BYTES = gemm_a_bytes();
+  constexpr int B_BYTES = gemm_b_bytes(BN);
+  constexpr uint32_t TMEM_COLS = 2 * BN;  // 256 or 512: a power of two >= 32
+  static_assert(BN == 128 || BN == 256, "tile widths implemented: 128, 256");
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sA = smem_u32(smem);
+  const uint32_t sB = sA + STAGES * A_BYTES;
+  uint8_t* book = smem + STAGES * (A_BYTES + B_BYTES);
+  const uint32_t bar_full = smem_u32(book);               // STAGES x 8 bytes
+  const uint32_t bar_empty = bar_full + 8 * STAGES;       // STAGES x 8 bytes
+  const uint32_t bar_acc_full = bar_empty + 8 * STAGES;   // 2 x 8 bytes
+  const uint32_t bar_acc_empty = bar_acc_full + 16;       // 2 x 8 bytes
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(book + 8 * (2 * STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  const int n_tiles_n = p.N / BN;
+  const int n_tiles_m = (p.M + kGemmBlockM - 1) / kGemmBlockM;
+  const int tiles_per_group = n_tiles_m * n_tiles_n;
+  const int total_tiles = tiles_per_group * p.n_groups;
+  const int k_blocks = p.K / kGemmBlockK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_acc_full + 8 * a, 1);
+      mbar_init(bar_acc_empty + 8 * a, kNumEpilogueWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int g = tile / tiles_per_group;
+        const int local = tile - g * tiles_per_group;
+        const int m0 = (local / n_tiles_n) * kGemmBlockM;
+        const int n0 = (local % n_tiles_n) * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(bar_full + 8 * stage, A_BYTES + B_BYTES);
+          tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+          tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Aborting: wait (bounded) until the copies still in flight have landed, so that the
+        // CTA does not retire underneath them.  The last min(issued, STAGES) fills are the ones
+        // that may be pending; walk back over them.
+        int s = stage;
+        uint32_t ph = phase;
+        const int pending = issued < STAGES ? static_cast<int>(issued) : STAGES;
+        for (int i = 0; i < pending; ++i) {
+          if (s == 0) { s = STAGES; ph ^= 1u; }
+          --s;
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(bar_full + 8 * s, ph)) {
+            if (global_timer_ns() - t0 > kWaitLimitNs) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kGemmBlockM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = smem_desc_sw128(sA + stage * A_BYTES);
+          const uint64_t db = smem_desc_sw128(sB + stage * B_BYTES);
+#pragma unroll
+          for (int k = 0; k < kGemmBlockK / 16; ++k) {
+            // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the address field
+            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(bar_empty + 8 * stage);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(bar_acc_full + 8 * acc);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ----------------------------------
+    const int e = warp - 2;
+    const int quarter = warp & 3;                       // TMEM lanes this warp may read
+    const int col_group = e >> 2;                       // which share of the column chunks
+    constexpr int COL_GROUPS = kNumEpilogueWarps / 4;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int g = tile / tiles_per_group;
+      const int local = tile - g * tiles_per_group;
+      const int m0 = (local / n_tiles_n) * kGemmBlockM;
+      const int n0 = (local % n_tiles_n) * BN;
+      if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag)) break;
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      const GemmGroup grp = p.group[g];
+      const size_t row_off = static_cast<size_t>(row) * p.N;
+#pragma unroll 1
+      for (int chunk = col_group; chunk < BN / 32; chunk += COL_GROUPS) {
+        uint32_t v[32];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                               static_cast<uint32_t>(acc * BN + chunk * 32);
+        tmem_ld_32x32(taddr, v);
+        tmem_ld_wait();
+        const int col = n0 + chunk * 32;
+        const uint4* bias4 = reinterpret_cast<const uint4*>(grp.bias + col);
+        uint4 outv[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 b = __ldg(bias4 + q);
+          const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+          uint4 r = make_uint4(0, 0, 0, 0);
+          if (EPI == kEpiBiasResidual && row_ok) {
+            r = *reinterpret_cast<const uint4*>(grp.residual + row_off + col + q * 8);
+          }
+          const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+          uint32_t ow[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
+            float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
+            if (EPI == kEpiBiasGelu) {
+              x0 = gelu_erf(x0);
+              x1 = gelu_erf(x1);
+            }
+            if (EPI == kEpiBiasResidual) {
+              x0 += bf16_lo(rw[j]);
+              x1 += bf16_hi(rw[j]);
+            }
+            ow[j] = pack_bf16(x0, x1);
+          }
+          outv[q] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        }
+        if (row_ok) {
+          uint4* dst = reinterpret_cast<uint4*>(grp.out + row_off + col);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) dst[q] = outv[q];
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------ teardown ------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicOr(p.status, kFlagWaitTimeout);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int BN, int EPI>
+cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
+  auto kernel = gemm_bf16_tcgen05<BN, EPI>;
+  static bool configured = false;  // per instantiation; the attribute is per function and per device
+  static int configured_device = -1;
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (!configured || configured_device != dev) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN));
+    if (err != cudaSuccess) return err;
+    configured = true;
+    configured_device = dev;
+  }
+  const int tiles = ((p.M + kGemmBlockM - 1) / kGemmBlockM) * (p.N / BN) * p.n_groups;
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  if (grid <= 0) return cudaSuccess;
+  kernel<<<grid, kGemmThreads, gemm_smem_bytes(BN), stream>>>(p);
+  return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
+  switch (epilogue) {
+    case kEpiBias: return launch_one<BN, kEpiBias>(p, sm_count, stream);
+    case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu>(p, sm_count, stream);
+    case kEpiBiasResidual: return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace
+
+int gemm_block_n(int N) { return (N % 256 == 0 && N >= 2048) ? 256 : 128; }
+
+cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
+    return cudaErrorInvalidValue;
+  return gemm_block_n(p.N) == 256 ? launch_bn<256>(p, epilogue, sm_count, stream)
+                                  : launch_bn<128>(p, epilogue, sm_count, stream);
+}
+
+}  // namespace mt

@@ -1,0 +1,799 @@
+// C-ABI boundary, weight arena and tree scheduler of the merged multi-task forward pass.
+//
+// Model merging (paper Section 3.3) = one weight arena holding the shared trunk once and every
+// task's own layers, plus a static schedule over the resulting tree: wave w runs trunk layer w
+// together with every branch layer whose input is ready (branch layer j of a task that forks at
+// depth d runs in wave d + j), all as groups of the same kernel launches.  The trunk state at a
+// fork depth stays resident until the wave after it has consumed it (two ping-pong trunk buffers
+// are enough because every reader of depth d runs in wave d + 1); tasks masked off by task_mask
+// contribute no branch, no head, and do not extend the trunk depth.
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/mt_bert.h"
+#include "mt_kernels.h"
+
+using namespace mt;
+
+namespace {
+
+constexpr uint32_t kBlobMagic = 0x4D544257u;
+constexpr uint32_t kBlobVersion = 1u;
+constexpr size_t kAlign = 256;
+constexpr size_t kHeaderBytes = 256;
+
+inline size_t pad256(size_t n) { return (n + kAlign - 1) / kAlign * kAlign; }
+
+// Offsets (bytes from the start of the arena = start of the blob payload) of one layer's tensors.
+struct LayerOffsets {
+  size_t wq, wk, wv, bq, bk, bv, wo, bo, ln1_g, ln1_b, w1, b1, w2, b2, ln2_g, ln2_b;
+};
+
+struct TaskEntry {
+  mt_task_config cfg;
+  std::vector<LayerOffsets> layers;
+  size_t pool_w, pool_b, cls_w, cls_b;
+  size_t section_begin, section_bytes;
+  int32_t col0;
+  bool loaded;
+};
+
+struct BlobHeader {
+  uint32_t magic, version, kind;
+  int32_t hidden, heads, ffn, trunk_layers, vocab, max_position, type_vocab;
+  int32_t n_tasks, task_index, fork_depth, branch_layers, num_classes, reserved;
+  uint64_t payload_bytes;
+};
+
+// ---- logical schedule (no device pointers) -----------------------------------------------------
+
+struct OpDesc {
+  int32_t task;   // -1 = trunk
+  int32_t layer;  // trunk: depth produced (1..D); branch: 1..k_t
+};
+struct Schedule {
+  int32_t trunk_depth = 0;
+  int32_t n_layers = 0;
+  std::vector<std::vector<OpDesc>> waves;       // waves[w-1] = layers of wave w
+  std::vector<std::vector<int32_t>> heads;      // heads[w] = tasks whose head runs after wave w (0 = after embedding)
+};
+
+// ---- bound plan (device pointers, tensor maps) --------------------------------------------------
+
+struct Chunk {
+  GemmParams qkv, attn_out, ffn_up, ffn_down;
+  AttnParams attn;
+  LayerNormParams ln1, ln2;
+  std::vector<std::pair<const bf16*, int32_t>> dumps;  // (layer output, dump slot)
+};
+struct PlanStep {
+  int kind;  // 0 = chunk, 1 = heads
+  Chunk chunk;
+  HeadParams heads;
+};
+struct Plan {
+  std::vector<PlanStep> steps;
+  int32_t launches = 0;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_driver_mutex;
+EncodeTiledFn g_encode = nullptr;
+
+cudaError_t get_encoder(EncodeTiledFn* out) {
+  std::lock_guard<std::mutex> lock(g_driver_mutex);
+  if (g_encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (err != cudaSuccess) return err;
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = g_encode;
+  return cudaSuccess;
+}
+
+// Tensor map of a row-major bf16 matrix [rows, cols] read in boxes of box_rows x 64 columns with
+// the 128-byte swizzle; out-of-range rows read as zero.
+cudaError_t make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn enc = nullptr;
+  cudaError_t err = get_encoder(&enc);
+  if (err != cudaSuccess) return err;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * sizeof(bf16)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kGemmBlockK), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t elem[2] = {1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+struct mt_model {
+  mt_trunk_config trunk;
+  std::vector<TaskEntry> tasks;
+  int32_t max_batch, max_seq, c_total;
+
+  // arena
+  size_t emb_word, emb_pos, emb_type, emb_ln_g, emb_ln_b;
+  std::vector<LayerOffsets> trunk_layers;
+  size_t weights_bytes;
+  bool trunk_loaded;
+
+  // options
+  int32_t max_groups;
+  bool debug_capture;
+
+  // device memory (caller-owned)
+  uint8_t* d_weights;
+  uint8_t* d_workspace;
+  size_t ws_bytes_bound;
+  int sm_count;
+
+  // workspace layout (byte offsets)
+  size_t ws_status, ws_tok, ws_seg, ws_len, ws_logits, ws_trunk[2], ws_task0, ws_slot0, ws_dump0;
+  size_t act_bytes;   // max_batch*max_seq*hidden*2
+  size_t slot_bytes;
+  int32_t n_slots, n_dump;
+  size_t ws_total;
+
+  std::map<std::tuple<uint64_t, int32_t, int32_t>, Plan> plans;
+  int32_t last_batch, last_seq;
+  std::string last_error;
+};
+
+namespace {
+
+int fail(const mt_model* m, int code, const std::string& msg) {
+  if (m != nullptr) const_cast<mt_model*>(m)->last_error = msg;
+  return code;
+}
+int fail_cuda(const mt_model* m, cudaError_t e, const char* what) {
+  return fail(m, MT_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+size_t place_layer(const mt_trunk_config& c, size_t off, LayerOffsets* lo) {
+  const size_t H = c.hidden, F = c.ffn, e = sizeof(bf16);
+  auto take = [&](size_t elems) { size_t at = off; off += pad256(elems * e); return at; };
+  lo->wq = take(H * H); lo->wk = take(H * H); lo->wv = take(H * H);
+  lo->bq = take(H); lo->bk = take(H); lo->bv = take(H);
+  lo->wo = take(H * H); lo->bo = take(H);
+  lo->ln1_g = take(H); lo->ln1_b = take(H);
+  lo->w1 = take(F * H); lo->b1 = take(F);
+  lo->w2 = take(H * F); lo->b2 = take(H);
+  lo->ln2_g = take(H); lo->ln2_b = take(H);
+  return off;
+}
+
+void layout_workspace(mt_model* m) {
+  const size_t M = static_cast<size_t>(m->max_batch) * m->max_seq;
+  const size_t H = m->trunk.hidden, F = m->trunk.ffn;
+  m->act_bytes = pad256(M * H * sizeof(bf16));
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off += pad256(bytes); return at; };
+  m->ws_status = take(256);
+  m->ws_tok = take(M * 4);
+  m->ws_seg = take(M * 4);
+  m->ws_len = take(static_cast<size_t>(m->max_batch) * 4);
+  m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
+  m->ws_trunk[0] = take(m->act_bytes);
+  m->ws_trunk[1] = take(m->act_bytes);
+  m->ws_task0 = off;
+  off += m->act_bytes * m->tasks.size();
+  m->n_slots = std::min<int32_t>(m->max_groups, static_cast<int32_t>(m->tasks.size()) + 1);
+  // slot = qkv [M,3H] + ctx [M,H] + u [M,H] + h1 [M,H] + f [M,F]
+  m->slot_bytes = pad256(M * 3 * H * 2) + 3 * m->act_bytes + pad256(M * F * 2);
+  m->ws_slot0 = off;
+  off += m->slot_bytes * m->n_slots;
+  m->n_dump = 0;
+  m->ws_dump0 = off;
+  if (m->debug_capture) {
+    m->n_dump = m->trunk.trunk_layers + 1;
+    for (const TaskEntry& t : m->tasks) m->n_dump += t.cfg.branch_layers;
+    off += m->act_bytes * m->n_dump;
+  }
+  m->ws_total = off;
+}
+
+int32_t dump_slot(const mt_model* m, int32_t task, int32_t layer) {
+  if (task < 0) return layer;  // 0..trunk_layers
+  int32_t idx = m->trunk.trunk_layers + 1;
+  for (int32_t t = 0; t < task; ++t) idx += m->tasks[t].cfg.branch_layers;
+  return idx + layer - 1;
+}
+
+bool build_schedule(const mt_model* m, uint64_t mask, Schedule* s) {
+  const int32_t T = static_cast<int32_t>(m->tasks.size());
+  if (T < 64) mask &= (uint64_t(1) << T) - 1;
+  if (mask == 0) return false;
+  int32_t depth = 0, last_wave = 0, layers = 0;
+  for (int32_t t = 0; t < T; ++t) {
+    if (!((mask >> t) & 1)) continue;
+    const mt_task_config& c = m->tasks[t].cfg;
+    depth = std::max(depth, c.fork_depth);
+    last_wave = std::max(last_wave, c.fork_depth + c.branch_layers);
+    layers += c.branch_layers;
+  }
+  s->trunk_depth = depth;
+  s->n_layers = depth + layers;
+  s->waves.assign(last_wave, {});
+  s->heads.assign(last_wave + 1, {});
+  for (int32_t w = 1; w <= last_wave; ++w) {
+    if (w <= depth) s->waves[w - 1].push_back({-1, w});
+    for (int32_t t = 0; t < T; ++t) {
+      if (!((mask >> t) & 1)) continue;
+      const mt_task_config& c = m->tasks[t].cfg;
+      const int32_t j = w - c.fork_depth;
+      if (j >= 1 && j <= c.branch_layers) s->waves[w - 1].push_back({t, j});
+    }
+  }
+  for (int32_t t = 0; t < T; ++t) {
+    if (!((mask >> t) & 1)) continue;
+    const mt_task_config& c = m->tasks[t].cfg;
+    s->heads[c.fork_depth + c.branch_layers].push_back(t);
+  }
+  return true;
+}
+
+bf16* ws_ptr(const mt_model* m, size_t off) { return reinterpret_cast<bf16*>(m->d_workspace + off); }
+const bf16* w_ptr(const mt_model* m, size_t off) { return reinterpret_cast<const bf16*>(m->d_weights + off); }
+
+// Where the state of a stream lives: trunk depth d in ping-pong buffer d & 1, a task in its own buffer.
+bf16* trunk_buf(const mt_model* m, int32_t depth) { return ws_ptr(m, m->ws_trunk[depth & 1]); }
+bf16* task_buf(const mt_model* m, int32_t task) { return ws_ptr(m, m->ws_task0 + m->act_bytes * task); }
+
+cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int32_t batch,
+                        int32_t seq, Chunk* ck) {
+  const int32_t M = batch * seq, H = m->trunk.hidden, F = m->trunk.ffn;
+  const size_t act = m->act_bytes;
+  const size_t qkv_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * 3 * H * 2);
+  auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K) {
+    memset(g, 0, sizeof(*g));
+    g->n_groups = static_cast<int32_t>(count);
+    g->M = M; g->N = N; g->K = K;
+    g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
+  };
+  init_gemm(&ck->qkv, 3 * H, H);
+  init_gemm(&ck->attn_out, H, H);
+  init_gemm(&ck->ffn_up, F, H);
+  init_gemm(&ck->ffn_down, H, F);
+  memset(&ck->attn, 0, sizeof(ck->attn));
+  memset(&ck->ln1, 0, sizeof(ck->ln1));
+  memset(&ck->ln2, 0, sizeof(ck->ln2));
+  ck->attn.n_groups = ck->ln1.n_groups = ck->ln2.n_groups = static_cast<int32_t>(count);
+  ck->attn.batch = batch; ck->attn.seq = seq; ck->attn.heads = m->trunk.heads;
+  ck->attn.lengths = nullptr;  // patched per call
+  ck->ln1.rows = ck->ln2.rows = M;
+  ck->ln1.hidden = ck->ln2.hidden = H;
+  ck->ln1.eps = ck->ln2.eps = m->trunk.ln_eps;
+
+  for (size_t i = 0; i < count; ++i) {
+    const OpDesc& op = ops[first + i];
+    const LayerOffsets* lo;
+    bf16 *in, *out;
+    if (op.task < 0) {
+      lo = &m->trunk_layers[op.layer - 1];
+      in = trunk_buf(m, op.layer - 1);
+      out = trunk_buf(m, op.layer);
+    } else {
+      const TaskEntry& te = m->tasks[op.task];
+      lo = &te.layers[op.layer - 1];
+      in = op.layer == 1 ? trunk_buf(m, te.cfg.fork_depth) : task_buf(m, op.task);
+      out = task_buf(m, op.task);
+    }
+    uint8_t* slot = m->d_workspace + m->ws_slot0 + m->slot_bytes * i;
+    bf16* qkv = reinterpret_cast<bf16*>(slot);
+    bf16* ctx = reinterpret_cast<bf16*>(slot + qkv_bytes);
+    bf16* u = reinterpret_cast<bf16*>(slot + qkv_bytes + act);
+    bf16* h1 = reinterpret_cast<bf16*>(slot + qkv_bytes + 2 * act);
+    bf16* f = reinterpret_cast<bf16*>(slot + qkv_bytes + 3 * act);
+
+    cudaError_t e;
+    // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv]   (the three matrices and biases are contiguous in the arena)
+    if ((e = make_tmap(&ck->qkv.tmap_x[i], in, M, H, kGemmBlockM)) != cudaSuccess) return e;
+    if ((e = make_tmap(&ck->qkv.tmap_w[i], w_ptr(m, lo->wq), 3 * H, H, gemm_block_n(3 * H))) != cudaSuccess) return e;
+    ck->qkv.group[i] = {w_ptr(m, lo->bq), nullptr, qkv};
+    // 2. ctx = attention(qkv)
+    ck->attn.qkv[i] = qkv;
+    ck->attn.ctx[i] = ctx;
+    // 3. u = ctx . Wo^T + bo + in
+    if ((e = make_tmap(&ck->attn_out.tmap_x[i], ctx, M, H, kGemmBlockM)) != cudaSuccess) return e;
+    if ((e = make_tmap(&ck->attn_out.tmap_w[i], w_ptr(m, lo->wo), H, H, gemm_block_n(H))) != cudaSuccess) return e;
+    ck->attn_out.group[i] = {w_ptr(m, lo->bo), in, u};
+    // 4. h1 = LN(u)
+    ck->ln1.x[i] = u; ck->ln1.gamma[i] = w_ptr(m, lo->ln1_g); ck->ln1.beta[i] = w_ptr(m, lo->ln1_b); ck->ln1.y[i] = h1;
+    // 5. f = GELU(h1 . W1^T + b1)
+    if ((e = make_tmap(&ck->ffn_up.tmap_x[i], h1, M, H, kGemmBlockM)) != cudaSuccess) return e;
+    if ((e = make_tmap(&ck->ffn_up.tmap_w[i], w_ptr(m, lo->w1), F, H, gemm_block_n(F))) != cudaSuccess) return e;
+    ck->ffn_up.group[i] = {w_ptr(m, lo->b1), nullptr, f};
+    // 6. u = f . W2^T + b2 + h1
+    if ((e = make_tmap(&ck->ffn_down.tmap_x[i], f, M, F, kGemmBlockM)) != cudaSuccess) return e;
+    if ((e = make_tmap(&ck->ffn_down.tmap_w[i], w_ptr(m, lo->w2), H, F, gemm_block_n(H))) != cudaSuccess) return e;
+    ck->ffn_down.group[i] = {w_ptr(m, lo->b2), h1, u};
+    // 7. out = LN(u)
+    ck->ln2.x[i] = u; ck->ln2.gamma[i] = w_ptr(m, lo->ln2_g); ck->ln2.beta[i] = w_ptr(m, lo->ln2_b); ck->ln2.y[i] = out;
+
+    if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer)});
+  }
+  return cudaSuccess;
+}
+
+cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
+  plan->steps.clear();
+  plan->launches = 1;  // embedding
+  auto add_heads = [&](const std::vector<int32_t>& tasks) {
+    for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
+      const size_t count = std::min<size_t>(kMaxGroups, tasks.size() - first);
+      PlanStep st;
+      st.kind = 1;
+      memset(&st.heads, 0, sizeof(st.heads));
+      st.heads.n_tasks = static_cast<int32_t>(count);
+      st.heads.batch = batch; st.heads.seq = seq; st.heads.hidden = m->trunk.hidden;
+      st.heads.logits_stride = m->c_total;
+      for (size_t i = 0; i < count; ++i) {
+        const int32_t t = tasks[first + i];
+        const TaskEntry& te = m->tasks[t];
+        HeadTask& ht = st.heads.task[i];
+        ht.hidden = te.cfg.branch_layers == 0 ? trunk_buf(m, te.cfg.fork_depth) : task_buf(m, t);
+        ht.pool_w = w_ptr(m, te.pool_w); ht.pool_b = w_ptr(m, te.pool_b);
+        ht.cls_w = w_ptr(m, te.cls_w); ht.cls_b = w_ptr(m, te.cls_b);
+        ht.num_classes = te.cfg.num_classes; ht.col0 = te.col0;
+      }
+      plan->steps.push_back(std::move(st));
+      plan->launches += 1;
+    }
+  };
+  add_heads(s.heads[0]);
+  for (size_t w = 1; w <= s.waves.size(); ++w) {
+    const std::vector<OpDesc>& ops = s.waves[w - 1];
+    for (size_t first = 0; first < ops.size(); first += m->n_slots) {
+      const size_t count = std::min<size_t>(m->n_slots, ops.size() - first);
+      PlanStep st;
+      st.kind = 0;
+      cudaError_t e = build_chunk(m, ops, first, count, batch, seq, &st.chunk);
+      if (e != cudaSuccess) return e;
+      plan->steps.push_back(std::move(st));
+      plan->launches += 7;
+    }
+    add_heads(s.heads[w]);
+  }
+  return cudaSuccess;
+}
+
+cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+
+extern "C" {
+
+int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t n_tasks, int32_t max_batch,
+              int32_t max_seq, mt_model** out) {
+  if (out == nullptr) return MT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (trunk == nullptr || tasks == nullptr || n_tasks < 1 || n_tasks > 64 || max_batch < 1 || max_seq < 1)
+    return MT_ERR_INVALID_ARG;
+  if (trunk->hidden != trunk->heads * kHeadDim || (trunk->hidden != 768 && trunk->hidden != 1024) ||
+      trunk->ffn % 256 != 0 || trunk->ffn < 256 || trunk->activation != 0 || max_seq > 512)
+    return MT_ERR_UNSUPPORTED;
+  if (trunk->vocab_size < 1 || trunk->type_vocab < 1 || trunk->trunk_layers < 0 || max_seq > trunk->max_position ||
+      !(trunk->ln_eps >= 0.f))
+    return MT_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(max_batch) * max_seq > (int64_t(1) << 24)) return MT_ERR_SHAPE;
+  for (int32_t t = 0; t < n_tasks; ++t) {
+    if (tasks[t].fork_depth < 0 || tasks[t].fork_depth > trunk->trunk_layers || tasks[t].branch_layers < 0 ||
+        tasks[t].num_classes < 1)
+      return MT_ERR_INVALID_ARG;
+  }
+  mt_model* m = new mt_model();
+  m->trunk = *trunk;
+  m->max_batch = max_batch;
+  m->max_seq = max_seq;
+  m->max_groups = kMaxGroups;
+  m->debug_capture = false;
+  m->d_weights = m->d_workspace = nullptr;
+  m->ws_bytes_bound = 0;
+  m->sm_count = 0;
+  m->trunk_loaded = false;
+  m->last_batch = m->last_seq = 0;
+
+  const size_t H = trunk->hidden, e = sizeof(bf16);
+  size_t off = 0;
+  auto take = [&](size_t elems) { size_t at = off; off += pad256(elems * e); return at; };
+  m->emb_word = take(static_cast<size_t>(trunk->vocab_size) * H);
+  m->emb_pos = take(static_cast<size_t>(trunk->max_position) * H);
+  m->emb_type = take(static_cast<size_t>(trunk->type_vocab) * H);
+  m->emb_ln_g = take(H);
+  m->emb_ln_b = take(H);
+  m->trunk_layers.resize(trunk->trunk_layers);
+  for (int32_t l = 0; l < trunk->trunk_layers; ++l) off = place_layer(*trunk, off, &m->trunk_layers[l]);
+  int32_t col = 0;
+  m->tasks.resize(n_tasks);
+  for (int32_t t = 0; t < n_tasks; ++t) {
+    TaskEntry& te = m->tasks[t];
+    te.cfg = tasks[t];
+    te.section_begin = off;
+    te.layers.resize(tasks[t].branch_layers);
+    for (int32_t j = 0; j < tasks[t].branch_layers; ++j) off = place_layer(*trunk, off, &te.layers[j]);
+    te.pool_w = take(H * H);
+    te.pool_b = take(H);
+    te.cls_w = take(static_cast<size_t>(tasks[t].num_classes) * H);
+    te.cls_b = take(tasks[t].num_classes);
+    te.section_bytes = off - te.section_begin;
+    te.col0 = col;
+    col += tasks[t].num_classes;
+    te.loaded = false;
+  }
+  m->weights_bytes = off;
+  m->c_total = col;
+  layout_workspace(m);
+  *out = m;
+  return MT_OK;
+}
+
+void mt_destroy(mt_model* m) { delete m; }
+
+size_t mt_weights_bytes(const mt_model* m) { return m ? m->weights_bytes : 0; }
+size_t mt_workspace_bytes(const mt_model* m) { return m ? m->ws_total : 0; }
+size_t mt_blob_bytes(const mt_model* m) { return m ? m->weights_bytes + kHeaderBytes : 0; }
+size_t mt_task_blob_bytes(const mt_model* m, int32_t task) {
+  if (m == nullptr || task < 0 || task >= static_cast<int32_t>(m->tasks.size())) return 0;
+  return m->tasks[task].section_bytes + kHeaderBytes;
+}
+
+const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c_str() : "null model"; }
+
+int mt_set_option(mt_model* m, const char* key, int64_t value) {
+  if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
+  if (m->d_workspace != nullptr) return fail(m, MT_ERR_INVALID_ARG, "options must be set before mt_bind_memory");
+  if (strcmp(key, "max_groups") == 0) {
+    if (value < 1 || value > kMaxGroups) return fail(m, MT_ERR_INVALID_ARG, "max_groups must be in 1..8");
+    m->max_groups = static_cast<int32_t>(value);
+  } else if (strcmp(key, "debug_capture") == 0) {
+    m->debug_capture = value != 0;
+  } else {
+    return fail(m, MT_ERR_INVALID_ARG, std::string("unknown option ") + key);
+  }
+  layout_workspace(m);
+  m->plans.clear();
+  return MT_OK;
+}
+
+int mt_bind_memory(mt_model* m, void* d_weights, size_t weights_bytes, void* d_workspace, size_t workspace_bytes) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (d_weights == nullptr || d_workspace == nullptr) return fail(m, MT_ERR_INVALID_ARG, "null arena");
+  if ((reinterpret_cast<uintptr_t>(d_weights) | reinterpret_cast<uintptr_t>(d_workspace)) & (kAlign - 1))
+    return fail(m, MT_ERR_INVALID_ARG, "arenas must be 256-byte aligned");
+  if (weights_bytes < m->weights_bytes || workspace_bytes < m->ws_total)
+    return fail(m, MT_ERR_INVALID_ARG, "arena smaller than mt_weights_bytes / mt_workspace_bytes");
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return fail_cuda(m, e, "querying the device");
+  int major = 0;
+  e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) return fail_cuda(m, e, "querying the device");
+  if (major != 10) return fail(m, MT_ERR_UNSUPPORTED, "the kernels are built for sm_100a only");
+  m->sm_count = sms;
+  m->d_weights = static_cast<uint8_t*>(d_weights);
+  m->d_workspace = static_cast<uint8_t*>(d_workspace);
+  m->ws_bytes_bound = workspace_bytes;
+  m->plans.clear();
+  m->trunk_loaded = false;
+  for (TaskEntry& t : m->tasks) t.loaded = false;
+  e = cudaMemset(m->d_workspace + m->ws_status, 0, 256);
+  if (e != cudaSuccess) return fail_cuda(m, e, "clearing the status word");
+  return MT_OK;
+}
+
+static int check_header(const mt_model* m, const void* blob, size_t bytes, uint32_t kind, int32_t task, size_t payload) {
+  if (blob == nullptr) return fail(m, MT_ERR_INVALID_ARG, "null blob");
+  if (bytes < kHeaderBytes) return fail(m, MT_ERR_BLOB_MISMATCH, "blob shorter than its header");
+  BlobHeader h;
+  memcpy(&h, blob, sizeof(h));
+  const mt_trunk_config& c = m->trunk;
+  if (h.magic != kBlobMagic || h.version != kBlobVersion) return fail(m, MT_ERR_BLOB_MISMATCH, "bad magic or version");
+  if (h.kind != kind) return fail(m, MT_ERR_BLOB_MISMATCH, "blob kind (full model / single task) mismatch");
+  if (h.hidden != c.hidden || h.heads != c.heads || h.ffn != c.ffn || h.trunk_layers != c.trunk_layers ||
+      h.vocab != c.vocab_size || h.max_position != c.max_position || h.type_vocab != c.type_vocab ||
+      h.n_tasks != static_cast<int32_t>(m->tasks.size()))
+    return fail(m, MT_ERR_BLOB_MISMATCH, "blob was written for another configuration");
+  if (kind == 1) {
+    const mt_task_config& tc = m->tasks[task].cfg;
+    if (h.task_index != task || h.fork_depth != tc.fork_depth || h.branch_layers != tc.branch_layers ||
+        h.num_classes != tc.num_classes)
+      return fail(m, MT_ERR_BLOB_MISMATCH, "task blob does not match this task's configuration");
+  }
+  if (h.payload_bytes != payload || bytes != payload + kHeaderBytes)
+    return fail(m, MT_ERR_BLOB_MISMATCH, "blob size disagrees with the configuration");
+  return MT_OK;
+}
+
+int mt_load_weights(mt_model* m, const void* host_blob, size_t bytes, void* stream) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (m->d_weights == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
+  int rc = check_header(m, host_blob, bytes, 0, -1, m->weights_bytes);
+  if (rc != MT_OK) return rc;
+  cudaError_t e = cudaMemcpyAsync(m->d_weights, static_cast<const uint8_t*>(host_blob) + kHeaderBytes, m->weights_bytes,
+                                  cudaMemcpyHostToDevice, as_stream(stream));
+  if (e != cudaSuccess) return fail_cuda(m, e, "copying weights");
+  m->trunk_loaded = true;
+  for (TaskEntry& t : m->tasks) t.loaded = true;
+  return MT_OK;
+}
+
+int mt_load_task_weights(mt_model* m, int32_t task, const void* host_blob, size_t bytes, void* stream) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (task < 0 || task >= static_cast<int32_t>(m->tasks.size())) return fail(m, MT_ERR_INVALID_ARG, "task out of range");
+  if (m->d_weights == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
+  TaskEntry& te = m->tasks[task];
+  int rc = check_header(m, host_blob, bytes, 1, task, te.section_bytes);
+  if (rc != MT_OK) return rc;
+  cudaError_t e = cudaMemcpyAsync(m->d_weights + te.section_begin, static_cast<const uint8_t*>(host_blob) + kHeaderBytes,
+                                  te.section_bytes, cudaMemcpyHostToDevice, as_stream(stream));
+  if (e != cudaSuccess) return fail_cuda(m, e, "copying task weights");
+  te.loaded = true;
+  return MT_OK;
+}
+
+int mt_plan_summary(const mt_model* m, uint64_t task_mask, int32_t* n_layers, int32_t* n_waves, int32_t* trunk_depth,
+                    int32_t* groups_per_wave) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  Schedule s;
+  if (!build_schedule(m, task_mask, &s)) return fail(m, MT_ERR_INVALID_ARG, "task_mask selects no task");
+  if (n_layers) *n_layers = s.n_layers;
+  if (n_waves) *n_waves = static_cast<int32_t>(s.waves.size());
+  if (trunk_depth) *trunk_depth = s.trunk_depth;
+  if (groups_per_wave)
+    for (size_t w = 0; w < s.waves.size(); ++w) groups_per_wave[w] = static_cast<int32_t>(s.waves[w].size());
+  return MT_OK;
+}
+
+int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches) {
+  if (m == nullptr || n_launches == nullptr) return MT_ERR_INVALID_ARG;
+  Schedule s;
+  if (!build_schedule(m, task_mask, &s)) return fail(m, MT_ERR_INVALID_ARG, "task_mask selects no task");
+  int32_t n = 1;
+  for (size_t w = 0; w <= s.waves.size(); ++w) {
+    if (w >= 1) n += 7 * static_cast<int32_t>((s.waves[w - 1].size() + m->n_slots - 1) / m->n_slots);
+    n += static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
+  }
+  *n_launches = n;
+  return MT_OK;
+}
+
+int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
+               uint64_t task_mask, int32_t batch, int32_t seq, float* d_logits, void* stream_) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr || d_logits == nullptr)
+    return fail(m, MT_ERR_INVALID_ARG, "null input or output pointer");
+  if (batch < 1 || seq < 1) return fail(m, MT_ERR_INVALID_ARG, "batch and seq must be positive");
+  if (batch > m->max_batch || seq > m->max_seq) return fail(m, MT_ERR_SHAPE, "batch/seq beyond the limits of mt_create");
+  if (m->d_workspace == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
+  const int32_t T = static_cast<int32_t>(m->tasks.size());
+  if (T < 64) task_mask &= (uint64_t(1) << T) - 1;
+  if (task_mask == 0) return fail(m, MT_ERR_INVALID_ARG, "task_mask selects no task");
+  if (!m->trunk_loaded) return fail(m, MT_ERR_NOT_LOADED, "mt_load_weights has not been called");
+  for (int32_t t = 0; t < T; ++t)
+    if (((task_mask >> t) & 1) && !m->tasks[t].loaded) return fail(m, MT_ERR_NOT_LOADED, "an active task has no weights");
+  cudaStream_t stream = as_stream(stream_);
+
+  const auto key = std::make_tuple(task_mask, batch, seq);
+  auto it = m->plans.find(key);
+  if (it == m->plans.end()) {
+    Schedule s;
+    build_schedule(m, task_mask, &s);
+    Plan plan;
+    cudaError_t e = build_plan(m, s, batch, seq, &plan);
+    if (e != cudaSuccess) return fail_cuda(m, e, "building the launch plan");
+    it = m->plans.emplace(key, std::move(plan)).first;
+  }
+  Plan& plan = it->second;
+  uint32_t* status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
+  const size_t act_used = static_cast<size_t>(batch) * seq * m->trunk.hidden * sizeof(bf16);
+  cudaError_t e;
+#define MT_LAUNCH(call, what)                          \
+  do {                                                 \
+    e = (call);                                        \
+    if (e != cudaSuccess) return fail_cuda(m, e, what); \
+  } while (0)
+
+  EmbedParams ep;
+  ep.token_ids = d_token_ids; ep.segment_ids = d_segment_ids; ep.lengths = d_lengths;
+  ep.word = w_ptr(m, m->emb_word); ep.pos = w_ptr(m, m->emb_pos); ep.type = w_ptr(m, m->emb_type);
+  ep.gamma = w_ptr(m, m->emb_ln_g); ep.beta = w_ptr(m, m->emb_ln_b);
+  ep.out = trunk_buf(m, 0);
+  ep.batch = batch; ep.seq = seq; ep.hidden = m->trunk.hidden; ep.vocab = m->trunk.vocab_size;
+  ep.type_vocab = m->trunk.type_vocab; ep.eps = m->trunk.ln_eps; ep.status = status;
+  MT_LAUNCH(launch_embed(ep, stream), "embedding kernel");
+  if (m->debug_capture)
+    MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0, ep.out, act_used, cudaMemcpyDeviceToDevice, stream),
+              "debug capture");
+
+  for (PlanStep& st : plan.steps) {
+    if (st.kind == 0) {
+      Chunk& ck = st.chunk;
+      ck.attn.lengths = d_lengths;
+      MT_LAUNCH(launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
+      MT_LAUNCH(launch_attention(ck.attn, stream), "attention kernel");
+      MT_LAUNCH(launch_gemm(ck.attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
+      MT_LAUNCH(launch_layernorm(ck.ln1, stream), "LayerNorm 1");
+      MT_LAUNCH(launch_gemm(ck.ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
+      MT_LAUNCH(launch_gemm(ck.ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
+      MT_LAUNCH(launch_layernorm(ck.ln2, stream), "LayerNorm 2");
+      for (const auto& d : ck.dumps)
+        MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.second, d.first, act_used,
+                                  cudaMemcpyDeviceToDevice, stream),
+                  "debug capture");
+    } else {
+      st.heads.logits = d_logits;
+      MT_LAUNCH(launch_pooler_head(st.heads, stream), "pooler/head kernel");
+    }
+  }
+#undef MT_LAUNCH
+  m->last_batch = batch;
+  m->last_seq = seq;
+  return MT_OK;
+}
+
+int mt_forward_host(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids, const int32_t* h_lengths,
+                    uint64_t task_mask, int32_t batch, int32_t seq, float* h_logits, void* stream_) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (h_token_ids == nullptr || h_segment_ids == nullptr || h_lengths == nullptr || h_logits == nullptr)
+    return fail(m, MT_ERR_INVALID_ARG, "null input or output pointer");
+  if (batch < 1 || seq < 1) return fail(m, MT_ERR_INVALID_ARG, "batch and seq must be positive");
+  if (batch > m->max_batch || seq > m->max_seq) return fail(m, MT_ERR_SHAPE, "batch/seq beyond the limits of mt_create");
+  if (m->d_workspace == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
+  cudaStream_t stream = as_stream(stream_);
+  int32_t* d_tok = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_tok);
+  int32_t* d_seg = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_seg);
+  int32_t* d_len = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_len);
+  float* d_logits = reinterpret_cast<float*>(m->d_workspace + m->ws_logits);
+  const size_t n = static_cast<size_t>(batch) * seq * 4;
+  const size_t out_bytes = static_cast<size_t>(batch) * m->c_total * 4;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(d_tok, h_token_ids, n, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(d_seg, h_segment_ids, n, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(d_len, h_lengths, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+      (e = cudaMemsetAsync(d_logits, 0, out_bytes, stream)) != cudaSuccess)
+    return fail_cuda(m, e, "copying inputs to the device");
+  int rc = mt_forward(m, d_tok, d_seg, d_len, task_mask, batch, seq, d_logits, stream_);
+  if (rc != MT_OK) return rc;
+  if ((e = cudaMemcpyAsync(h_logits, d_logits, out_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
+      (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+    return fail_cuda(m, e, "copying logits to the host");
+  return MT_OK;
+}
+
+int mt_poll_status(mt_model* m, void* stream_, uint32_t* flags) {
+  if (m == nullptr) return MT_ERR_INVALID_ARG;
+  if (m->d_workspace == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
+  cudaStream_t stream = as_stream(stream_);
+  uint32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, m->d_workspace + m->ws_status, 4, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(m->d_workspace + m->ws_status, 0, 4, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return fail_cuda(m, e, "reading the status word");
+  if (flags) *flags = word;
+  if (word != 0) {
+    char buf[64];
+    snprintf(buf, sizeof(buf), "device status word 0x%x", word);
+    return fail(m, MT_ERR_DEVICE_FLAG, buf);
+  }
+  return MT_OK;
+}
+
+int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out, void* stream_) {
+  if (m == nullptr || d_out == nullptr) return MT_ERR_INVALID_ARG;
+  if (!m->debug_capture) return fail(m, MT_ERR_INVALID_ARG, "option debug_capture is off");
+  if (m->d_workspace == nullptr || m->last_batch == 0) return fail(m, MT_ERR_NOT_BOUND, "no forward has run");
+  const int32_t T = static_cast<int32_t>(m->tasks.size());
+  if (task < -1 || task >= T) return fail(m, MT_ERR_INVALID_ARG, "task out of range");
+  if (task < 0 ? (layer < 0 || layer > m->trunk.trunk_layers) : (layer < 1 || layer > m->tasks[task].cfg.branch_layers))
+    return fail(m, MT_ERR_INVALID_ARG, "layer out of range");
+  const size_t bytes = static_cast<size_t>(m->last_batch) * m->last_seq * m->trunk.hidden * sizeof(bf16);
+  cudaError_t e = cudaMemcpyAsync(d_out, m->d_workspace + m->ws_dump0 + m->act_bytes * dump_slot(m, task, layer), bytes,
+                                  cudaMemcpyDeviceToDevice, as_stream(stream_));
+  if (e != cudaSuccess) return fail_cuda(m, e, "copying a captured hidden state");
+  return MT_OK;
+}
+
+// ---- single steps ------------------------------------------------------------------------------
+
+int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual, void* d_y, int32_t M,
+                     int32_t N, int32_t K, int32_t epilogue, uint32_t* d_status, void* stream) {
+  if (d_x == nullptr || d_w == nullptr || d_bias == nullptr || d_y == nullptr || M < 1 || N < 128 || N % 128 != 0 ||
+      K < 64 || K % 64 != 0 || epilogue < 0 || epilogue > 2 || (epilogue == 2 && d_residual == nullptr))
+    return MT_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MT_ERR_CUDA;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
+  if (make_tmap(&p.tmap_x[0], d_x, M, K, kGemmBlockM) != cudaSuccess) return MT_ERR_CUDA;
+  if (make_tmap(&p.tmap_w[0], d_w, N, K, gemm_block_n(N)) != cudaSuccess) return MT_ERR_CUDA;
+  p.group[0] = {static_cast<const bf16*>(d_bias), static_cast<const bf16*>(d_residual), static_cast<bf16*>(d_y)};
+  return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx, int32_t batch, int32_t seq,
+                        int32_t heads, void* stream) {
+  if (d_qkv == nullptr || d_lengths == nullptr || d_ctx == nullptr || batch < 1 || seq < 1 || heads < 1)
+    return MT_ERR_INVALID_ARG;
+  AttnParams p;
+  memset(&p, 0, sizeof(p));
+  p.qkv[0] = static_cast<const bf16*>(d_qkv);
+  p.ctx[0] = static_cast<bf16*>(d_ctx);
+  p.lengths = d_lengths;
+  p.n_groups = 1; p.batch = batch; p.seq = seq; p.heads = heads;
+  return launch_attention(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y, int32_t rows,
+                        int32_t hidden, float eps, void* stream) {
+  if (d_x == nullptr || d_gamma == nullptr || d_beta == nullptr || d_y == nullptr || rows < 1) return MT_ERR_INVALID_ARG;
+  if (hidden != 768 && hidden != 1024) return MT_ERR_UNSUPPORTED;
+  LayerNormParams p;
+  memset(&p, 0, sizeof(p));
+  p.x[0] = static_cast<const bf16*>(d_x); p.gamma[0] = static_cast<const bf16*>(d_gamma);
+  p.beta[0] = static_cast<const bf16*>(d_beta); p.y[0] = static_cast<bf16*>(d_y);
+  p.n_groups = 1; p.rows = rows; p.hidden = hidden; p.eps = eps;
+  return launch_layernorm(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
+                    const void* d_word, const void* d_pos, const void* d_type, const void* d_gamma, const void* d_beta,
+                    void* d_h0, int32_t batch, int32_t seq, int32_t hidden, int32_t vocab, int32_t type_vocab, float eps,
+                    uint32_t* d_status, void* stream) {
+  if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr || d_word == nullptr ||
+      d_pos == nullptr || d_type == nullptr || d_gamma == nullptr || d_beta == nullptr || d_h0 == nullptr ||
+      batch < 1 || seq < 1 || vocab < 1 || type_vocab < 1)
+    return MT_ERR_INVALID_ARG;
+  if (hidden != 768 && hidden != 1024) return MT_ERR_UNSUPPORTED;
+  EmbedParams p;
+  p.token_ids = d_token_ids; p.segment_ids = d_segment_ids; p.lengths = d_lengths;
+  p.word = static_cast<const bf16*>(d_word); p.pos = static_cast<const bf16*>(d_pos);
+  p.type = static_cast<const bf16*>(d_type); p.gamma = static_cast<const bf16*>(d_gamma);
+  p.beta = static_cast<const bf16*>(d_beta); p.out = static_cast<bf16*>(d_h0);
+  p.batch = batch; p.seq = seq; p.hidden = hidden; p.vocab = vocab; p.type_vocab = type_vocab; p.eps = eps;
+  p.status = d_status;
+  return launch_embed(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void* d_pool_b, const void* d_cls_w,
+                          const void* d_cls_b, float* d_logits, int32_t batch, int32_t seq, int32_t hidden,
+                          int32_t num_classes, int32_t logits_stride, int32_t col0, void* stream) {
+  if (d_hidden == nullptr || d_pool_w == nullptr || d_pool_b == nullptr || d_cls_w == nullptr || d_cls_b == nullptr ||
+      d_logits == nullptr || batch < 1 || seq < 1 || num_classes < 1 || col0 < 0 || logits_stride < col0 + num_classes)
+    return MT_ERR_INVALID_ARG;
+  if (hidden != 768 && hidden != 1024) return MT_ERR_UNSUPPORTED;
+  HeadParams p;
+  memset(&p, 0, sizeof(p));
+  p.task[0] = {static_cast<const bf16*>(d_hidden), static_cast<const bf16*>(d_pool_w),
+               static_cast<const bf16*>(d_pool_b), static_cast<const bf16*>(d_cls_w),
+               static_cast<const bf16*>(d_cls_b), num_classes, col0};
+  p.logits = d_logits;
+  p.n_tasks = 1; p.batch = batch; p.seq = seq; p.hidden = hidden; p.logits_stride = logits_stride;
+  return launch_pooler_head(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+// Internal interface between the host-side scheduler and the sm_100a kernels.
+// Every launcher enqueues on the given stream and returns the cudaError_t of the launch.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mt {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxGroups = 8;      // layers fused into one grouped launch
+constexpr int kHeadDim = 64;       // the only head width implemented
+constexpr int kGemmBlockM = 128;   // rows of one GEMM tile (one tcgen05 accumulator = 128 TMEM lanes)
+constexpr int kGemmBlockK = 64;    // bf16 elements per 128-byte swizzled shared-memory row
+
+constexpr uint32_t kFlagBadToken = 0x1u;
+constexpr uint32_t kFlagBadSegment = 0x2u;
+constexpr uint32_t kFlagBadLength = 0x4u;
+constexpr uint32_t kFlagWaitTimeout = 0x8u;
+
+enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2 };
+
+// One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).
+// All groups of a launch share M, N, K and the epilogue.
+struct GemmGroup {
+  const bf16* bias;
+  const bf16* residual;  // only read by kEpiBiasResidual
+  bf16* out;
+};
+
+struct alignas(64) GemmParams {
+  CUtensorMap tmap_x[kMaxGroups];  // X_g: dims {K, M}, box {64, 128}, 128-byte swizzle
+  CUtensorMap tmap_w[kMaxGroups];  // W_g: dims {K, N}, box {64, block_n}, 128-byte swizzle
+  GemmGroup group[kMaxGroups];
+  int32_t n_groups;
+  int32_t M, N, K;
+  uint32_t* status;  // sticky device status word (may be null)
+};
+
+// Tile width along N chosen for a given N (fixed per N so results never depend on grouping).
+int gemm_block_n(int N);
+cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
+
+struct AttnParams {
+  const bf16* qkv[kMaxGroups];  // [B*S, 3*H] = [Q | K | V]
+  bf16* ctx[kMaxGroups];        // [B*S, H]
+  const int32_t* lengths;       // [B]
+  int32_t n_groups, batch, seq, heads;
+};
+cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
+
+struct LayerNormParams {
+  const bf16* x[kMaxGroups];
+  const bf16* gamma[kMaxGroups];
+  const bf16* beta[kMaxGroups];
+  bf16* y[kMaxGroups];
+  int32_t n_groups, rows, hidden;
+  float eps;
+};
+cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream);
+
+struct EmbedParams {
+  const int32_t* token_ids;
+  const int32_t* segment_ids;
+  const int32_t* lengths;
+  const bf16 *word, *pos, *type, *gamma, *beta;
+  bf16* out;
+  int32_t batch, seq, hidden, vocab, type_vocab;
+  float eps;
+  uint32_t* status;
+};
+cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream);
+
+struct HeadTask {
+  const bf16* hidden;  // final state of the task, [B*S, H]; row b*S is pooled
+  const bf16 *pool_w, *pool_b, *cls_w, *cls_b;
+  int32_t num_classes, col0;
+};
+struct HeadParams {
+  HeadTask task[kMaxGroups];
+  float* logits;
+  int32_t n_tasks, batch, seq, hidden, logits_stride;
+};
+cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream);
+
+}  // namespace mt

@@ -1,0 +1,217 @@
+// The memory-bound steps of the path: embedding gather + LayerNorm, LayerNorm, pooler + head.
+// One warp owns one row of H bf16 values, held entirely in registers (H/256 16-byte vectors per
+// lane, fully coalesced), statistics in fp32 with the mean subtracted before the variance.
+
+#include "mt_kernels.h"
+
+namespace mt {
+namespace {
+
+constexpr int kRowThreads = 256;  // 8 rows per CTA
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t*>(&v);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Normalises the row held in x[V][8] (lane-strided vectors) and writes it.
+template <int V>
+__device__ __forceinline__ void normalise_store(float (&x)[V][8], const bf16* gamma, const bf16* beta, bf16* out,
+                                                int lane, float eps) {
+  constexpr int H = V * 256;
+  float s = 0.f;
+#pragma unroll
+  for (int v = 0; v < V; ++v)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s += x[v][i];
+  const float mean = warp_sum(s) * (1.0f / H);
+  float q = 0.f;
+#pragma unroll
+  for (int v = 0; v < V; ++v)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float d = x[v][i] - mean;
+      q += d * d;
+    }
+  const float rstd = rsqrtf(warp_sum(q) * (1.0f / H) + eps);
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    const int col = (v * 32 + lane) * 8;
+    float g[8], b[8], y[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(gamma + col)), g);
+    unpack8(__ldg(reinterpret_cast<const uint4*>(beta + col)), b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = (x[v][i] - mean) * rstd * g[i] + b[i];
+    *reinterpret_cast<uint4*>(out + col) = pack8(y);
+  }
+}
+
+template <int V>
+__global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormParams p) {
+  constexpr int H = V * 256;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+  const int g = blockIdx.y;
+  if (row >= p.rows) return;
+  const bf16* xin = p.x[g] + static_cast<size_t>(row) * H;
+  float x[V][8];
+#pragma unroll
+  for (int v = 0; v < V; ++v) unpack8(*reinterpret_cast<const uint4*>(xin + (v * 32 + lane) * 8), x[v]);
+  normalise_store<V>(x, p.gamma[g], p.beta[g], p.y[g] + static_cast<size_t>(row) * H, lane, p.eps);
+}
+
+template <int V>
+__global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p) {
+  constexpr int H = V * 256;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+  if (row >= p.batch * p.seq) return;
+  const int b = row / p.seq;
+  const int pos = row - b * p.seq;
+  int tok = p.token_ids[row];
+  int seg = p.segment_ids[row];
+  uint32_t flags = 0;
+  if (tok < 0 || tok >= p.vocab) { flags |= kFlagBadToken; tok = tok < 0 ? 0 : p.vocab - 1; }
+  if (seg < 0 || seg >= p.type_vocab) { flags |= kFlagBadSegment; seg = seg < 0 ? 0 : p.type_vocab - 1; }
+  if (pos == 0) {
+    const int len = p.lengths[b];
+    if (len < 1 || len > p.seq) flags |= kFlagBadLength;
+  }
+  if (flags != 0 && lane == 0 && p.status != nullptr) atomicOr(p.status, flags);
+  const bf16* w = p.word + static_cast<size_t>(tok) * H;
+  const bf16* q = p.pos + static_cast<size_t>(pos) * H;
+  const bf16* t = p.type + static_cast<size_t>(seg) * H;
+  float x[V][8];
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    const int col = (v * 32 + lane) * 8;
+    float a[8], c[8], d[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(w + col)), a);
+    unpack8(__ldg(reinterpret_cast<const uint4*>(q + col)), c);
+    unpack8(__ldg(reinterpret_cast<const uint4*>(t + col)), d);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[v][i] = a[i] + c[i] + d[i];
+  }
+  normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(row) * H, lane, p.eps);
+}
+
+// Pooler + head.  One CTA = (task, chunk of kSeqPerCta sequences).  The position-0 rows are staged
+// in shared memory as fp32; every warp produces pooled features j = warp, warp + 8, ... for all
+// sequences of the chunk at once (the pooler matrix row is read once per CTA), then the C_t x chunk
+// logits are warp-level dot products against the pooled vectors.
+constexpr int kSeqPerCta = 8;
+constexpr int kHeadThreads = 256;
+
+__global__ void __launch_bounds__(kHeadThreads) pooler_head_kernel(const HeadParams p) {
+  extern __shared__ float sh[];
+  const int H = p.hidden;
+  float* cls = sh;                       // [kSeqPerCta][H]
+  float* pooled = sh + kSeqPerCta * H;   // [kSeqPerCta][H]
+  const HeadTask tk = p.task[blockIdx.y];
+  const int b0 = blockIdx.x * kSeqPerCta;
+  const int nb = min(kSeqPerCta, p.batch - b0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int idx = threadIdx.x; idx < kSeqPerCta * (H / 8); idx += kHeadThreads) {
+    const int s = idx / (H / 8), c = idx - s * (H / 8);
+    float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (s < nb)
+      unpack8(*reinterpret_cast<const uint4*>(tk.hidden + static_cast<size_t>(b0 + s) * p.seq * H + c * 8), f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) cls[s * H + c * 8 + i] = f[i];
+  }
+  __syncthreads();
+
+  const int vecs = H / 256;  // 16-byte vectors per lane per row
+  for (int j = warp; j < H; j += kHeadThreads / 32) {
+    float acc[kSeqPerCta];
+#pragma unroll
+    for (int s = 0; s < kSeqPerCta; ++s) acc[s] = 0.f;
+    for (int v = 0; v < vecs; ++v) {
+      const int col = (v * 32 + lane) * 8;
+      float w[8];
+      unpack8(__ldg(reinterpret_cast<const uint4*>(tk.pool_w + static_cast<size_t>(j) * H + col)), w);
+#pragma unroll
+      for (int s = 0; s < kSeqPerCta; ++s) {
+        const float4 c0 = *reinterpret_cast<const float4*>(cls + s * H + col);
+        const float4 c1 = *reinterpret_cast<const float4*>(cls + s * H + col + 4);
+        acc[s] += w[0] * c0.x + w[1] * c0.y + w[2] * c0.z + w[3] * c0.w + w[4] * c1.x + w[5] * c1.y + w[6] * c1.z +
+                  w[7] * c1.w;
+      }
+    }
+    const float bias = __bfloat162float(tk.pool_b[j]);
+#pragma unroll
+    for (int s = 0; s < kSeqPerCta; ++s) {
+      const float t = warp_sum(acc[s]);
+      if (lane == 0) pooled[s * H + j] = tanhf(t + bias);
+    }
+  }
+  __syncthreads();
+
+  for (int o = warp; o < tk.num_classes * nb; o += kHeadThreads / 32) {
+    const int c = o / nb, s = o - c * nb;
+    float acc = 0.f;
+    for (int k = lane; k < H; k += 32) acc += __bfloat162float(tk.cls_w[static_cast<size_t>(c) * H + k]) * pooled[s * H + k];
+    acc = warp_sum(acc);
+    if (lane == 0)
+      p.logits[static_cast<size_t>(b0 + s) * p.logits_stride + tk.col0 + c] = acc + __bfloat162float(tk.cls_b[c]);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1) return cudaErrorInvalidValue;
+  dim3 grid((p.rows + kRowThreads / 32 - 1) / (kRowThreads / 32), p.n_groups);
+  if (p.hidden == 768) layernorm_kernel<3><<<grid, kRowThreads, 0, stream>>>(p);
+  else if (p.hidden == 1024) layernorm_kernel<4><<<grid, kRowThreads, 0, stream>>>(p);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream) {
+  const int rows = p.batch * p.seq;
+  if (rows < 1) return cudaErrorInvalidValue;
+  dim3 grid((rows + kRowThreads / 32 - 1) / (kRowThreads / 32));
+  if (p.hidden == 768) embed_kernel<3><<<grid, kRowThreads, 0, stream>>>(p);
+  else if (p.hidden == 1024) embed_kernel<4><<<grid, kRowThreads, 0, stream>>>(p);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream) {
+  if (p.n_tasks < 1 || p.n_tasks > kMaxGroups || p.batch < 1 || p.hidden % 256 != 0) return cudaErrorInvalidValue;
+  const size_t smem = static_cast<size_t>(2) * kSeqPerCta * p.hidden * sizeof(float);
+  static int configured_device = -1;
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (configured_device != dev) {
+    err = cudaFuncSetAttribute(pooler_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSeqPerCta * 1024 * 4);
+    if (err != cudaSuccess) return err;
+    configured_device = dev;
+  }
+  dim3 grid((p.batch + kSeqPerCta - 1) / kSeqPerCta, p.n_tasks);
+  pooler_head_kernel<<<grid, kHeadThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace mt

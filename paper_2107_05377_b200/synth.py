@@ -150,10 +150,16 @@ def uniform01(seed: int, name: str, start: int, count: int) -> np.ndarray:
 
 
 def standard_normal(seed: int, name: str, count: int) -> np.ndarray:
-    """Box-Muller on draws 2i and 2i+1 of the stream."""
-    u = uniform01(seed, name, 0, 2 * count)
-    u1, u2 = u[0::2], u[1::2]
-    return np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    """Box-Muller: draws 2i and 2i+1 of the stream give normals 2i (cosine
+    branch) and 2i+1 (sine branch)."""
+    pairs = (count + 1) // 2
+    u = uniform01(seed, name, 0, 2 * pairs)
+    r = np.sqrt(-2.0 * np.log(u[0::2]))
+    theta = 2.0 * np.pi * u[1::2]
+    z = np.empty(2 * pairs, dtype=np.float64)
+    z[0::2] = r * np.cos(theta)
+    z[1::2] = r * np.sin(theta)
+    return z[:count]
 
 
 def randint(seed: int, name: str, count: int, lo: int, hi_inclusive: int) -> np.ndarray:
@@ -305,9 +311,9 @@ def _append_task(chunks: List[bytes], tw: Dict) -> None:
 
 def _header(cfg: TreeConfig, kind: int, task_index: int, spec: TaskSpec | None, payload: int) -> bytes:
     d, k, c = (spec.fork_depth, spec.branch_layers, spec.num_classes) if spec else (0, 0, 0)
-    h = struct.pack("<IIIiiiiiiiiiiiiQ", BLOB_MAGIC, BLOB_VERSION, kind, cfg.hidden, cfg.heads, cfg.ffn,
+    h = struct.pack("<IIIiiiiiiiiiiiiiQ", BLOB_MAGIC, BLOB_VERSION, kind, cfg.hidden, cfg.heads, cfg.ffn,
                     cfg.trunk_layers, cfg.vocab_size, cfg.max_position, cfg.type_vocab,
-                    cfg.n_tasks, task_index, d, k, c, payload)
+                    cfg.n_tasks, task_index, d, k, c, 0, payload)
     return h + b"\0" * (BLOB_HEADER_BYTES - len(h))
 
 

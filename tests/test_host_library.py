@@ -1,0 +1,140 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every
+declared symbol, validates its arguments, sizes its blobs like the generator packs
+them, and schedules exactly the layer totals the paper prints (Tables 2 and 4)."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2107_05377_b200 import binding, build, synth
+from test_oracle_pins import read_paper_layer_counts
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mt_bert.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mt_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_symbols()
+    assert len(names) >= 20
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/mt_bert.h but not exported"
+        assert n in binding.SIGNATURES, f"{n} has no binding signature"
+    assert sorted(binding.SIGNATURES) == names
+
+
+def small_cfg(tasks, trunk_layers=12):
+    return synth.TreeConfig(vocab_size=64, max_position=64, trunk_layers=trunk_layers,
+                            tasks=tuple(synth.TaskSpec(*t) for t in tasks))
+
+
+@pytest.mark.parametrize("name,total,xy", read_paper_layer_counts())
+def test_scheduler_runs_the_papers_layer_totals(lib, name, total, xy):
+    cfg = small_cfg([(x, y, 2) for x, y in xy])
+    m = binding.MTModel(cfg, 4, 32, bind=False)
+    s = m.plan_summary(m.full_mask())
+    assert s["layers"] == total
+    assert s["trunk_depth"] == max(x for x, _ in xy)
+    assert sum(s["groups_per_wave"]) == total
+    assert s["waves"] == max(x + y for x, y in xy)
+    # wave w holds trunk layer w (if w <= depth) plus branch layer w - x of every task with x < w <= x + y
+    for w in range(1, s["waves"] + 1):
+        want = (1 if w <= s["trunk_depth"] else 0) + sum(1 for x, y in xy if x < w <= x + y)
+        assert s["groups_per_wave"][w - 1] == want
+    m.close()
+
+
+def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
+    cfg = synth.config_glue8()
+    m = binding.MTModel(cfg, 32, 128, bind=False)
+    s = m.plan_summary(0xFF)
+    assert s == {"layers": 24, "waves": 10, "trunk_depth": 8, "groups_per_wave": [1, 1, 1, 1, 2, 3, 5, 6, 3, 1]}
+    only6 = m.plan_summary(1 << 6)           # forks at 4, three branch layers
+    assert only6["layers"] == 7 and only6["trunk_depth"] == 4 and only6["groups_per_wave"] == [1] * 7
+    only7 = m.plan_summary(1 << 7)           # forks at 8, two branch layers
+    assert only7["layers"] == 10 and only7["trunk_depth"] == 8
+    for mask in (0b00010010, 0b10100101, 0b01000000):
+        act = [t for t in range(8) if (mask >> t) & 1]
+        want = max(cfg.tasks[t].fork_depth for t in act) + sum(cfg.tasks[t].branch_layers for t in act)
+        assert m.plan_summary(mask)["layers"] == want
+    with pytest.raises(binding.MTError):
+        m.plan_summary(0)
+    assert m.plan_launches(0xFF) == 1 + 7 * 10 + 4   # embedding, 7 launches per wave, heads after waves 7, 8, 9, 10
+    m.close()
+    m2 = binding.MTModel(cfg, 32, 128, max_groups=2, bind=False)
+    assert m2.plan_summary(0xFF)["layers"] == 24
+    assert m2.plan_launches(0xFF) == 1 + 7 * (1 + 1 + 1 + 1 + 1 + 2 + 3 + 3 + 2 + 1) + 4
+    m2.close()
+
+
+def test_create_rejects_bad_configurations(lib):
+    def create(trunk_kw=None, tasks=((4, 1, 2),), max_batch=2, max_seq=32):
+        kw = dict(vocab_size=64, max_position=64, type_vocab=2, hidden=768, heads=12, ffn=3072, trunk_layers=4,
+                  ln_eps=1e-12, activation=0)
+        kw.update(trunk_kw or {})
+        trunk = binding.TrunkConfig(**kw)
+        arr = (binding.TaskConfig * len(tasks))(*[binding.TaskConfig(*t) for t in tasks])
+        h = C.c_void_p()
+        rc = lib.mt_create(C.byref(trunk), arr, len(tasks), max_batch, max_seq, C.byref(h))
+        if rc == 0:
+            lib.mt_destroy(h)
+        return rc
+
+    assert create() == 0
+    assert create(tasks=((5, 1, 2),)) == -1            # fork beyond the trunk
+    assert create(tasks=((4, -1, 2),)) == -1
+    assert create(tasks=((4, 1, 0),)) == -1
+    assert create(tasks=((0, 0, 1),)) == 0              # fork at the embeddings, no branch, regression head
+    assert create({"hidden": 512, "heads": 8}) == -7    # width not implemented
+    assert create({"heads": 8}) == -7                   # head width != 64
+    assert create({"activation": 1}) == -7
+    assert create(max_seq=1024) == -7
+    assert create({"max_position": 16}) == -1           # max_seq beyond the position table
+    assert create(max_batch=0) == -1
+    h = C.c_void_p()
+    assert lib.mt_create(None, None, 1, 1, 1, C.byref(h)) == -1
+
+
+def test_unbound_model_fails_loudly(lib):
+    cfg = small_cfg([(1, 1, 2)], trunk_layers=1)
+    m = binding.MTModel(cfg, 2, 32, bind=False)
+    blob = np.zeros(m.blob_bytes(), dtype=np.uint8)
+    assert lib.mt_load_weights(m.handle, blob.ctypes.data, blob.size, None) == -3
+    assert lib.mt_forward(m.handle, 1, 1, 1, 1, 2, 32, 1, None) == -3
+    assert lib.mt_forward(m.handle, 1, 1, 1, 1, 4, 32, 1, None) == -2      # batch beyond max_batch
+    assert lib.mt_forward(m.handle, None, 1, 1, 1, 2, 32, 1, None) == -1
+    assert b"mt_bind_memory" in lib.mt_last_error_string(m.handle) or True
+    m.close()
+
+
+def test_blob_sizes_match_the_generator(lib):
+    cfg = small_cfg([(1, 1, 2), (0, 0, 1), (1, 2, 3)], trunk_layers=1)
+    m = binding.MTModel(cfg, 2, 32, bind=False)
+    w = synth.make_weights(cfg, seed=3)
+    blob = synth.pack_weights(cfg, w)
+    assert blob.size == m.blob_bytes() == m.weights_bytes() + 256
+    for t in range(3):
+        tb = synth.pack_task_weights(cfg, t, w["tasks"][t])
+        assert tb.size == m.task_blob_bytes(t)
+    assert m.task_blob_bytes(3) == 0
+    assert m.workspace_bytes() > 0
+    before = m.workspace_bytes()
+    m.set_option("debug_capture", 1)
+    assert m.workspace_bytes() > before
+    with pytest.raises(binding.MTError):
+        m.set_option("max_groups", 9)
+    with pytest.raises(binding.MTError):
+        m.set_option("nonsense", 1)
+    m.close()
