@@ -157,8 +157,26 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
 
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
  * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
- * mt_workspace_bytes; set before mt_bind_memory). */
+ * mt_workspace_bytes); both must be set before mt_bind_memory.  key "profile" (0/1): see
+ * mt_profile_read. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);
+
+/* Per-launch timing.  With option "profile" = 1 (may be toggled at any time) every kernel launch of
+ * mt_forward is bracketed by two CUDA events on the caller's stream (events are created on the host
+ * on first use).  mt_profile_read waits for the recorded events, adds the elapsed milliseconds and the
+ * launch counts per kernel class since the last read into the two arrays (MT_NUM_CLASSES entries
+ * each) and forgets them.  Classes follow the steps of the encoder layer. */
+#define MT_CLASS_EMBED     0  /* embedding gather + LayerNorm                       */
+#define MT_CLASS_QKV       1  /* GEMM: Q,K,V projections                            */
+#define MT_CLASS_ATTENTION 2  /* masked softmax attention                           */
+#define MT_CLASS_ATTN_OUT  3  /* GEMM: attention output projection + residual       */
+#define MT_CLASS_LN1       4  /* LayerNorm after attention                          */
+#define MT_CLASS_FFN_UP    5  /* GEMM: FFN up projection + GELU                     */
+#define MT_CLASS_FFN_DOWN  6  /* GEMM: FFN down projection + residual               */
+#define MT_CLASS_LN2       7  /* LayerNorm after the FFN                            */
+#define MT_CLASS_HEAD      8  /* pooler + head                                      */
+#define MT_NUM_CLASSES     9
+int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class);
 
 /* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out.
  * task = -1: trunk state after `layer` layers (0 = embedding output); task >= 0: state after branch

@@ -18,6 +18,7 @@ MT_OK = 0
 ERRORS = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "NOT_BOUND", -4: "NOT_LOADED", -5: "BLOB_MISMATCH",
           -6: "CUDA", -7: "UNSUPPORTED", -8: "DEVICE_FLAG"}
 FLAG_BAD_TOKEN, FLAG_BAD_SEGMENT, FLAG_BAD_LENGTH, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
+KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head")
 
 
 class TrunkConfig(C.Structure):
@@ -49,6 +50,7 @@ SIGNATURES = {
     "mt_plan_launches": (C.c_int, [_P, _U64, C.POINTER(_I32)]),
     "mt_set_option": (C.c_int, [_P, C.c_char_p, C.c_int64]),
     "mt_debug_copy_hidden": (C.c_int, [_P, _I32, _I32, _P, _P]),
+    "mt_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "mt_last_error_string": (C.c_char_p, [_P]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _P]),
@@ -239,6 +241,13 @@ class MTModel:
         if rc not in (MT_OK, -8):
             _check(rc, "mt_poll_status", self.handle)
         return flags.value
+
+    def profile_read(self):
+        """{class name: (milliseconds, launches)} since the last read (option "profile")."""
+        ms = (C.c_double * len(KERNEL_CLASSES))()
+        n = (C.c_int64 * len(KERNEL_CLASSES))()
+        _check(lib().mt_profile_read(self.handle, ms, n), "mt_profile_read", self.handle)
+        return {name: (ms[i], n[i]) for i, name in enumerate(KERNEL_CLASSES)}
 
     def debug_hidden(self, task: int, layer: int, batch: int, seq: int):
         import torch

@@ -153,6 +153,12 @@ struct mt_model {
 
   std::map<std::tuple<uint64_t, int32_t, int32_t>, Plan> plans;
   int32_t last_batch, last_seq;
+
+  // optional per-launch timing (option "profile"): event pairs recorded around every launch
+  bool profile;
+  std::vector<cudaEvent_t> events;                 // pool, two per recorded launch
+  std::vector<int32_t> event_class;                // class of the i-th recorded launch
+  size_t events_used;
   std::string last_error;
 };
 
@@ -413,6 +419,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->sm_count = 0;
   m->trunk_loaded = false;
   m->last_batch = m->last_seq = 0;
+  m->profile = false;
+  m->events_used = 0;
 
   const size_t H = trunk->hidden, e = sizeof(bf16);
   size_t off = 0;
@@ -448,7 +456,11 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   return MT_OK;
 }
 
-void mt_destroy(mt_model* m) { delete m; }
+void mt_destroy(mt_model* m) {
+  if (m == nullptr) return;
+  for (cudaEvent_t ev : m->events) cudaEventDestroy(ev);
+  delete m;
+}
 
 size_t mt_weights_bytes(const mt_model* m) { return m ? m->weights_bytes : 0; }
 size_t mt_workspace_bytes(const mt_model* m) { return m ? m->ws_total : 0; }
@@ -462,6 +474,12 @@ const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c
 
 int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
+  if (strcmp(key, "profile") == 0) {
+    m->profile = value != 0;
+    m->events_used = 0;
+    m->event_class.clear();
+    return MT_OK;
+  }
   if (m->d_workspace != nullptr) return fail(m, MT_ERR_INVALID_ARG, "options must be set before mt_bind_memory");
   if (strcmp(key, "max_groups") == 0) {
     if (value < 1 || value > kMaxGroups) return fail(m, MT_ERR_INVALID_ARG, "max_groups must be in 1..8");
@@ -614,6 +632,24 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
     e = (call);                                        \
     if (e != cudaSuccess) return fail_cuda(m, e, what); \
   } while (0)
+  // With option "profile" every kernel launch sits between two events of a pool that grows on the host.
+#define MT_TIMED(cls, call, what)                                                            \
+  do {                                                                                       \
+    if (m->profile) {                                                                        \
+      while (m->events.size() < m->events_used + 2) {                                        \
+        cudaEvent_t ev;                                                                      \
+        MT_LAUNCH(cudaEventCreate(&ev), "creating a timing event");                          \
+        m->events.push_back(ev);                                                             \
+      }                                                                                      \
+      MT_LAUNCH(cudaEventRecord(m->events[m->events_used], stream), "recording an event");   \
+    }                                                                                        \
+    MT_LAUNCH(call, what);                                                                   \
+    if (m->profile) {                                                                        \
+      MT_LAUNCH(cudaEventRecord(m->events[m->events_used + 1], stream), "recording an event"); \
+      m->events_used += 2;                                                                   \
+      m->event_class.push_back(cls);                                                         \
+    }                                                                                        \
+  } while (0)
 
   EmbedParams ep;
   ep.token_ids = d_token_ids; ep.segment_ids = d_segment_ids; ep.lengths = d_lengths;
@@ -622,7 +658,7 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
   ep.out = trunk_buf(m, 0);
   ep.batch = batch; ep.seq = seq; ep.hidden = m->trunk.hidden; ep.vocab = m->trunk.vocab_size;
   ep.type_vocab = m->trunk.type_vocab; ep.eps = m->trunk.ln_eps; ep.status = status;
-  MT_LAUNCH(launch_embed(ep, stream), "embedding kernel");
+  MT_TIMED(MT_CLASS_EMBED, launch_embed(ep, stream), "embedding kernel");
   if (m->debug_capture)
     MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0, ep.out, act_used, cudaMemcpyDeviceToDevice, stream),
               "debug capture");
@@ -631,22 +667,23 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
     if (st.kind == 0) {
       Chunk& ck = st.chunk;
       ck.attn.lengths = d_lengths;
-      MT_LAUNCH(launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
-      MT_LAUNCH(launch_attention(ck.attn, stream), "attention kernel");
-      MT_LAUNCH(launch_gemm(ck.attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
-      MT_LAUNCH(launch_layernorm(ck.ln1, stream), "LayerNorm 1");
-      MT_LAUNCH(launch_gemm(ck.ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
-      MT_LAUNCH(launch_gemm(ck.ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
-      MT_LAUNCH(launch_layernorm(ck.ln2, stream), "LayerNorm 2");
+      MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
+      MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
+      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(ck.attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
+      MT_TIMED(MT_CLASS_LN1, launch_layernorm(ck.ln1, stream), "LayerNorm 1");
+      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(ck.ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(ck.ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
+      MT_TIMED(MT_CLASS_LN2, launch_layernorm(ck.ln2, stream), "LayerNorm 2");
       for (const auto& d : ck.dumps)
         MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.second, d.first, act_used,
                                   cudaMemcpyDeviceToDevice, stream),
                   "debug capture");
     } else {
       st.heads.logits = d_logits;
-      MT_LAUNCH(launch_pooler_head(st.heads, stream), "pooler/head kernel");
+      MT_TIMED(MT_CLASS_HEAD, launch_pooler_head(st.heads, stream), "pooler/head kernel");
     }
   }
+#undef MT_TIMED
 #undef MT_LAUNCH
   m->last_batch = batch;
   m->last_seq = seq;
@@ -697,6 +734,22 @@ int mt_poll_status(mt_model* m, void* stream_, uint32_t* flags) {
     snprintf(buf, sizeof(buf), "device status word 0x%x", word);
     return fail(m, MT_ERR_DEVICE_FLAG, buf);
   }
+  return MT_OK;
+}
+
+int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class) {
+  if (m == nullptr || ms_by_class == nullptr || launches_by_class == nullptr) return MT_ERR_INVALID_ARG;
+  for (int c = 0; c < MT_NUM_CLASSES; ++c) { ms_by_class[c] = 0.0; launches_by_class[c] = 0; }
+  for (size_t i = 0; i < m->event_class.size(); ++i) {
+    cudaError_t e = cudaEventSynchronize(m->events[2 * i + 1]);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, m->events[2 * i], m->events[2 * i + 1]);
+    if (e != cudaSuccess) return fail_cuda(m, e, "reading a timing event");
+    ms_by_class[m->event_class[i]] += ms;
+    launches_by_class[m->event_class[i]] += 1;
+  }
+  m->events_used = 0;
+  m->event_class.clear();
   return MT_OK;
 }
 

@@ -1,0 +1,235 @@
+"""End-to-end parity of mt_forward (through the C ABI) against the fp64 oracle, and
+the paper's structural claims on the GPU path: merged == stand-alone students
+(bit-exact), per-task modularity, task masking, grouping invariance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mt_oracle as orc
+from paper_2107_05377_b200 import binding as mt
+from paper_2107_05377_b200 import synth
+from gpu_util import cached_weights, dev_batch, dev_bf16_to_f64, rel_l2, task_triples
+
+pytestmark = pytest.mark.gpu
+
+HIDDEN_REL_L2 = 1e-2   # tolerance on hidden states (valid rows)
+LOGIT_MAX_ABS = 2e-2   # tolerance on logits
+
+
+def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None):
+    B, S = batch.token_ids.shape
+    model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
+    model.load_weights(blob)
+    tok, seg, lens = dev_batch(batch)
+    logits = torch.full((B, cfg.total_classes), float("nan") if fill is None else fill, dtype=torch.float32,
+                        device="cuda")
+    model.forward(tok, seg, lens, logits, task_mask=mask)
+    torch.cuda.synchronize()
+    assert model.poll_status() == 0
+    return model, logits
+
+
+def check_against_oracle(cfg, wf, batch, model, logits, rows, mask=None, check_hidden=True):
+    B, S = batch.token_ids.shape
+    tasks = task_triples(cfg)
+    hid = []
+    want = orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, wf, tasks, cfg.heads, cfg.ln_eps,
+                                task_mask=mask, rows=rows, hidden_out=hid)
+    got = logits.cpu().numpy().astype(np.float64)
+    worst = 0.0
+    for b in rows:
+        ok = ~np.isnan(want[b])
+        assert ok.any()
+        assert np.all(np.isfinite(got[b][ok]))
+        worst = max(worst, float(np.max(np.abs(got[b][ok] - want[b][ok]))))
+    assert worst <= LOGIT_MAX_ABS, f"logits max-abs {worst}"
+    if check_hidden:
+        states = {}
+        for key in hid[0]:
+            t, layer = (-1, key[1]) if key[0] == "trunk" else (key[1], key[2])
+            states[key] = dev_bf16_to_f64(model.debug_hidden(t, layer, B, S)).reshape(B, S, cfg.hidden)
+        for i, b in enumerate(rows):
+            n = int(batch.lengths[b])
+            for key, ref in hid[i].items():
+                err = rel_l2(states[key][b, :n], ref)
+                assert err <= HIDDEN_REL_L2, f"hidden {key} row {b}: rel-L2 {err}"
+    return worst
+
+
+def test_tiny_tree_matches_oracle_everywhere():
+    cfg = synth.config_tiny()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_tiny(cfg)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    check_against_oracle(cfg, wf, batch, model, logits, rows=[0, 1])
+
+
+def test_ragged_batch_random_affine_matches_oracle():
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 5, 72, 1, 72, seed=9)
+    batch.lengths[:3] = [72, 1, 33]
+    batch = synth.Batch(np.where(np.arange(72)[None, :] < batch.lengths[:, None], batch.token_ids, 0).astype(np.int32),
+                        np.where(np.arange(72)[None, :] < batch.lengths[:, None], batch.segment_ids, 0).astype(np.int32),
+                        batch.lengths)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    check_against_oracle(cfg, wf, batch, model, logits, rows=range(5))
+
+
+def test_merged_equals_standalone_students_bit_exact():
+    """Section 3.3: merging only shares the frozen layers; each task's output is that of its own student."""
+    cfg = synth.config_tiny()
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 3, 64, 20, 64, seed=2)
+    _, merged = run_model(cfg, blob, batch)
+    offs = cfg.logit_offsets
+    for t in range(cfg.n_tasks):
+        st_cfg = synth.config_single_task(cfg, t)
+        st_blob = synth.pack_weights(st_cfg, synth.select_task_weights(w, t))
+        _, single = run_model(st_cfg, st_blob, batch)
+        cols = slice(offs[t], offs[t] + cfg.tasks[t].num_classes)
+        assert torch.equal(merged[:, cols], single), f"task {t}: merged and stand-alone logits differ"
+
+
+def test_grouping_and_masking_do_not_change_any_bit():
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 3, 64, 20, 64, seed=2)
+    _, base = run_model(cfg, blob, batch)
+    _, serial = run_model(cfg, blob, batch, max_groups=1)
+    assert torch.equal(base, serial)
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    for mask in (0b001, 0b010, 0b100, 0b101, 0b110):
+        _, part = run_model(cfg, blob, batch, mask=mask, fill=-55.0)
+        for t in range(3):
+            cols = slice(offs[t], offs[t + 1])
+            if (mask >> t) & 1:
+                assert torch.equal(part[:, cols], base[:, cols])
+            else:
+                assert torch.all(part[:, cols] == -55.0), "columns of inactive tasks must be left untouched"
+
+
+def test_per_task_update_leaves_other_tasks_bit_identical():
+    """Sections 1 and 5.1: a task is updated without affecting the others."""
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 3, 64, 20, 64, seed=2)
+    model, base = run_model(cfg, blob, batch)
+    new_task = synth.make_task_weights(cfg, 1, seed=77)
+    model.load_task_weights(1, synth.pack_task_weights(cfg, 1, new_task))
+    tok, seg, lens = dev_batch(batch)
+    after = torch.empty_like(base)
+    model.forward(tok, seg, lens, after)
+    torch.cuda.synchronize()
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    assert torch.equal(after[:, offs[0]:offs[1]], base[:, offs[0]:offs[1]])
+    assert torch.equal(after[:, offs[2]:offs[3]], base[:, offs[2]:offs[3]])
+    assert not torch.equal(after[:, offs[1]:offs[2]], base[:, offs[1]:offs[2]])
+    wf2 = dict(wf)
+    wf2["tasks"] = list(wf["tasks"])
+    wf2["tasks"][1] = synth.widen(new_task)
+    check_against_oracle(cfg, wf2, batch, model, after, rows=range(3), check_hidden=False)
+    # a blob written for another task is refused
+    with pytest.raises(mt.MTError) as e:
+        model.load_task_weights(0, synth.pack_task_weights(cfg, 1, new_task))
+    assert e.value.code == -5
+
+
+def test_padding_does_not_change_valid_outputs():
+    cfg = synth.config_tiny()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_tiny(cfg)
+    _, base = run_model(cfg, blob, batch)
+    rng = np.random.default_rng(3)
+    tok = np.concatenate([batch.token_ids, rng.integers(0, 30522, (2, 40)).astype(np.int32)], axis=1)
+    seg = np.concatenate([batch.segment_ids, rng.integers(0, 2, (2, 40)).astype(np.int32)], axis=1)
+    _, padded = run_model(cfg, blob, synth.Batch(tok, seg, batch.lengths))
+    assert float((padded - base).abs().max()) <= 1e-3
+
+
+def test_host_entry_point_and_error_paths():
+    cfg = synth.config_tiny()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_tiny(cfg)
+    model, dev_logits = run_model(cfg, blob, batch)
+    tok = torch.from_numpy(batch.token_ids).pin_memory()
+    seg = torch.from_numpy(batch.segment_ids).pin_memory()
+    lens = torch.from_numpy(batch.lengths).pin_memory()
+    host_logits = torch.empty(2, cfg.total_classes, dtype=torch.float32).pin_memory()
+    model.forward_host(tok, seg, lens, host_logits)
+    assert torch.equal(host_logits, dev_logits.cpu())
+    # out-of-range ids are clamped and flagged, the context stays usable
+    bad = batch.token_ids.copy()
+    bad[0, 3] = 40000
+    out = torch.empty_like(dev_logits)
+    model.forward(torch.from_numpy(bad).cuda(), *dev_batch(batch)[1:], out)
+    assert model.poll_status() == mt.FLAG_BAD_TOKEN
+    assert model.poll_status() == 0
+    # errors: empty mask, shape beyond the limits, truncated blob, unloaded model
+    for kwargs, code in (({"task_mask": 0}, -1),):
+        with pytest.raises(mt.MTError) as e:
+            model.forward(*dev_batch(batch), out, **kwargs)
+        assert e.value.code == code
+    big = synth.make_batch(cfg, 3, 32, 32, 32)
+    with pytest.raises(mt.MTError) as e:
+        model.forward(*dev_batch(big), torch.empty(3, cfg.total_classes, device="cuda"))
+    assert e.value.code == -2
+    with pytest.raises(mt.MTError) as e:
+        model.load_weights(blob[:-256].copy())
+    assert e.value.code == -5
+    corrupt = blob.copy()
+    corrupt[0] ^= 0xFF
+    with pytest.raises(mt.MTError) as e:
+        model.load_weights(corrupt)
+    assert e.value.code == -5
+    fresh = mt.MTModel(cfg, 2, 32)
+    with pytest.raises(mt.MTError) as e:
+        fresh.forward(*dev_batch(batch), out)
+    assert e.value.code == -4
+
+
+def test_glue8_tree_batch32_seq128_sampled_rows():
+    """The 8-task BERT-base tree at 32 x 128 with lengths in [16, 128], in the launch
+    configuration the benchmark times; the oracle is evaluated on sampled sequences
+    (sequences are independent, so each sampled row is an exact check)."""
+    cfg = synth.config_glue8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_glue8(cfg)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    order = np.argsort(batch.lengths)
+    rows = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), 0, 31})
+    check_against_oracle(cfg, wf, batch, model, logits, rows=rows)
+    assert torch.isfinite(logits).all()
+    # same result without the debug capture and with every wave run layer by layer
+    _, plain = run_model(cfg, blob, batch)
+    assert torch.equal(plain, logits)
+    # task masks: one task and a random half (seeded draw)
+    half = int(sum(1 << int(t) for t in np.random.default_rng(2).permutation(8)[:4]))
+    for mask in (1 << 6, 1 << 7, half):
+        _, part = run_model(cfg, blob, batch, mask=mask, fill=0.0)
+        offs = cfg.logit_offsets + [cfg.total_classes]
+        for t in range(8):
+            if (mask >> t) & 1:
+                assert torch.equal(part[:, offs[t]:offs[t + 1]], logits[:, offs[t]:offs[t + 1]])
+
+
+def test_glue8_tree_long_sequences_sampled_rows():
+    cfg = synth.config_glue8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 4, 512, 128, 512, seed=1)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    order = np.argsort(batch.lengths)
+    check_against_oracle(cfg, wf, batch, model, logits, rows=[int(order[0]), int(order[-1])])
+
+
+def test_large_width_tree_sampled_rows():
+    cfg = synth.config_large8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 8, 128, 32, 128, seed=1)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    check_against_oracle(cfg, wf, batch, model, logits, rows=[0, 5])

@@ -1,0 +1,161 @@
+"""Per-kernel parity: each step of the path, called through the C ABI on the GPU,
+against the matching fp64 oracle function on the same seeded bf16 inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mt_oracle as orc
+from paper_2107_05377_b200 import binding as mt
+from gpu_util import dev_bf16_to_f64, rand_bf16, rel_l2, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+# One bf16 rounding of the output (2^-9 relative) on top of fp32 accumulation.
+OUT_REL_L2 = 3e-3
+
+
+def bf16_round_tol(want):
+    """max-abs bound for a result rounded once to bf16: half an ulp of the largest value + slack."""
+    return float(np.max(np.abs(want))) * 2.0 ** -8 + 1e-3
+
+
+@pytest.mark.parametrize("M,N,K,epi", [
+    (64, 768, 768, 0),        # fewer rows than one tile
+    (128, 128, 64, 0),        # a single tile, a single k-block
+    (200, 768, 768, 2),       # ragged last tile, residual
+    (333, 2304, 768, 0),      # wide tile (N=2304 uses 256-wide tiles), ragged
+    (4096, 2304, 768, 0),     # QKV projection of the 32 x 128 batch
+    (4096, 768, 768, 2),      # attention output + residual
+    (4096, 3072, 768, 1),     # FFN up + GELU
+    (4096, 768, 3072, 2),     # FFN down + residual
+    (1000, 1024, 4096, 2),    # BERT-large width
+    (520, 4096, 1024, 1),
+])
+def test_linear_matches_oracle(M, N, K, epi):
+    xb, x = rand_bf16(11, f"x{M}.{N}.{K}", (M, K), 1.0)
+    wb, w = rand_bf16(12, f"w{M}.{N}.{K}", (N, K), 0.05)
+    bb, b = rand_bf16(13, f"b{M}.{N}.{K}", (N,), 0.5)
+    rb, r = rand_bf16(14, f"r{M}.{N}.{K}", (M, N), 1.0)
+    y = torch.full((M + 8, N), float("nan"), dtype=torch.bfloat16, device="cuda")   # 8 guard rows
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mt.mt_kernel_linear(to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(bb), to_dev_bf16(rb) if epi == 2 else None,
+                        y[:M], epi, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = orc.linear(x, w, b)
+    if epi == 1:
+        want = orc.gelu(want)
+    if epi == 2:
+        want = want + r
+    got = dev_bf16_to_f64(y[:M])
+    assert np.all(np.isfinite(got))
+    assert torch.isnan(y[M:].float()).all(), "rows beyond M were written"
+    assert rel_l2(got, want) <= OUT_REL_L2
+    assert np.max(np.abs(got - want)) <= bf16_round_tol(want)
+
+
+def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
+    H = heads * 64
+    ctx = np.zeros((B * S, H))
+    for b in range(B):
+        n = int(lengths[b])
+        blk = qkv[b * S:b * S + n]
+        for a in range(heads):
+            q, k, v = (blk[:, i * H + a * 64:i * H + (a + 1) * 64] for i in range(3))
+            ctx[b * S:b * S + n, a * 64:(a + 1) * 64] = orc.softmax_rows(q @ k.T / 8.0) @ v
+    return ctx
+
+
+@pytest.mark.parametrize("B,S,heads,lengths", [
+    (2, 32, 12, [32, 32]),
+    (4, 128, 12, [128, 37, 1, 64]),
+    (3, 100, 2, [100, 65, 9]),       # seq not a multiple of the tile
+    (2, 512, 16, [512, 300]),
+    (1, 1, 1, [1]),
+])
+def test_attention_matches_oracle(B, S, heads, lengths):
+    H = heads * 64
+    qb, qkv = rand_bf16(21, f"qkv{B}.{S}.{heads}", (B * S, 3 * H), 1.5)
+    # poison the padded rows of the input: they must not leak into valid rows
+    qkv_dev = to_dev_bf16(qb)
+    lens = torch.tensor(lengths, dtype=torch.int32, device="cuda")
+    for b, n in enumerate(lengths):
+        qkv_dev[b * S + n:(b + 1) * S] = float("nan")
+    ctx = torch.full((B * S, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    mt.mt_kernel_attention(qkv_dev, lens, ctx, B, S, heads)
+    torch.cuda.synchronize()
+    got = dev_bf16_to_f64(ctx)
+    want = oracle_attention_from_qkv(qkv, lengths, B, S, heads)
+    assert np.all(np.isfinite(got))
+    for b, n in enumerate(lengths):
+        assert np.all(got[b * S + n:(b + 1) * S] == 0), "padded query rows must be written as zero"
+    # probabilities are rounded to bf16 before the second product: 2^-9 relative per term
+    assert rel_l2(got, want) <= 5e-3
+    assert np.max(np.abs(got - want)) <= 2e-2 * max(1.0, float(np.max(np.abs(want))))
+
+
+@pytest.mark.parametrize("rows,H", [(1, 768), (8, 768), (4099, 768), (1000, 1024)])
+def test_layernorm_matches_oracle(rows, H):
+    xb, x = rand_bf16(31, f"ln{rows}", (rows, H), 2.0, mean=0.7)
+    gb, g = rand_bf16(32, f"g{H}", (H,), 0.2, mean=1.0)
+    bb, b = rand_bf16(33, f"b{H}", (H,), 0.2)
+    y = torch.empty(rows, H, dtype=torch.bfloat16, device="cuda")
+    mt.mt_kernel_layernorm(to_dev_bf16(xb), to_dev_bf16(gb), to_dev_bf16(bb), y, 1e-12)
+    torch.cuda.synchronize()
+    want = orc.layer_norm(x, g, b, 1e-12)
+    got = dev_bf16_to_f64(y)
+    assert rel_l2(got, want) <= OUT_REL_L2
+    assert np.max(np.abs(got - want)) <= bf16_round_tol(want)
+
+
+@pytest.mark.parametrize("H", [768, 1024])
+def test_embed_matches_oracle_and_flags_bad_ids(H):
+    B, S, V = 3, 40, 500
+    wb, w = rand_bf16(41, f"word{H}", (V, H), 0.02)
+    pb, p = rand_bf16(42, f"pos{H}", (64, H), 0.02)
+    tb, t = rand_bf16(43, f"type{H}", (2, H), 0.02)
+    gb, g = rand_bf16(44, f"eg{H}", (H,), 0.2, mean=1.0)
+    bb, b = rand_bf16(45, f"eb{H}", (H,), 0.2)
+    rng = np.random.default_rng(5)
+    tok = rng.integers(0, V, (B, S)).astype(np.int32)
+    seg = rng.integers(0, 2, (B, S)).astype(np.int32)
+    lens = np.array([40, 17, 1], dtype=np.int32)
+    out = torch.empty(B * S, H, dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = [to_dev_bf16(a) for a in (wb, pb, tb, gb, bb)]
+    mt.mt_kernel_embed(torch.from_numpy(tok).cuda(), torch.from_numpy(seg).cuda(), torch.from_numpy(lens).cuda(),
+                       *args, out, 1e-12, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    emb = {"word": w, "pos": p, "type": t, "ln_g": g, "ln_b": b}
+    got = dev_bf16_to_f64(out).reshape(B, S, H)
+    for i in range(B):
+        want = orc.embed(tok[i], seg[i], emb, 1e-12)   # every position, padded ones included
+        assert rel_l2(got[i], want) <= OUT_REL_L2
+        assert np.max(np.abs(got[i] - want)) <= bf16_round_tol(want)
+    # out-of-range ids are clamped and reported, never dereferenced
+    tok[0, 0], seg[1, 1], lens[2] = V + 7, 5, 0
+    mt.mt_kernel_embed(torch.from_numpy(tok).cuda(), torch.from_numpy(seg).cuda(), torch.from_numpy(lens).cuda(),
+                       *args, out, 1e-12, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == (mt.FLAG_BAD_TOKEN | mt.FLAG_BAD_SEGMENT | mt.FLAG_BAD_LENGTH)
+    assert torch.isfinite(out.float()).all()
+
+
+@pytest.mark.parametrize("B,S,H,C", [(2, 32, 768, 2), (32, 128, 768, 3), (9, 16, 1024, 1), (1, 8, 768, 1)])
+def test_pooler_head_matches_oracle(B, S, H, C):
+    hb, h = rand_bf16(51, f"h{B}.{S}.{H}", (B * S, H), 1.0)
+    pwb, pw = rand_bf16(52, f"pw{H}", (H, H), 0.05)
+    pbb, pb = rand_bf16(53, f"pb{H}", (H,), 0.1)
+    cwb, cw = rand_bf16(54, f"cw{H}.{C}", (C, H), 0.05)
+    cbb, cb = rand_bf16(55, f"cb{C}", (C,), 0.1)
+    logits = torch.full((B, C + 3), -77.0, dtype=torch.float32, device="cuda")
+    mt.mt_kernel_pooler_head(to_dev_bf16(hb), to_dev_bf16(pwb), to_dev_bf16(pbb), to_dev_bf16(cwb), to_dev_bf16(cbb),
+                             logits, B, S, col0=2)
+    torch.cuda.synchronize()
+    got = logits.cpu().numpy().astype(np.float64)
+    tw = {"pool_w": pw, "pool_b": pb, "cls_w": cw, "cls_b": cb}
+    for i in range(B):
+        want = orc.pooler_head(h[i * S:(i + 1) * S], tw)
+        assert np.max(np.abs(got[i, 2:2 + C] - want)) <= 1e-4
+    assert np.all(got[:, :2] == -77.0) and np.all(got[:, 2 + C:] == -77.0), "other tasks' columns must be untouched"
