@@ -1,0 +1,311 @@
+#!/usr/bin/env python
+"""Throughput of the merged multi-task forward pass: the 8-task BERT-base tree at
+batch 32 x seq 128 (valid lengths uniform in [16, 128]), sequences per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one mt_forward over one synthetic batch (all 24 transformer layers of the
+tree, embeddings, poolers and heads).  Prints ONE JSON line (rank 0).  With N > 1
+(launched by torch.distributed.run) every rank runs an independent replica on its own
+GPU - sequences are independent, the path has no exchange step - and the value is the
+sum over ranks divided by the slowest rank's time.
+
+--impl reference times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2107_05377_b200 import synth  # noqa: E402
+
+METRIC = "8-task BERT-base seq/s (seq128, b32)"
+UNIT = "sequences/s"
+BATCH, SEQ, LEN_LO, LEN_HI = 32, 128, 16, 128
+N_INPUT_BATCHES = 4
+REFERENCE_SAMPLE = 8          # sequences per step of the oracle arm
+L2_FLUSH_BYTES = 256 << 20    # larger than the 126 MB L2
+
+# DRAM traffic of the dominant kernel from one ncu capture (bytes per launch, averaged over the GEMM
+# launches of one forward), valid only for the kernel source it was taken on.
+NCU_TRAFFIC = {"gemm_source_sha256": None, "bytes_per_launch": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"tflops": float(p.get("bf16_tflops_sustained", p.get("bf16_tflops"))), "hbm_gbs": float(p["hbm_gbs"]),
+                "source": "measured (sustained)"}
+    return {"tflops": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def tasks_of(cfg):
+    return [(t.fork_depth, t.branch_layers, t.num_classes) for t in cfg.tasks]
+
+
+def gemm_flops_per_forward(cfg, n_layers, m_rows):
+    return n_layers * 2.0 * m_rows * (3 * cfg.hidden * cfg.hidden + cfg.hidden * cfg.hidden + 2 * cfg.hidden * cfg.ffn)
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(cfg, weights_f64, batch, rows):
+    from oracle import mt_oracle as orc
+    t0 = time.perf_counter()
+    orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, weights_f64, tasks_of(cfg), cfg.heads,
+                         cfg.ln_eps, rows=rows)
+    return time.perf_counter() - t0
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(device_index)], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            # the highest samples are the ones taken under load; report the median of the upper half
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    cfg = synth.config_glue8()
+    wf = synth.widen(synth.make_weights(cfg, seed=0))
+    batch = synth.batch_glue8(cfg, BATCH, SEQ, LEN_LO, LEN_HI, seed=1)
+    rows_of = lambda i: [(i * REFERENCE_SAMPLE + j) % BATCH for j in range(REFERENCE_SAMPLE)]  # noqa: E731
+    for i in range(args.warmup):
+        time_oracle(cfg, wf, batch, rows_of(i)[:2])
+    total = 0.0
+    for i in range(args.steps):
+        total += time_oracle(cfg, wf, batch, rows_of(i))
+    value = REFERENCE_SAMPLE * args.steps / total
+    cores = oracle_threads()
+    sample = f"{REFERENCE_SAMPLE} of the {BATCH} sequences per step (sequences are independent)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "glue8 tree (8 tasks, 24 layers), batch 32 x seq 128, lengths U[16,128]",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the oracle (N=1 only)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.impl == "reference" and args.steps == 50:
+            args.steps = 10
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2107_05377_b200 import binding
+    from paper_2107_05377_b200 import build as builder
+
+    args.warmup = max(args.warmup, 3)
+    if rank == 0 or world == 1:
+        builder.build()
+    distributed = world > 1
+    if distributed:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+
+    cfg = synth.config_glue8()
+    weights = synth.make_weights(cfg, seed=0)
+    model = binding.MTModel(cfg, BATCH, SEQ, device=str(device))
+    blob = torch.from_numpy(synth.pack_weights(cfg, weights)).pin_memory()
+    model.load_weights(blob)
+    mask = model.full_mask()
+    plan = model.plan_summary(mask)
+    launches_per_step = model.plan_launches(mask)
+
+    batches = [synth.batch_glue8(cfg, BATCH, SEQ, LEN_LO, LEN_HI, seed=1 + i) for i in range(N_INPUT_BATCHES)]
+    dev_in = [(torch.from_numpy(b.token_ids).to(device), torch.from_numpy(b.segment_ids).to(device),
+               torch.from_numpy(b.lengths).to(device)) for b in batches]
+    host_in = [(torch.from_numpy(b.token_ids).pin_memory(), torch.from_numpy(b.segment_ids).pin_memory(),
+                torch.from_numpy(b.lengths).pin_memory()) for b in batches]
+    logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32, device=device)
+    host_logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if distributed:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed_pass(steps):
+        """K forwards, each between two events on the launching stream, L2 flushed (untimed) before each."""
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        sync_all()
+        for i in range(steps):
+            flush.fill_(i & 0xFF)
+            starts[i].record(stream)
+            model.forward(*dev_in[i % N_INPUT_BATCHES], logits, task_mask=mask)
+            ends[i].record(stream)
+        sync_all()
+        return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+    for i in range(args.warmup):
+        model.forward(*dev_in[i % N_INPUT_BATCHES], logits, task_mask=mask)
+    sync_all()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    step_ms = timed_pass(args.steps)
+    total_ms = sum(step_ms)
+    clocks = sampler.stop() if sampler else None
+    assert model.poll_status() == 0, "device status word set during the timed region"
+
+    # end to end through the host entry point: pinned host inputs -> device, forward, logits -> host
+    for i in range(3):
+        model.forward_host(*host_in[i % N_INPUT_BATCHES], host_logits, task_mask=mask)
+    sync_all()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        model.forward_host(*host_in[i % N_INPUT_BATCHES], host_logits, task_mask=mask)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    # second pass of the same K steps with an event pair around every launch: per-kernel durations
+    model.set_option("profile", 1)
+    timed_pass(args.steps)
+    prof = model.profile_read()
+    model.set_option("profile", 0)
+
+    if distributed:
+        t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks = measured_peaks()
+        m_rows = BATCH * SEQ
+        gemm_classes = ("qkv", "attn_out", "ffn_up", "ffn_down")
+        gemm_ms = sum(prof[c][0] for c in gemm_classes)
+        gemm_launches = sum(prof[c][1] for c in gemm_classes)
+        gemm_flops = gemm_flops_per_forward(cfg, plan["layers"], m_rows) * args.steps
+        achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+        src = open(os.path.join(ROOT, "paper_2107_05377_b200", "csrc", "gemm_tcgen05.cu"), "rb").read()
+        traffic = NCU_TRAFFIC["bytes_per_launch"] \
+            if NCU_TRAFFIC["gemm_source_sha256"] == hashlib.sha256(src).hexdigest() else None
+        valid_tokens = float(np.mean([b.lengths.sum() for b in batches]))
+        padded_flops = gemm_flops_per_forward(cfg, plan["layers"], m_rows) + \
+            plan["layers"] * BATCH * 4.0 * cfg.hidden * SEQ * SEQ
+        value = world * BATCH * args.steps / (total_ms * 1e-3)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "glue8 tree (8 tasks, 24 transformer layers run), batch 32 x seq 128, "
+                                   "lengths U[16,128], bf16 weights N(0,0.02)",
+                       "global_batch": BATCH * world, "seq_len": SEQ, "parallelism": f"replicas x{world}",
+                       "l2": "256 MB buffer written before every timed step (untimed); each step also streams "
+                             "340 MB of weights, larger than L2",
+                       "layers_run": plan["layers"], "waves": plan["waves"], "groups_per_wave": plan["groups_per_wave"],
+                       "valid_tokens_per_step": valid_tokens, "padded_tokens_per_step": m_rows},
+            "gpu_launches": launches_per_step * args.steps,
+            "e2e": {"value": world * BATCH * args.steps / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": 2 * BATCH * SEQ * 4 + BATCH * 4,
+                    "d2h_bytes_per_step": BATCH * cfg.total_classes * 4},
+            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches)",
+                         "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                         "frac": achieved / peaks["tflops"], "peak_source": peaks["source"], "traffic": traffic,
+                         "launches": int(gemm_launches), "avg_launch_us": 1e3 * gemm_ms / max(gemm_launches, 1)},
+            "forward_tflops_padded": padded_flops * args.steps / (total_ms * 1e-3) / 1e12,
+            "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            wf = synth.widen(weights)
+            secs = time_oracle(cfg, wf, batches[0], range(BATCH))
+            out["cpu_baseline"] = {"value": BATCH / secs, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                                   "sample": f"one forward of all {BATCH} sequences of the first batch ({secs:.1f} s)"}
+        print(json.dumps(out))
+    if distributed:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -13,7 +13,9 @@
  *  - All device memory and all streams belong to the caller.  The library allocates only host
  *    metadata.  Pointers named d_* are DEVICE pointers, everything else is a HOST pointer.
  *  - cudaStream_t is passed as a plain `void*` (the value of the stream handle; NULL = default stream).
- *  - Activations and weights are bf16, accumulation and statistics fp32, logits fp32.
+ *  - Weights and the operands of every matrix product are bf16; accumulation, LayerNorm statistics
+ *    and the residual stream (every LayerNorm input and the residual it is added to) are fp32; logits
+ *    are fp32.
  *  - Every entry point returns an mt_status (0 = OK, negative = error); nothing throws, aborts or
  *    traps.  mt_last_error_string() describes the most recent failure on that model.
  *  - Encoder layer (the published post-LayerNorm BERT layer the paper builds on, Section 3):
@@ -188,9 +190,10 @@ const char* mt_last_error_string(const mt_model* m);
 /* ---- the individual steps, callable on their own (used by the per-kernel parity tests) -------- */
 /* All pointers are device pointers; d_status may be NULL or point to one uint32 status word.      */
 
-/* Y[M,N] = epilogue(X[M,K] . W[N,K]^T + bias[N]) on tcgen05 tensor cores (bf16 in, fp32 accumulate).
- * epilogue 0: +bias; 1: +bias then erf-GELU; 2: +bias +residual[M,N].  K % 64 == 0, N % 128 == 0,
- * all pointers 16-byte aligned.  This is one linear map of the layer above. */
+/* Y[M,N] = epilogue(X[M,K] . W[N,K]^T + bias[N]) on tcgen05 tensor cores (X, W, bias bf16; fp32
+ * accumulate).  epilogue 0: +bias, Y bf16; 1: +bias then erf-GELU, Y bf16; 2: +bias +residual with
+ * residual fp32 [M,N] and Y fp32 [M,N] (the LayerNorm input).  K % 64 == 0, N % 128 == 0, all
+ * pointers 16-byte aligned.  This is one linear map of the layer above. */
 int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
                      void* d_y, int32_t M, int32_t N, int32_t K, int32_t epilogue,
                      uint32_t* d_status, void* stream);
@@ -200,14 +203,15 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
 int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx,
                         int32_t batch, int32_t seq, int32_t heads, void* stream);
 
-/* y[rows, hidden] = LayerNorm(x) * gamma + beta (fp32 statistics, biased variance). hidden in {768, 1024}. */
-int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y,
+/* y[rows, hidden] = LayerNorm(x) * gamma + beta (fp32 statistics, biased variance) for fp32 x;
+ * written as bf16 to d_y and, when d_y_f32 is not NULL, as fp32 too.  hidden in {768, 1024}. */
+int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32,
                         int32_t rows, int32_t hidden, float eps, void* stream);
 
-/* h0[B*S, hidden] = LayerNorm(word[tok] + pos[position] + type[seg]). */
+/* h0[B*S, hidden] = LayerNorm(word[tok] + pos[position] + type[seg]), bf16 (and fp32 if d_h0_f32 != NULL). */
 int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
                     const void* d_word, const void* d_pos, const void* d_type,
-                    const void* d_gamma, const void* d_beta, void* d_h0,
+                    const void* d_gamma, const void* d_beta, void* d_h0, void* d_h0_f32,
                     int32_t batch, int32_t seq, int32_t hidden, int32_t vocab, int32_t type_vocab,
                     float eps, uint32_t* d_status, void* stream);
 

@@ -54,8 +54,9 @@ SIGNATURES = {
     "mt_last_error_string": (C.c_char_p, [_P]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _P]),
-    "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
-    "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P, _P]),
+    "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
+    "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
+                                  _P]),
     "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
 }
 
@@ -114,17 +115,17 @@ def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, str
            "mt_kernel_attention")
 
 
-def mt_kernel_layernorm(x, gamma, beta, y, eps: float, stream=None) -> None:
+def mt_kernel_layernorm(x, gamma, beta, y, eps: float, y_f32=None, stream=None) -> None:
     rows, hidden = x.shape
-    _check(lib().mt_kernel_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), rows, hidden, eps, _stream(stream)),
-           "mt_kernel_layernorm")
+    _check(lib().mt_kernel_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), _ptr(y_f32), rows, hidden, eps,
+                                     _stream(stream)), "mt_kernel_layernorm")
 
 
-def mt_kernel_embed(token_ids, segment_ids, lengths, word, pos, type_, gamma, beta, h0, eps: float, status=None,
-                    stream=None) -> None:
+def mt_kernel_embed(token_ids, segment_ids, lengths, word, pos, type_, gamma, beta, h0, eps: float, h0_f32=None,
+                    status=None, stream=None) -> None:
     batch, seq = token_ids.shape
     _check(lib().mt_kernel_embed(_ptr(token_ids), _ptr(segment_ids), _ptr(lengths), _ptr(word), _ptr(pos), _ptr(type_),
-                                 _ptr(gamma), _ptr(beta), _ptr(h0), batch, seq, word.shape[1], word.shape[0],
+                                 _ptr(gamma), _ptr(beta), _ptr(h0), _ptr(h0_f32), batch, seq, word.shape[1], word.shape[0],
                                  type_.shape[0], eps, _ptr(status), _stream(stream)), "mt_kernel_embed")
 
 

@@ -12,7 +12,8 @@
 //   warp 1      : allocates tensor memory; one thread issues tcgen05.mma (128 x BN x 16 per
 //                 instruction) with the accumulator in TMEM, and tcgen05.commit to release stages
 //   warps 2..   : epilogue - tcgen05.ld the fp32 accumulator (each warp its own 32-lane quarter),
-//                 add bias (+GELU or +residual), round once to bf16, 16-byte stores
+//                 add bias (+GELU) and round once to bf16, or add bias + fp32 residual and keep
+//                 fp32; 16-byte stores
 // The accumulator is double buffered in TMEM (2 x BN columns) so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Every output element is the sum over K in a fixed order inside a single
 // tile, so a result never depends on which other groups share the launch.
@@ -308,37 +309,53 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
         tmem_ld_wait();
         const int col = n0 + chunk * 32;
         const uint4* bias4 = reinterpret_cast<const uint4*>(grp.bias + col);
-        uint4 outv[4];
+        if (EPI == kEpiBiasResidual) {
+          // fp32 residual in, fp32 out: the pre-LayerNorm sum keeps full precision
+          const float4* res4 = reinterpret_cast<const float4*>(grp.residual + row_off + col);
+          float4* dst4 = reinterpret_cast<float4*>(static_cast<float*>(grp.out) + row_off + col);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint4 b = __ldg(bias4 + q);
-          const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-          uint4 r = make_uint4(0, 0, 0, 0);
-          if (EPI == kEpiBiasResidual && row_ok) {
-            r = *reinterpret_cast<const uint4*>(grp.residual + row_off + col + q * 8);
-          }
-          const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-          uint32_t ow[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
-            float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
-            if (EPI == kEpiBiasGelu) {
-              x0 = gelu_erf(x0);
-              x1 = gelu_erf(x1);
+          for (int q = 0; q < 4; ++q) {
+            const uint4 b = __ldg(bias4 + q);
+            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+            if (row_ok) {
+              const float4 r0 = res4[2 * q], r1 = res4[2 * q + 1];
+              float4 o0, o1;
+              o0.x = __uint_as_float(v[q * 8 + 0]) + bf16_lo(bw[0]) + r0.x;
+              o0.y = __uint_as_float(v[q * 8 + 1]) + bf16_hi(bw[0]) + r0.y;
+              o0.z = __uint_as_float(v[q * 8 + 2]) + bf16_lo(bw[1]) + r0.z;
+              o0.w = __uint_as_float(v[q * 8 + 3]) + bf16_hi(bw[1]) + r0.w;
+              o1.x = __uint_as_float(v[q * 8 + 4]) + bf16_lo(bw[2]) + r1.x;
+              o1.y = __uint_as_float(v[q * 8 + 5]) + bf16_hi(bw[2]) + r1.y;
+              o1.z = __uint_as_float(v[q * 8 + 6]) + bf16_lo(bw[3]) + r1.z;
+              o1.w = __uint_as_float(v[q * 8 + 7]) + bf16_hi(bw[3]) + r1.w;
+              dst4[2 * q] = o0;
+              dst4[2 * q + 1] = o1;
             }
-            if (EPI == kEpiBiasResidual) {
-              x0 += bf16_lo(rw[j]);
-              x1 += bf16_hi(rw[j]);
-            }
-            ow[j] = pack_bf16(x0, x1);
           }
-          outv[q] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-        }
-        if (row_ok) {
-          uint4* dst = reinterpret_cast<uint4*>(grp.out + row_off + col);
+        } else {
+          uint4 outv[4];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) dst[q] = outv[q];
+          for (int q = 0; q < 4; ++q) {
+            const uint4 b = __ldg(bias4 + q);
+            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+            uint32_t ow[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
+              float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
+              if (EPI == kEpiBiasGelu) {
+                x0 = gelu_erf(x0);
+                x1 = gelu_erf(x1);
+              }
+              ow[j] = pack_bf16(x0, x1);
+            }
+            outv[q] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+          }
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(grp.out) + row_off + col);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) dst[q] = outv[q];
+          }
         }
       }
       tc_fence_before();

@@ -146,7 +146,9 @@ struct mt_model {
 
   // workspace layout (byte offsets)
   size_t ws_status, ws_tok, ws_seg, ws_len, ws_logits, ws_trunk[2], ws_task0, ws_slot0, ws_dump0;
-  size_t act_bytes;   // max_batch*max_seq*hidden*2
+  size_t act_bytes;    // max_batch*max_seq*hidden bf16
+  size_t act32_bytes;  // the same tensor in fp32
+  size_t state_bytes;  // one hidden state = its bf16 copy (GEMM operand) followed by its fp32 copy (residual)
   size_t slot_bytes;
   int32_t n_slots, n_dump;
   size_t ws_total;
@@ -189,6 +191,8 @@ void layout_workspace(mt_model* m) {
   const size_t M = static_cast<size_t>(m->max_batch) * m->max_seq;
   const size_t H = m->trunk.hidden, F = m->trunk.ffn;
   m->act_bytes = pad256(M * H * sizeof(bf16));
+  m->act32_bytes = pad256(M * H * sizeof(float));
+  m->state_bytes = m->act_bytes + m->act32_bytes;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t at = off; off += pad256(bytes); return at; };
   m->ws_status = take(256);
@@ -196,13 +200,13 @@ void layout_workspace(mt_model* m) {
   m->ws_seg = take(M * 4);
   m->ws_len = take(static_cast<size_t>(m->max_batch) * 4);
   m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
-  m->ws_trunk[0] = take(m->act_bytes);
-  m->ws_trunk[1] = take(m->act_bytes);
+  m->ws_trunk[0] = take(m->state_bytes);
+  m->ws_trunk[1] = take(m->state_bytes);
   m->ws_task0 = off;
-  off += m->act_bytes * m->tasks.size();
+  off += m->state_bytes * m->tasks.size();
   m->n_slots = std::min<int32_t>(m->max_groups, static_cast<int32_t>(m->tasks.size()) + 1);
-  // slot = qkv [M,3H] + ctx [M,H] + u [M,H] + h1 [M,H] + f [M,F]
-  m->slot_bytes = pad256(M * 3 * H * 2) + 3 * m->act_bytes + pad256(M * F * 2);
+  // slot = qkv [M,3H] bf16 + ctx [M,H] bf16 + u [M,H] fp32 + h1 [M,H] bf16 and fp32 + f [M,F] bf16
+  m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2);
   m->ws_slot0 = off;
   off += m->slot_bytes * m->n_slots;
   m->n_dump = 0;
@@ -260,7 +264,11 @@ const bf16* w_ptr(const mt_model* m, size_t off) { return reinterpret_cast<const
 
 // Where the state of a stream lives: trunk depth d in ping-pong buffer d & 1, a task in its own buffer.
 bf16* trunk_buf(const mt_model* m, int32_t depth) { return ws_ptr(m, m->ws_trunk[depth & 1]); }
-bf16* task_buf(const mt_model* m, int32_t task) { return ws_ptr(m, m->ws_task0 + m->act_bytes * task); }
+bf16* task_buf(const mt_model* m, int32_t task) { return ws_ptr(m, m->ws_task0 + m->state_bytes * task); }
+// fp32 copy of a state: stored right after its bf16 copy
+float* f32_of(const mt_model* m, bf16* state) {
+  return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(state) + m->act_bytes);
+}
 
 cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int32_t batch,
                         int32_t seq, Chunk* ck) {
@@ -304,9 +312,9 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     uint8_t* slot = m->d_workspace + m->ws_slot0 + m->slot_bytes * i;
     bf16* qkv = reinterpret_cast<bf16*>(slot);
     bf16* ctx = reinterpret_cast<bf16*>(slot + qkv_bytes);
-    bf16* u = reinterpret_cast<bf16*>(slot + qkv_bytes + act);
-    bf16* h1 = reinterpret_cast<bf16*>(slot + qkv_bytes + 2 * act);
-    bf16* f = reinterpret_cast<bf16*>(slot + qkv_bytes + 3 * act);
+    float* u = reinterpret_cast<float*>(slot + qkv_bytes + act);
+    bf16* h1 = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes);
+    bf16* f = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes + m->state_bytes);
 
     cudaError_t e;
     // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv]   (the three matrices and biases are contiguous in the arena)
@@ -316,12 +324,13 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     // 2. ctx = attention(qkv)
     ck->attn.qkv[i] = qkv;
     ck->attn.ctx[i] = ctx;
-    // 3. u = ctx . Wo^T + bo + in
+    // 3. u = ctx . Wo^T + bo + in   (fp32 residual, fp32 result)
     if ((e = make_tmap(&ck->attn_out.tmap_x[i], ctx, M, H, kGemmBlockM)) != cudaSuccess) return e;
     if ((e = make_tmap(&ck->attn_out.tmap_w[i], w_ptr(m, lo->wo), H, H, gemm_block_n(H))) != cudaSuccess) return e;
-    ck->attn_out.group[i] = {w_ptr(m, lo->bo), in, u};
+    ck->attn_out.group[i] = {w_ptr(m, lo->bo), f32_of(m, in), u};
     // 4. h1 = LN(u)
-    ck->ln1.x[i] = u; ck->ln1.gamma[i] = w_ptr(m, lo->ln1_g); ck->ln1.beta[i] = w_ptr(m, lo->ln1_b); ck->ln1.y[i] = h1;
+    ck->ln1.x[i] = u; ck->ln1.gamma[i] = w_ptr(m, lo->ln1_g); ck->ln1.beta[i] = w_ptr(m, lo->ln1_b);
+    ck->ln1.y[i] = h1; ck->ln1.y32[i] = f32_of(m, h1);
     // 5. f = GELU(h1 . W1^T + b1)
     if ((e = make_tmap(&ck->ffn_up.tmap_x[i], h1, M, H, kGemmBlockM)) != cudaSuccess) return e;
     if ((e = make_tmap(&ck->ffn_up.tmap_w[i], w_ptr(m, lo->w1), F, H, gemm_block_n(F))) != cudaSuccess) return e;
@@ -329,9 +338,10 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     // 6. u = f . W2^T + b2 + h1
     if ((e = make_tmap(&ck->ffn_down.tmap_x[i], f, M, F, kGemmBlockM)) != cudaSuccess) return e;
     if ((e = make_tmap(&ck->ffn_down.tmap_w[i], w_ptr(m, lo->w2), H, F, gemm_block_n(H))) != cudaSuccess) return e;
-    ck->ffn_down.group[i] = {w_ptr(m, lo->b2), h1, u};
+    ck->ffn_down.group[i] = {w_ptr(m, lo->b2), f32_of(m, h1), u};
     // 7. out = LN(u)
-    ck->ln2.x[i] = u; ck->ln2.gamma[i] = w_ptr(m, lo->ln2_g); ck->ln2.beta[i] = w_ptr(m, lo->ln2_b); ck->ln2.y[i] = out;
+    ck->ln2.x[i] = u; ck->ln2.gamma[i] = w_ptr(m, lo->ln2_g); ck->ln2.beta[i] = w_ptr(m, lo->ln2_b);
+    ck->ln2.y[i] = out; ck->ln2.y32[i] = f32_of(m, out);
 
     if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer)});
   }
@@ -656,6 +666,7 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
   ep.word = w_ptr(m, m->emb_word); ep.pos = w_ptr(m, m->emb_pos); ep.type = w_ptr(m, m->emb_type);
   ep.gamma = w_ptr(m, m->emb_ln_g); ep.beta = w_ptr(m, m->emb_ln_b);
   ep.out = trunk_buf(m, 0);
+  ep.out32 = f32_of(m, ep.out);
   ep.batch = batch; ep.seq = seq; ep.hidden = m->trunk.hidden; ep.vocab = m->trunk.vocab_size;
   ep.type_vocab = m->trunk.type_vocab; ep.eps = m->trunk.ln_eps; ep.status = status;
   MT_TIMED(MT_CLASS_EMBED, launch_embed(ep, stream), "embedding kernel");
@@ -784,7 +795,7 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
   if (make_tmap(&p.tmap_x[0], d_x, M, K, kGemmBlockM) != cudaSuccess) return MT_ERR_CUDA;
   if (make_tmap(&p.tmap_w[0], d_w, N, K, gemm_block_n(N)) != cudaSuccess) return MT_ERR_CUDA;
-  p.group[0] = {static_cast<const bf16*>(d_bias), static_cast<const bf16*>(d_residual), static_cast<bf16*>(d_y)};
+  p.group[0] = {static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual), d_y};
   return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
@@ -801,22 +812,23 @@ int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx
   return launch_attention(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
-int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y, int32_t rows,
-                        int32_t hidden, float eps, void* stream) {
+int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32,
+                        int32_t rows, int32_t hidden, float eps, void* stream) {
   if (d_x == nullptr || d_gamma == nullptr || d_beta == nullptr || d_y == nullptr || rows < 1) return MT_ERR_INVALID_ARG;
   if (hidden != 768 && hidden != 1024) return MT_ERR_UNSUPPORTED;
   LayerNormParams p;
   memset(&p, 0, sizeof(p));
-  p.x[0] = static_cast<const bf16*>(d_x); p.gamma[0] = static_cast<const bf16*>(d_gamma);
+  p.x[0] = static_cast<const float*>(d_x); p.gamma[0] = static_cast<const bf16*>(d_gamma);
   p.beta[0] = static_cast<const bf16*>(d_beta); p.y[0] = static_cast<bf16*>(d_y);
+  p.y32[0] = static_cast<float*>(d_y_f32);
   p.n_groups = 1; p.rows = rows; p.hidden = hidden; p.eps = eps;
   return launch_layernorm(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
 int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
                     const void* d_word, const void* d_pos, const void* d_type, const void* d_gamma, const void* d_beta,
-                    void* d_h0, int32_t batch, int32_t seq, int32_t hidden, int32_t vocab, int32_t type_vocab, float eps,
-                    uint32_t* d_status, void* stream) {
+                    void* d_h0, void* d_h0_f32, int32_t batch, int32_t seq, int32_t hidden, int32_t vocab,
+                    int32_t type_vocab, float eps, uint32_t* d_status, void* stream) {
   if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr || d_word == nullptr ||
       d_pos == nullptr || d_type == nullptr || d_gamma == nullptr || d_beta == nullptr || d_h0 == nullptr ||
       batch < 1 || seq < 1 || vocab < 1 || type_vocab < 1)
@@ -827,6 +839,7 @@ int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, co
   p.word = static_cast<const bf16*>(d_word); p.pos = static_cast<const bf16*>(d_pos);
   p.type = static_cast<const bf16*>(d_type); p.gamma = static_cast<const bf16*>(d_gamma);
   p.beta = static_cast<const bf16*>(d_beta); p.out = static_cast<bf16*>(d_h0);
+  p.out32 = static_cast<float*>(d_h0_f32);
   p.batch = batch; p.seq = seq; p.hidden = hidden; p.vocab = vocab; p.type_vocab = type_vocab; p.eps = eps;
   p.status = d_status;
   return launch_embed(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;

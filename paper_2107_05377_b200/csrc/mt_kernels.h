@@ -24,11 +24,12 @@ constexpr uint32_t kFlagWaitTimeout = 0x8u;
 enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2 };
 
 // One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).
-// All groups of a launch share M, N, K and the epilogue.
+// All groups of a launch share M, N, K and the epilogue.  kEpiBias and kEpiBiasGelu write bf16;
+// kEpiBiasResidual adds an fp32 residual and writes fp32 (the pre-LayerNorm sum is never rounded).
 struct GemmGroup {
   const bf16* bias;
-  const bf16* residual;  // only read by kEpiBiasResidual
-  bf16* out;
+  const float* residual;  // fp32 [M,N], only read by kEpiBiasResidual
+  void* out;              // bf16 [M,N], or fp32 [M,N] for kEpiBiasResidual
 };
 
 struct alignas(64) GemmParams {
@@ -52,11 +53,14 @@ struct AttnParams {
 };
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
 
+// y = LN(x): x fp32; y is written as bf16 (the next GEMM's operand) and, if y32 is not null, also
+// as fp32 (the residual of the next sub-layer, so the residual stream is never rounded to bf16).
 struct LayerNormParams {
-  const bf16* x[kMaxGroups];
+  const float* x[kMaxGroups];
   const bf16* gamma[kMaxGroups];
   const bf16* beta[kMaxGroups];
   bf16* y[kMaxGroups];
+  float* y32[kMaxGroups];
   int32_t n_groups, rows, hidden;
   float eps;
 };
@@ -68,6 +72,7 @@ struct EmbedParams {
   const int32_t* lengths;
   const bf16 *word, *pos, *type, *gamma, *beta;
   bf16* out;
+  float* out32;  // may be null
   int32_t batch, seq, hidden, vocab, type_vocab;
   float eps;
   uint32_t* status;

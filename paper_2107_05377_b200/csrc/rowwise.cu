@@ -1,6 +1,8 @@
 // The memory-bound steps of the path: embedding gather + LayerNorm, LayerNorm, pooler + head.
-// One warp owns one row of H bf16 values, held entirely in registers (H/256 16-byte vectors per
-// lane, fully coalesced), statistics in fp32 with the mean subtracted before the variance.
+// One warp owns one row of H values, held entirely in registers (H/256 groups of 8 per lane,
+// 16-byte accesses, fully coalesced), statistics in fp32 with the mean subtracted before the
+// variance.  LayerNorm reads the fp32 pre-normalisation sum and writes the result twice: bf16 for
+// the next GEMM's operand and fp32 for the next residual add.
 
 #include "mt_kernels.h"
 
@@ -35,7 +37,7 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
 // Normalises the row held in x[V][8] (lane-strided vectors) and writes it.
 template <int V>
 __device__ __forceinline__ void normalise_store(float (&x)[V][8], const bf16* gamma, const bf16* beta, bf16* out,
-                                                int lane, float eps) {
+                                                float* out32, int lane, float eps) {
   constexpr int H = V * 256;
   float s = 0.f;
 #pragma unroll
@@ -61,6 +63,10 @@ __device__ __forceinline__ void normalise_store(float (&x)[V][8], const bf16* ga
 #pragma unroll
     for (int i = 0; i < 8; ++i) y[i] = (x[v][i] - mean) * rstd * g[i] + b[i];
     *reinterpret_cast<uint4*>(out + col) = pack8(y);
+    if (out32 != nullptr) {
+      *reinterpret_cast<float4*>(out32 + col) = make_float4(y[0], y[1], y[2], y[3]);
+      *reinterpret_cast<float4*>(out32 + col + 4) = make_float4(y[4], y[5], y[6], y[7]);
+    }
   }
 }
 
@@ -71,11 +77,17 @@ __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormP
   const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
   const int g = blockIdx.y;
   if (row >= p.rows) return;
-  const bf16* xin = p.x[g] + static_cast<size_t>(row) * H;
+  const float* xin = p.x[g] + static_cast<size_t>(row) * H;
   float x[V][8];
 #pragma unroll
-  for (int v = 0; v < V; ++v) unpack8(*reinterpret_cast<const uint4*>(xin + (v * 32 + lane) * 8), x[v]);
-  normalise_store<V>(x, p.gamma[g], p.beta[g], p.y[g] + static_cast<size_t>(row) * H, lane, p.eps);
+  for (int v = 0; v < V; ++v) {
+    const float4 a = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8);
+    const float4 b = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8 + 4);
+    x[v][0] = a.x; x[v][1] = a.y; x[v][2] = a.z; x[v][3] = a.w;
+    x[v][4] = b.x; x[v][5] = b.y; x[v][6] = b.z; x[v][7] = b.w;
+  }
+  float* y32 = p.y32[g] != nullptr ? p.y32[g] + static_cast<size_t>(row) * H : nullptr;
+  normalise_store<V>(x, p.gamma[g], p.beta[g], p.y[g] + static_cast<size_t>(row) * H, y32, lane, p.eps);
 }
 
 template <int V>
@@ -110,7 +122,8 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
 #pragma unroll
     for (int i = 0; i < 8; ++i) x[v][i] = a[i] + c[i] + d[i];
   }
-  normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(row) * H, lane, p.eps);
+  float* out32 = p.out32 != nullptr ? p.out32 + static_cast<size_t>(row) * H : nullptr;
+  normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(row) * H, out32, lane, p.eps);
 }
 
 // Pooler + head.  One CTA = (task, chunk of kSeqPerCta sequences).  The position-0 rows are staged
