@@ -82,14 +82,14 @@ def time_oracle(cfg, weights_f64, batch, rows):
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,utilization.gpu")
 
     def __init__(self, device_index: int):
         self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(device_index)], stdout=self.file,
+                                          "-lms", "50", "-i", str(device_index)], stdout=self.file,
                                          stderr=subprocess.DEVNULL)
         except OSError:
             pass
@@ -105,7 +105,7 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, busy = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.file.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
@@ -116,14 +116,19 @@ class ClockSampler:
                 mx.append(float(parts[2]))
             except ValueError:
                 continue
+            try:
+                busy.append(float(parts[9]) >= 50.0)
+            except (ValueError, IndexError):
+                busy.append(True)
             for name, val in zip(names, parts[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         self.file.close()
         os.unlink(self.file.name)
         if sm:
-            # the highest samples are the ones taken under load; report the median of the upper half
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            loaded = [c for c, b in zip(sm, busy) if b] or sm   # samples taken while the GPU was busy
+            out.update(sm_mhz=statistics.median(loaded), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), samples_under_load=len(loaded))
         return out
 
 
@@ -156,7 +161,7 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the oracle (N=1 only)")
@@ -166,7 +171,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     if args.impl == "reference":
-        if args.impl == "reference" and args.steps == 50:
+        if args.steps == 200:
             args.steps = 10
         run_reference(args, rank)
         return
@@ -227,14 +232,13 @@ def main():
         sync_all()
         return [s.elapsed_time(e) for s, e in zip(starts, ends)]
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None   # samples through all passes below
     for i in range(args.warmup):
         model.forward(*dev_in[i % N_INPUT_BATCHES], logits, task_mask=mask)
     sync_all()
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     step_ms = timed_pass(args.steps)
     total_ms = sum(step_ms)
-    clocks = sampler.stop() if sampler else None
     assert model.poll_status() == 0, "device status word set during the timed region"
 
     # end to end through the host entry point: pinned host inputs -> device, forward, logits -> host
@@ -252,6 +256,7 @@ def main():
     timed_pass(args.steps)
     prof = model.profile_read()
     model.set_option("profile", 0)
+    clocks = sampler.stop() if sampler else None
 
     if distributed:
         t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=device)

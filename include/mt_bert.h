@@ -215,9 +215,11 @@ int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, co
                     int32_t batch, int32_t seq, int32_t hidden, int32_t vocab, int32_t type_vocab,
                     float eps, uint32_t* d_status, void* stream);
 
-/* logits[b, col0 + c] = cls_w[c,:] . tanh(pool_w . h[b*seq, :] + pool_b) + cls_b[c], c < num_classes. */
+/* logits[b, col0 + c] = cls_w[c,:] . tanh(pool_w . h[b*seq, :] + pool_b) + cls_b[c], c < num_classes.
+ * Two launches (pooler, head); d_pooled_scratch is caller-provided scratch of batch*hidden floats that
+ * carries the tanh features between them (contents afterwards: those features). */
 int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void* d_pool_b,
-                          const void* d_cls_w, const void* d_cls_b, float* d_logits,
+                          const void* d_cls_w, const void* d_cls_b, float* d_pooled_scratch, float* d_logits,
                           int32_t batch, int32_t seq, int32_t hidden, int32_t num_classes,
                           int32_t logits_stride, int32_t col0, void* stream);
 

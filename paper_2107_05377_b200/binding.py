@@ -57,7 +57,7 @@ SIGNATURES = {
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
                                   _P]),
-    "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
+    "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
 }
 
 _lib = None
@@ -129,9 +129,10 @@ def mt_kernel_embed(token_ids, segment_ids, lengths, word, pos, type_, gamma, be
                                  type_.shape[0], eps, _ptr(status), _stream(stream)), "mt_kernel_embed")
 
 
-def mt_kernel_pooler_head(hidden, pool_w, pool_b, cls_w, cls_b, logits, batch: int, seq: int, col0: int = 0,
-                          stream=None) -> None:
-    _check(lib().mt_kernel_pooler_head(_ptr(hidden), _ptr(pool_w), _ptr(pool_b), _ptr(cls_w), _ptr(cls_b), _ptr(logits),
+def mt_kernel_pooler_head(hidden, pool_w, pool_b, cls_w, cls_b, pooled_scratch, logits, batch: int, seq: int,
+                          col0: int = 0, stream=None) -> None:
+    _check(lib().mt_kernel_pooler_head(_ptr(hidden), _ptr(pool_w), _ptr(pool_b), _ptr(cls_w), _ptr(cls_b),
+                                       _ptr(pooled_scratch), _ptr(logits),
                                        batch, seq, pool_w.shape[0], cls_w.shape[0], logits.shape[1], col0,
                                        _stream(stream)), "mt_kernel_pooler_head")
 

@@ -145,7 +145,7 @@ struct mt_model {
   int sm_count;
 
   // workspace layout (byte offsets)
-  size_t ws_status, ws_tok, ws_seg, ws_len, ws_logits, ws_trunk[2], ws_task0, ws_slot0, ws_dump0;
+  size_t ws_status, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0, ws_slot0, ws_dump0;
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
   size_t state_bytes;  // one hidden state = its bf16 copy (GEMM operand) followed by its fp32 copy (residual)
@@ -200,6 +200,8 @@ void layout_workspace(mt_model* m) {
   m->ws_seg = take(M * 4);
   m->ws_len = take(static_cast<size_t>(m->max_batch) * 4);
   m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
+  // tanh pooler outputs of the tasks of one head launch: fp32 [kMaxGroups][max_batch][H]
+  m->ws_pooled = take(static_cast<size_t>(kMaxGroups) * m->max_batch * H * sizeof(float));
   m->ws_trunk[0] = take(m->state_bytes);
   m->ws_trunk[1] = take(m->state_bytes);
   m->ws_task0 = off;
@@ -360,6 +362,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       st.heads.n_tasks = static_cast<int32_t>(count);
       st.heads.batch = batch; st.heads.seq = seq; st.heads.hidden = m->trunk.hidden;
       st.heads.logits_stride = m->c_total;
+      st.heads.pooled = reinterpret_cast<float*>(m->d_workspace + m->ws_pooled);
       for (size_t i = 0; i < count; ++i) {
         const int32_t t = tasks[first + i];
         const TaskEntry& te = m->tasks[t];
@@ -370,7 +373,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         ht.num_classes = te.cfg.num_classes; ht.col0 = te.col0;
       }
       plan->steps.push_back(std::move(st));
-      plan->launches += 1;
+      plan->launches += 2;
     }
   };
   add_heads(s.heads[0]);
@@ -601,7 +604,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
   int32_t n = 1;
   for (size_t w = 0; w <= s.waves.size(); ++w) {
     if (w >= 1) n += 7 * static_cast<int32_t>((s.waves[w - 1].size() + m->n_slots - 1) / m->n_slots);
-    n += static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
+    n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
   }
   *n_launches = n;
   return MT_OK;
@@ -846,8 +849,9 @@ int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, co
 }
 
 int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void* d_pool_b, const void* d_cls_w,
-                          const void* d_cls_b, float* d_logits, int32_t batch, int32_t seq, int32_t hidden,
-                          int32_t num_classes, int32_t logits_stride, int32_t col0, void* stream) {
+                          const void* d_cls_b, float* d_pooled_scratch, float* d_logits, int32_t batch, int32_t seq,
+                          int32_t hidden, int32_t num_classes, int32_t logits_stride, int32_t col0, void* stream) {
+  if (d_pooled_scratch == nullptr) return MT_ERR_INVALID_ARG;
   if (d_hidden == nullptr || d_pool_w == nullptr || d_pool_b == nullptr || d_cls_w == nullptr || d_cls_b == nullptr ||
       d_logits == nullptr || batch < 1 || seq < 1 || num_classes < 1 || col0 < 0 || logits_stride < col0 + num_classes)
     return MT_ERR_INVALID_ARG;
@@ -858,6 +862,7 @@ int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void
                static_cast<const bf16*>(d_pool_b), static_cast<const bf16*>(d_cls_w),
                static_cast<const bf16*>(d_cls_b), num_classes, col0};
   p.logits = d_logits;
+  p.pooled = d_pooled_scratch;
   p.n_tasks = 1; p.batch = batch; p.seq = seq; p.hidden = hidden; p.logits_stride = logits_stride;
   return launch_pooler_head(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }

@@ -87,8 +87,10 @@ struct HeadTask {
 struct HeadParams {
   HeadTask task[kMaxGroups];
   float* logits;
+  float* pooled;  // scratch, fp32 [n_tasks][batch][hidden]: tanh pooler outputs between the two launches
   int32_t n_tasks, batch, seq, hidden, logits_stride;
 };
+// Two launches: pooler (tanh features into `pooled`), then head (logits).
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream);
 
 }  // namespace mt

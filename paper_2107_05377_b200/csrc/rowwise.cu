@@ -126,20 +126,21 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
   normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(row) * H, out32, lane, p.eps);
 }
 
-// Pooler + head.  One CTA = (task, chunk of kSeqPerCta sequences).  The position-0 rows are staged
-// in shared memory as fp32; every warp produces pooled features j = warp, warp + 8, ... for all
-// sequences of the chunk at once (the pooler matrix row is read once per CTA), then the C_t x chunk
-// logits are warp-level dot products against the pooled vectors.
+// Pooler + head, two launches.
+//   pooler_kernel: one CTA = (64 pooled features, task, chunk of kSeqPerCta sequences).  The
+//     position-0 rows of the chunk are staged in shared memory as fp32; each warp produces 8 features
+//     for all sequences of the chunk at once (every pooler-matrix row is read once per CTA, 16-byte
+//     loads), applies tanh and writes fp32 pooled vectors to the scratch buffer [task][B][H].
+//   head_kernel: one CTA = (task, chunk); the C_t x chunk logits are warp-level dot products.
 constexpr int kSeqPerCta = 8;
 constexpr int kHeadThreads = 256;
+constexpr int kPoolFeaturesPerCta = 64;
 
-__global__ void __launch_bounds__(kHeadThreads) pooler_head_kernel(const HeadParams p) {
-  extern __shared__ float sh[];
+__global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p) {
+  extern __shared__ float cls[];  // [kSeqPerCta][H]
   const int H = p.hidden;
-  float* cls = sh;                       // [kSeqPerCta][H]
-  float* pooled = sh + kSeqPerCta * H;   // [kSeqPerCta][H]
   const HeadTask tk = p.task[blockIdx.y];
-  const int b0 = blockIdx.x * kSeqPerCta;
+  const int b0 = blockIdx.z * kSeqPerCta;
   const int nb = min(kSeqPerCta, p.batch - b0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -148,13 +149,16 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_head_kernel(const HeadPar
     float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (s < nb)
       unpack8(*reinterpret_cast<const uint4*>(tk.hidden + static_cast<size_t>(b0 + s) * p.seq * H + c * 8), f);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) cls[s * H + c * 8 + i] = f[i];
+    *reinterpret_cast<float4*>(cls + s * H + c * 8) = make_float4(f[0], f[1], f[2], f[3]);
+    *reinterpret_cast<float4*>(cls + s * H + c * 8 + 4) = make_float4(f[4], f[5], f[6], f[7]);
   }
   __syncthreads();
 
   const int vecs = H / 256;  // 16-byte vectors per lane per row
-  for (int j = warp; j < H; j += kHeadThreads / 32) {
+  float* pooled = p.pooled + static_cast<size_t>(blockIdx.y) * p.batch * H;
+  constexpr int kPerWarp = kPoolFeaturesPerCta / (kHeadThreads / 32);
+  for (int i = 0; i < kPerWarp; ++i) {
+    const int j = blockIdx.x * kPoolFeaturesPerCta + warp * kPerWarp + i;
     float acc[kSeqPerCta];
 #pragma unroll
     for (int s = 0; s < kSeqPerCta; ++s) acc[s] = 0.f;
@@ -174,15 +178,23 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_head_kernel(const HeadPar
 #pragma unroll
     for (int s = 0; s < kSeqPerCta; ++s) {
       const float t = warp_sum(acc[s]);
-      if (lane == 0) pooled[s * H + j] = tanhf(t + bias);
+      if (lane == 0 && s < nb) pooled[static_cast<size_t>(b0 + s) * H + j] = tanhf(t + bias);
     }
   }
-  __syncthreads();
+}
 
+__global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) {
+  const int H = p.hidden;
+  const HeadTask tk = p.task[blockIdx.y];
+  const int b0 = blockIdx.x * kSeqPerCta;
+  const int nb = min(kSeqPerCta, p.batch - b0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* pooled = p.pooled + static_cast<size_t>(blockIdx.y) * p.batch * H;
   for (int o = warp; o < tk.num_classes * nb; o += kHeadThreads / 32) {
     const int c = o / nb, s = o - c * nb;
     float acc = 0.f;
-    for (int k = lane; k < H; k += 32) acc += __bfloat162float(tk.cls_w[static_cast<size_t>(c) * H + k]) * pooled[s * H + k];
+    for (int k = lane; k < H; k += 32)
+      acc += __bfloat162float(tk.cls_w[static_cast<size_t>(c) * H + k]) * pooled[static_cast<size_t>(b0 + s) * H + k];
     acc = warp_sum(acc);
     if (lane == 0)
       p.logits[static_cast<size_t>(b0 + s) * p.logits_stride + tk.col0 + c] = acc + __bfloat162float(tk.cls_b[c]);
@@ -211,19 +223,15 @@ cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream) {
 }
 
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream) {
-  if (p.n_tasks < 1 || p.n_tasks > kMaxGroups || p.batch < 1 || p.hidden % 256 != 0) return cudaErrorInvalidValue;
-  const size_t smem = static_cast<size_t>(2) * kSeqPerCta * p.hidden * sizeof(float);
-  static int configured_device = -1;
-  int dev = 0;
-  cudaError_t err = cudaGetDevice(&dev);
+  if (p.n_tasks < 1 || p.n_tasks > kMaxGroups || p.batch < 1 || p.hidden % 256 != 0 || p.hidden > 1024 ||
+      p.pooled == nullptr)
+    return cudaErrorInvalidValue;
+  const size_t smem = static_cast<size_t>(kSeqPerCta) * p.hidden * sizeof(float);  // <= 32 KB
+  const int chunks = (p.batch + kSeqPerCta - 1) / kSeqPerCta;
+  pooler_kernel<<<dim3(p.hidden / kPoolFeaturesPerCta, p.n_tasks, chunks), kHeadThreads, smem, stream>>>(p);
+  cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
-  if (configured_device != dev) {
-    err = cudaFuncSetAttribute(pooler_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSeqPerCta * 1024 * 4);
-    if (err != cudaSuccess) return err;
-    configured_device = dev;
-  }
-  dim3 grid((p.batch + kSeqPerCta - 1) / kSeqPerCta, p.n_tasks);
-  pooler_head_kernel<<<grid, kHeadThreads, smem, stream>>>(p);
+  head_kernel<<<dim3(chunks, p.n_tasks), kHeadThreads, 0, stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -166,8 +166,9 @@ def test_pooler_head_matches_oracle(B, S, H, C):
     cwb, cw = rand_bf16(54, f"cw{H}.{C}", (C, H), 0.05)
     cbb, cb = rand_bf16(55, f"cb{C}", (C,), 0.1)
     logits = torch.full((B, C + 3), -77.0, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(B, H, dtype=torch.float32, device="cuda")
     mt.mt_kernel_pooler_head(to_dev_bf16(hb), to_dev_bf16(pwb), to_dev_bf16(pbb), to_dev_bf16(cwb), to_dev_bf16(cbb),
-                             logits, B, S, col0=2)
+                             scratch, logits, B, S, col0=2)
     torch.cuda.synchronize()
     got = logits.cpu().numpy().astype(np.float64)
     tw = {"pool_w": pw, "pool_b": pb, "cls_w": cw, "cls_b": cb}
