@@ -223,6 +223,28 @@ int mt_kernel_pooler_head(const void* d_hidden, const void* d_pool_w, const void
                           int32_t batch, int32_t seq, int32_t hidden, int32_t num_classes,
                           int32_t logits_stride, int32_t col0, void* stream);
 
+/* The same pooler + head for callers that cannot allocate device memory (no counterpart in the
+ * paper: it is a convenience of this library).  Meant for code that lives inside a process whose
+ * device memory is owned by someone else - an inference server that handed all of it out at start-up,
+ * a plug-in that only ever sees input and output pointers - or that must not call cudaMalloc because
+ * it stalls the device.  The tanh pooler features, which mt_kernel_pooler_head passes through
+ * d_pooled_scratch, go through an array built into the library instead: MT_STATIC_POOLER_MAX_FLOATS
+ * floats (1 MiB) that every GPU loading the library keeps until the process ends.
+ *  - batch * hidden must not exceed MT_STATIC_POOLER_MAX_FLOATS, else MT_ERR_SHAPE (nothing is launched).
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current); make that first call before starting any stream capture.
+ *  - It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *  - All calls on a device share the one array, which keeps the previous call's features (the pooler
+ *    launch overwrites every entry the head launch reads, so nothing needs clearing).  Two calls whose
+ *    kernels can overlap on the GPU - different streams, no ordering between them - race on it:
+ *    order them, or use mt_kernel_pooler_head with separate scratch buffers.
+ * All other arguments, results and errors are those of mt_kernel_pooler_head. */
+#define MT_STATIC_POOLER_MAX_FLOATS (256 * 1024)
+int mt_kernel_pooler_head_static(const void* d_hidden, const void* d_pool_w, const void* d_pool_b,
+                                 const void* d_cls_w, const void* d_cls_b, float* d_logits,
+                                 int32_t batch, int32_t seq, int32_t hidden, int32_t num_classes,
+                                 int32_t logits_stride, int32_t col0, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

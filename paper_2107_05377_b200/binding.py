@@ -58,6 +58,7 @@ SIGNATURES = {
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
                                   _P]),
     "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
+    "mt_kernel_pooler_head_static": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
 }
 
 _lib = None
@@ -135,6 +136,19 @@ def mt_kernel_pooler_head(hidden, pool_w, pool_b, cls_w, cls_b, pooled_scratch, 
                                        _ptr(pooled_scratch), _ptr(logits),
                                        batch, seq, pool_w.shape[0], cls_w.shape[0], logits.shape[1], col0,
                                        _stream(stream)), "mt_kernel_pooler_head")
+
+
+STATIC_POOLER_MAX_FLOATS = 256 * 1024
+
+
+def mt_kernel_pooler_head_static(hidden, pool_w, pool_b, cls_w, cls_b, logits, batch: int, seq: int, col0: int = 0,
+                                 stream=None) -> None:
+    """Pooler + head without a scratch argument, for callers that cannot allocate device memory:
+    the features between the two launches go through a 1 MiB array built into the library
+    (batch * hidden <= STATIC_POOLER_MAX_FLOATS).  Calls sharing a device must not overlap."""
+    _check(lib().mt_kernel_pooler_head_static(_ptr(hidden), _ptr(pool_w), _ptr(pool_b), _ptr(cls_w), _ptr(cls_b),
+                                              _ptr(logits), batch, seq, pool_w.shape[0], cls_w.shape[0],
+                                              logits.shape[1], col0, _stream(stream)), "mt_kernel_pooler_head_static")
 
 
 # ---------------------------------------------------------------------------
