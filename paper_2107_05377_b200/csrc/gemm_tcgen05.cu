@@ -13,7 +13,10 @@
 //                 instruction) with the accumulator in TMEM, and tcgen05.commit to release stages
 //   warps 2..   : epilogue - tcgen05.ld the fp32 accumulator (each warp its own 32-lane quarter),
 //                 add bias (+GELU) and round once to bf16, or add bias + fp32 residual and keep
-//                 fp32; 16-byte stores
+//                 fp32.  Each warp owns small 128-byte-swizzled staging buffers in shared memory:
+//                 results leave through TMA stores (and the fp32 residual arrives through TMA
+//                 loads, prefetched one chunk ahead), so every global access is a full 128-byte
+//                 row segment and no epilogue thread ever waits on a global load
 // The accumulator is double buffered in TMEM (2 x BN columns) so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Every output element is the sum over K in a fixed order inside a single
 // tile, so a result never depends on which other groups share the launch.
@@ -31,12 +34,16 @@ constexpr int kNumEpilogueWarps = 8;
 constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s
 
-__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 256 ? 4 : 6; }
+constexpr int kStagingBytes = 4096;  // 32 rows x 128 bytes, one epilogue chunk of one warp
+__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 256 ? 4 : 5; }
+// staging buffers per epilogue warp: two where shared memory allows (needed to prefetch residuals)
+__host__ __device__ constexpr int gemm_staging_bufs(int bn) { return bn == 256 ? 1 : 2; }
 __host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
 __host__ __device__ constexpr int gemm_b_bytes(int bn) { return bn * kGemmBlockK * 2; }
 __host__ __device__ constexpr int gemm_smem_bytes(int bn) {
-  // stages + barriers/bookkeeping + slack for manual 1024-byte alignment
-  return gemm_stages(bn) * (gemm_a_bytes() + gemm_b_bytes(bn)) + 256 + 1024;
+  // stages + staging + barriers/bookkeeping + slack for manual 1024-byte alignment
+  return gemm_stages(bn) * (gemm_a_bytes() + gemm_b_bytes(bn)) +
+         kNumEpilogueWarps * gemm_staging_bufs(bn) * kStagingBytes + 512 + 1024;
 }
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -94,6 +101,21 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+
+// Shared -> global tile store; rows/columns outside the tensor are clipped by the hardware.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until at most N of this thread's store groups still have shared memory left to read.
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// Makes this thread's shared-memory writes visible to the TMA unit.
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -164,24 +186,35 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 
 // ---- the kernel -------------------------------------------------------------------------------
 
+// Byte offset of 16-byte chunk `c` (0..7) of row `r` in a staging buffer (rows of 128 bytes,
+// 128-byte swizzle as TMA reads and writes it): threads of a quarter-warp that touch the same chunk
+// index of eight consecutive rows land in eight different bank groups.
+__device__ __forceinline__ uint32_t staging_off(int r, int c) {
+  return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4));
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __grid_constant__ GemmParams p) {
   constexpr int STAGES = gemm_stages(BN);
   constexpr int A_BYTES = gemm_a_bytes();
   constexpr int B_BYTES = gemm_b_bytes(BN);
+  constexpr int NBUF = gemm_staging_bufs(BN);
   constexpr uint32_t TMEM_COLS = 2 * BN;  // 256 or 512: a power of two >= 32
   static_assert(BN == 128 || BN == 256, "tile widths implemented: 128, 256");
+  static_assert(EPI != kEpiBiasResidual || NBUF == 2, "the residual epilogue prefetches: two staging buffers");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sA = smem_u32(smem);
   const uint32_t sB = sA + STAGES * A_BYTES;
-  uint8_t* book = smem + STAGES * (A_BYTES + B_BYTES);
+  const uint32_t sStage = sB + STAGES * B_BYTES;          // kNumEpilogueWarps x NBUF x 4 KB
+  uint8_t* book = smem + STAGES * (A_BYTES + B_BYTES) + kNumEpilogueWarps * NBUF * kStagingBytes;
   const uint32_t bar_full = smem_u32(book);               // STAGES x 8 bytes
   const uint32_t bar_empty = bar_full + 8 * STAGES;       // STAGES x 8 bytes
   const uint32_t bar_acc_full = bar_empty + 8 * STAGES;   // 2 x 8 bytes
   const uint32_t bar_acc_empty = bar_acc_full + 16;       // 2 x 8 bytes
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(book + 8 * (2 * STAGES + 4));
+  const uint32_t bar_res = bar_acc_empty + 16;            // kNumEpilogueWarps x 2 x 8 bytes
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(book + 8 * (2 * STAGES + 4 + 2 * kNumEpilogueWarps));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -202,6 +235,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       mbar_init(bar_acc_full + 8 * a, 1);
       mbar_init(bar_acc_empty + 8 * a, kNumEpilogueWarps);
     }
+    for (int i = 0; i < 2 * kNumEpilogueWarps; ++i) mbar_init(bar_res + 8 * i, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -283,86 +317,137 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     }
   } else {
     // ------------------------------ epilogue ----------------------------------
+    // A chunk is 32 rows (this warp's TMEM lanes) x 128 bytes of output: 32 fp32 columns for the
+    // residual epilogue, 64 bf16 columns otherwise.  Thread t owns row t of the chunk.
     const int e = warp - 2;
     const int quarter = warp & 3;                       // TMEM lanes this warp may read
     const int col_group = e >> 2;                       // which share of the column chunks
     constexpr int COL_GROUPS = kNumEpilogueWarps / 4;
+    constexpr int CHUNK_COLS = (EPI == kEpiBiasResidual) ? 32 : 64;
+    constexpr int CHUNKS = BN / CHUNK_COLS;
+    const uint32_t my_stage = sStage + static_cast<uint32_t>(e * NBUF * kStagingBytes);
+    const uint32_t my_res_bar = bar_res + 16 * e;       // two barriers, one per staging buffer
+    uint8_t* my_stage_ptr = smem + STAGES * (A_BYTES + B_BYTES) + e * NBUF * kStagingBytes;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    int buf = 0;                  // staging buffer of the next chunk
+    uint32_t res_phase[2] = {0, 0};
+    bool ok = true;
+
+    // (residual epilogue) asks for the residual chunk `chunk` of tile `tile` into staging buffer b
+    auto prefetch_residual = [&](int tile, int chunk, int b) {
+      const int g = tile / tiles_per_group;
+      const int local = tile - g * tiles_per_group;
+      const int row0 = (local / n_tiles_n) * kGemmBlockM + quarter * 32;
+      const int col0 = (local % n_tiles_n) * BN + chunk * CHUNK_COLS;
+      // the store issued last read this very buffer: it must be done with it before TMA refills it
+      tma_store_wait_read<0>();
+      mbar_expect_tx(my_res_bar + 8 * b, kStagingBytes);
+      tma_load_2d(my_stage + b * kStagingBytes, &p.tmap_res[g], col0, row0, my_res_bar + 8 * b);
+    };
+
+    if (EPI == kEpiBiasResidual && lane == 0 && static_cast<int>(blockIdx.x) < total_tiles)
+      prefetch_residual(blockIdx.x, col_group, 0);
+
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int g = tile / tiles_per_group;
       const int local = tile - g * tiles_per_group;
       const int m0 = (local / n_tiles_n) * kGemmBlockM;
       const int n0 = (local % n_tiles_n) * BN;
-      if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag)) break;
+      // warp-uniform decisions: the TMEM loads below are warp-collective
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag))) break;
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
-      const bool row_ok = row < p.M;
-      const GemmGroup grp = p.group[g];
-      const size_t row_off = static_cast<size_t>(row) * p.N;
+      const bf16* bias = p.group[g].bias;
+      const bool rows_in_range = m0 + quarter * 32 < p.M;
 #pragma unroll 1
-      for (int chunk = col_group; chunk < BN / 32; chunk += COL_GROUPS) {
-        uint32_t v[32];
+      for (int chunk = col_group; chunk < CHUNKS; chunk += COL_GROUPS) {
+        const int col = n0 + chunk * CHUNK_COLS;
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                               static_cast<uint32_t>(acc * BN + chunk * 32);
-        tmem_ld_32x32(taddr, v);
-        tmem_ld_wait();
-        const int col = n0 + chunk * 32;
-        const uint4* bias4 = reinterpret_cast<const uint4*>(grp.bias + col);
+                               static_cast<uint32_t>(acc * BN + chunk * CHUNK_COLS);
+        uint8_t* sbuf = my_stage_ptr + buf * kStagingBytes;
         if (EPI == kEpiBiasResidual) {
-          // fp32 residual in, fp32 out: the pre-LayerNorm sum keeps full precision
-          const float4* res4 = reinterpret_cast<const float4*>(grp.residual + row_off + col);
-          float4* dst4 = reinterpret_cast<float4*>(static_cast<float*>(grp.out) + row_off + col);
+          // prefetch the residual of the chunk after this one (next chunk of this tile, or the first
+          // chunk of this CTA's next tile) into the other buffer
+          if (lane == 0) {
+            int nt = tile, nc = chunk + COL_GROUPS;
+            if (nc >= CHUNKS) { nt = tile + gridDim.x; nc = col_group; }
+            if (nt < total_tiles) prefetch_residual(nt, nc, buf ^ 1);
+          }
+          __syncwarp();
+          uint32_t v[32];
+          tmem_ld_32x32(taddr, v);
+          tmem_ld_wait();
+          if (!__all_sync(0xffffffffu, mbar_wait(my_res_bar + 8 * buf, res_phase[buf], abort_flag))) {
+            ok = false;
+            break;
+          }
+          res_phase[buf] ^= 1u;
+          const uint4* bias4 = reinterpret_cast<const uint4*>(bias + col);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const uint4 b = __ldg(bias4 + q);
             const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-            if (row_ok) {
-              const float4 r0 = res4[2 * q], r1 = res4[2 * q + 1];
-              float4 o0, o1;
-              o0.x = __uint_as_float(v[q * 8 + 0]) + bf16_lo(bw[0]) + r0.x;
-              o0.y = __uint_as_float(v[q * 8 + 1]) + bf16_hi(bw[0]) + r0.y;
-              o0.z = __uint_as_float(v[q * 8 + 2]) + bf16_lo(bw[1]) + r0.z;
-              o0.w = __uint_as_float(v[q * 8 + 3]) + bf16_hi(bw[1]) + r0.w;
-              o1.x = __uint_as_float(v[q * 8 + 4]) + bf16_lo(bw[2]) + r1.x;
-              o1.y = __uint_as_float(v[q * 8 + 5]) + bf16_hi(bw[2]) + r1.y;
-              o1.z = __uint_as_float(v[q * 8 + 6]) + bf16_lo(bw[3]) + r1.z;
-              o1.w = __uint_as_float(v[q * 8 + 7]) + bf16_hi(bw[3]) + r1.w;
-              dst4[2 * q] = o0;
-              dst4[2 * q + 1] = o1;
-            }
+            float4* s0 = reinterpret_cast<float4*>(sbuf + staging_off(lane, 2 * q));
+            float4* s1 = reinterpret_cast<float4*>(sbuf + staging_off(lane, 2 * q + 1));
+            float4 r0 = *s0, r1 = *s1;
+            r0.x += __uint_as_float(v[q * 8 + 0]) + bf16_lo(bw[0]);
+            r0.y += __uint_as_float(v[q * 8 + 1]) + bf16_hi(bw[0]);
+            r0.z += __uint_as_float(v[q * 8 + 2]) + bf16_lo(bw[1]);
+            r0.w += __uint_as_float(v[q * 8 + 3]) + bf16_hi(bw[1]);
+            r1.x += __uint_as_float(v[q * 8 + 4]) + bf16_lo(bw[2]);
+            r1.y += __uint_as_float(v[q * 8 + 5]) + bf16_hi(bw[2]);
+            r1.z += __uint_as_float(v[q * 8 + 6]) + bf16_lo(bw[3]);
+            r1.w += __uint_as_float(v[q * 8 + 7]) + bf16_hi(bw[3]);
+            *s0 = r0;
+            *s1 = r1;
           }
         } else {
-          uint4 outv[4];
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint4 b = __ldg(bias4 + q);
-            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-            uint32_t ow[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
-              float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
-              if (EPI == kEpiBiasGelu) {
-                x0 = gelu_erf(x0);
-                x1 = gelu_erf(x1);
-              }
-              ow[j] = pack_bf16(x0, x1);
-            }
-            outv[q] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+          // the store that last read this staging buffer must be done with it
+          if (lane == 0) {
+            if (NBUF == 2) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
           }
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(grp.out) + row_off + col);
+          __syncwarp();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) dst[q] = outv[q];
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            tmem_ld_32x32(taddr + half * 32, v);
+            tmem_ld_wait();
+            const uint4* bias4 = reinterpret_cast<const uint4*>(bias + col + half * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 b = __ldg(bias4 + q);
+              const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+              uint32_t ow[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
+                float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
+                if (EPI == kEpiBiasGelu) {
+                  x0 = gelu_erf(x0);
+                  x1 = gelu_erf(x1);
+                }
+                ow[j] = pack_bf16(x0, x1);
+              }
+              *reinterpret_cast<uint4*>(sbuf + staging_off(lane, half * 4 + q)) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+            }
           }
         }
+        fence_async_shared();
+        __syncwarp();
+        if (lane == 0 && rows_in_range) {
+          tma_store_2d(&p.tmap_out[g], my_stage + buf * kStagingBytes, col, m0 + quarter * 32);
+          tma_store_commit();
+        }
+        if (NBUF == 2) buf ^= 1;
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    // shared memory must outlive the stores that still read it
+    if (lane == 0) tma_store_wait_read<0>();
+    __syncwarp();
   }
 
   // ------------------------------ teardown ------------------------------------
@@ -402,19 +487,24 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
   switch (epilogue) {
     case kEpiBias: return launch_one<BN, kEpiBias>(p, sm_count, stream);
     case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu>(p, sm_count, stream);
-    case kEpiBiasResidual: return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
+    case kEpiBiasResidual:
+      if constexpr (BN == 128) return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
+      return cudaErrorInvalidValue;  // the residual epilogue exists for 128-wide tiles only
     default: return cudaErrorInvalidValue;
   }
 }
 
 }  // namespace
 
-int gemm_block_n(int N) { return (N % 256 == 0 && N >= 2048) ? 256 : 128; }
+int gemm_block_n(int N, int epilogue) {
+  return (epilogue != kEpiBiasResidual && N % 256 == 0 && N >= 2048) ? 256 : 128;
+}
+int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
     return cudaErrorInvalidValue;
-  return gemm_block_n(p.N) == 256 ? launch_bn<256>(p, epilogue, sm_count, stream)
+  return gemm_block_n(p.N, epilogue) == 256 ? launch_bn<256>(p, epilogue, sm_count, stream)
                                   : launch_bn<128>(p, epilogue, sm_count, stream);
 }
 

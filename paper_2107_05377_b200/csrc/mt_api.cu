@@ -105,20 +105,38 @@ cudaError_t get_encoder(EncodeTiledFn* out) {
   return cudaSuccess;
 }
 
-// Tensor map of a row-major bf16 matrix [rows, cols] read in boxes of box_rows x 64 columns with
-// the 128-byte swizzle; out-of-range rows read as zero.
-cudaError_t make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+// Tensor map of a row-major matrix [rows, cols] (bf16, or fp32 when `fp32`) accessed in boxes of
+// box_rows x box_cols whose rows are 128 bytes, with the 128-byte swizzle; out-of-range parts of a
+// box read as zero and are skipped on stores.
+cudaError_t make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows, int box_cols,
+                      bool fp32) {
   EncodeTiledFn enc = nullptr;
   cudaError_t err = get_encoder(&enc);
   if (err != cudaSuccess) return err;
+  const size_t elem_bytes = fp32 ? sizeof(float) : sizeof(bf16);
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * sizeof(bf16)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kGemmBlockK), static_cast<cuuint32_t>(box_rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t elem[2] = {1, 1};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                   const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// Fills group i of a grouped GEMM Y = epi(X[M,K] . W[N,K]^T + bias (+ residual)): operand maps, the
+// output map (bf16, or fp32 for the residual epilogue) and the fp32 residual map.
+cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, const void* w, const bf16* bias,
+                           const float* residual, void* y) {
+  const int M = g->M, N = g->N, K = g->K;
+  const bool res = epilogue == kEpiBiasResidual;
+  cudaError_t e;
+  if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_block_n(N, epilogue), kGemmBlockK, false)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), res)) != cudaSuccess) return e;
+  if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
+  g->group[i].bias = bias;
+  return cudaSuccess;
 }
 
 }  // namespace
@@ -320,27 +338,26 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
 
     cudaError_t e;
     // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv]   (the three matrices and biases are contiguous in the arena)
-    if ((e = make_tmap(&ck->qkv.tmap_x[i], in, M, H, kGemmBlockM)) != cudaSuccess) return e;
-    if ((e = make_tmap(&ck->qkv.tmap_w[i], w_ptr(m, lo->wq), 3 * H, H, gemm_block_n(3 * H))) != cudaSuccess) return e;
-    ck->qkv.group[i] = {w_ptr(m, lo->bq), nullptr, qkv};
+    if ((e = set_gemm_group(&ck->qkv, i, kEpiBias, in, w_ptr(m, lo->wq), w_ptr(m, lo->bq), nullptr, qkv)) != cudaSuccess)
+      return e;
     // 2. ctx = attention(qkv)
     ck->attn.qkv[i] = qkv;
     ck->attn.ctx[i] = ctx;
     // 3. u = ctx . Wo^T + bo + in   (fp32 residual, fp32 result)
-    if ((e = make_tmap(&ck->attn_out.tmap_x[i], ctx, M, H, kGemmBlockM)) != cudaSuccess) return e;
-    if ((e = make_tmap(&ck->attn_out.tmap_w[i], w_ptr(m, lo->wo), H, H, gemm_block_n(H))) != cudaSuccess) return e;
-    ck->attn_out.group[i] = {w_ptr(m, lo->bo), f32_of(m, in), u};
+    if ((e = set_gemm_group(&ck->attn_out, i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), f32_of(m, in),
+                            u)) != cudaSuccess)
+      return e;
     // 4. h1 = LN(u)
     ck->ln1.x[i] = u; ck->ln1.gamma[i] = w_ptr(m, lo->ln1_g); ck->ln1.beta[i] = w_ptr(m, lo->ln1_b);
     ck->ln1.y[i] = h1; ck->ln1.y32[i] = f32_of(m, h1);
     // 5. f = GELU(h1 . W1^T + b1)
-    if ((e = make_tmap(&ck->ffn_up.tmap_x[i], h1, M, H, kGemmBlockM)) != cudaSuccess) return e;
-    if ((e = make_tmap(&ck->ffn_up.tmap_w[i], w_ptr(m, lo->w1), F, H, gemm_block_n(F))) != cudaSuccess) return e;
-    ck->ffn_up.group[i] = {w_ptr(m, lo->b1), nullptr, f};
+    if ((e = set_gemm_group(&ck->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
+        cudaSuccess)
+      return e;
     // 6. u = f . W2^T + b2 + h1
-    if ((e = make_tmap(&ck->ffn_down.tmap_x[i], f, M, F, kGemmBlockM)) != cudaSuccess) return e;
-    if ((e = make_tmap(&ck->ffn_down.tmap_w[i], w_ptr(m, lo->w2), H, F, gemm_block_n(H))) != cudaSuccess) return e;
-    ck->ffn_down.group[i] = {w_ptr(m, lo->b2), f32_of(m, h1), u};
+    if ((e = set_gemm_group(&ck->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), f32_of(m, h1),
+                            u)) != cudaSuccess)
+      return e;
     // 7. out = LN(u)
     ck->ln2.x[i] = u; ck->ln2.gamma[i] = w_ptr(m, lo->ln2_g); ck->ln2.beta[i] = w_ptr(m, lo->ln2_b);
     ck->ln2.y[i] = out; ck->ln2.y32[i] = f32_of(m, out);
@@ -796,9 +813,9 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
-  if (make_tmap(&p.tmap_x[0], d_x, M, K, kGemmBlockM) != cudaSuccess) return MT_ERR_CUDA;
-  if (make_tmap(&p.tmap_w[0], d_w, N, K, gemm_block_n(N)) != cudaSuccess) return MT_ERR_CUDA;
-  p.group[0] = {static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual), d_y};
+  if (set_gemm_group(&p, 0, epilogue, d_x, d_w, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
+                     d_y) != cudaSuccess)
+    return MT_ERR_CUDA;
   return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 

@@ -26,23 +26,26 @@ enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2 };
 // One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).
 // All groups of a launch share M, N, K and the epilogue.  kEpiBias and kEpiBiasGelu write bf16;
 // kEpiBiasResidual adds an fp32 residual and writes fp32 (the pre-LayerNorm sum is never rounded).
+// The output and the residual are reached through the tensor maps of GemmParams.
 struct GemmGroup {
   const bf16* bias;
-  const float* residual;  // fp32 [M,N], only read by kEpiBiasResidual
-  void* out;              // bf16 [M,N], or fp32 [M,N] for kEpiBiasResidual
 };
 
 struct alignas(64) GemmParams {
-  CUtensorMap tmap_x[kMaxGroups];  // X_g: dims {K, M}, box {64, 128}, 128-byte swizzle
-  CUtensorMap tmap_w[kMaxGroups];  // W_g: dims {K, N}, box {64, block_n}, 128-byte swizzle
+  CUtensorMap tmap_x[kMaxGroups];    // X_g: dims {K, M}, box {64, 128}, 128-byte swizzle
+  CUtensorMap tmap_w[kMaxGroups];    // W_g: dims {K, N}, box {64, block_n}, 128-byte swizzle
+  CUtensorMap tmap_out[kMaxGroups];  // Y_g: dims {N, M}, box {64 bf16 | 32 fp32, 32}, 128-byte swizzle
+  CUtensorMap tmap_res[kMaxGroups];  // residual_g (fp32): dims {N, M}, box {32, 32}; kEpiBiasResidual only
   GemmGroup group[kMaxGroups];
   int32_t n_groups;
   int32_t M, N, K;
   uint32_t* status;  // sticky device status word (may be null)
 };
 
-// Tile width along N chosen for a given N (fixed per N so results never depend on grouping).
-int gemm_block_n(int N);
+// Tile width along N chosen for a given N and epilogue (fixed, so results never depend on grouping),
+// and the width in elements of the 128-byte output box (64 bf16 or 32 fp32 columns; 32 rows).
+int gemm_block_n(int N, int epilogue);
+int gemm_out_box_cols(int epilogue);
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
 
 struct AttnParams {

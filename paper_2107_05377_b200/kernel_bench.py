@@ -21,6 +21,7 @@ import torch
 from . import binding as mt
 
 L2_FLUSH_BYTES = 256 << 20
+USE_GRAPH = False
 
 
 def _time(fn, iters, warmup, flush):
@@ -29,6 +30,21 @@ def _time(fn, iters, warmup, flush):
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
+    if USE_GRAPH and not flush:
+        # the launches are recorded once into a CUDA graph and replayed, so that the host's launch
+        # rate does not bound the measurement of short kernels
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(iters):
+                fn()
+        graph.replay()
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        graph.replay()
+        end.record()
+        torch.cuda.synchronize()
+        return start.elapsed_time(end) / iters
     if not flush:
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         start.record(stream)
@@ -102,7 +118,10 @@ def main():
     ap.add_argument("--iters", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--flush", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
     a = ap.parse_args()
+    global USE_GRAPH
+    USE_GRAPH = a.graph
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
