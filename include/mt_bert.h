@@ -160,7 +160,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
  * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
  * mt_workspace_bytes); both must be set before mt_bind_memory.  key "profile" (0/1): see
- * mt_profile_read. */
+ * mt_profile_read.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
+ * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);
 
 /* Per-launch timing.  With option "profile" = 1 (may be toggled at any time) every kernel launch of

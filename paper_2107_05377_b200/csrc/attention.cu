@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
   const int H = p.heads * kHeadDim;
   const int ld = 3 * H;
 
+  grid_dependency_wait();
+  grid_launch_dependents();
   int len = p.lengths[b];
   len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
 
@@ -246,8 +248,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1) return cudaErrorInvalidValue;
   dim3 grid((p.seq + kTileQ - 1) / kTileQ, p.heads, p.batch * p.n_groups);
-  attention_kernel<<<grid, kAttnThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(attention_kernel, grid, dim3(kAttnThreads), 0, stream, p);
 }
 
 }  // namespace mt

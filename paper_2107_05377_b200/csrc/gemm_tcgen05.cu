@@ -245,6 +245,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above touched no global data; from here on the previous kernel must have completed
+  grid_dependency_wait();
+  grid_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -478,8 +481,7 @@ cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
   const int tiles = ((p.M + kGemmBlockM - 1) / kGemmBlockM) * (p.N / BN) * p.n_groups;
   const int grid = tiles < sm_count ? tiles : sm_count;
   if (grid <= 0) return cudaSuccess;
-  kernel<<<grid, kGemmThreads, gemm_smem_bytes(BN), stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(kernel, dim3(grid), dim3(kGemmThreads), gemm_smem_bytes(BN), stream, p);
 }
 
 template <int BN>

@@ -23,6 +23,10 @@
 
 using namespace mt;
 
+namespace mt {
+bool g_use_pdl = true;
+}
+
 namespace {
 
 constexpr uint32_t kBlobMagic = 0x4D544257u;
@@ -504,6 +508,10 @@ const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c
 
 int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
+  if (strcmp(key, "pdl") == 0) {  // process-wide: programmatic dependent launch on or off
+    g_use_pdl = value != 0;
+    return MT_OK;
+  }
   if (strcmp(key, "profile") == 0) {
     m->profile = value != 0;
     m->events_used = 0;

@@ -21,6 +21,34 @@ constexpr uint32_t kFlagBadSegment = 0x2u;
 constexpr uint32_t kFlagBadLength = 0x4u;
 constexpr uint32_t kFlagWaitTimeout = 0x8u;
 
+// Programmatic dependent launch.  Every kernel of the path is launched with the "programmatic stream
+// serialization" attribute and begins with grid_dependency_wait(): it may be scheduled, and run the
+// part of its prologue that touches no global data, while the previous kernel in the stream is still
+// draining, and only proceeds once that kernel has completed and its writes are visible.  Because
+// every kernel waits (before its first global read or write), completion is transitive along the
+// stream, exactly as with ordinary stream order.  g_use_pdl = false falls back to plain launches.
+extern bool g_use_pdl;
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename Param>
+cudaError_t launch_kernel(void (*kernel)(Param), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                          const Param& param) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_use_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, param);
+}
+#endif
+
 enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2 };
 
 // One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).

@@ -76,6 +76,8 @@ __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormP
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
   const int g = blockIdx.y;
+  grid_dependency_wait();
+  grid_launch_dependents();
   if (row >= p.rows) return;
   const float* xin = p.x[g] + static_cast<size_t>(row) * H;
   float x[V][8];
@@ -95,6 +97,8 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
   constexpr int H = V * 256;
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+  grid_dependency_wait();
+  grid_launch_dependents();
   if (row >= p.batch * p.seq) return;
   const int b = row / p.seq;
   const int pos = row - b * p.seq;
@@ -143,6 +147,8 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p
   const int b0 = blockIdx.z * kSeqPerCta;
   const int nb = min(kSeqPerCta, p.batch - b0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  grid_dependency_wait();
+  grid_launch_dependents();
 
   for (int idx = threadIdx.x; idx < kSeqPerCta * (H / 8); idx += kHeadThreads) {
     const int s = idx / (H / 8), c = idx - s * (H / 8);
@@ -190,6 +196,8 @@ __global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) 
   const int nb = min(kSeqPerCta, p.batch - b0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* pooled = p.pooled + static_cast<size_t>(blockIdx.y) * p.batch * H;
+  grid_dependency_wait();
+  grid_launch_dependents();
   for (int o = warp; o < tk.num_classes * nb; o += kHeadThreads / 32) {
     const int c = o / nb, s = o - c * nb;
     float acc = 0.f;
@@ -206,20 +214,18 @@ __global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) 
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1) return cudaErrorInvalidValue;
   dim3 grid((p.rows + kRowThreads / 32 - 1) / (kRowThreads / 32), p.n_groups);
-  if (p.hidden == 768) layernorm_kernel<3><<<grid, kRowThreads, 0, stream>>>(p);
-  else if (p.hidden == 1024) layernorm_kernel<4><<<grid, kRowThreads, 0, stream>>>(p);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (p.hidden == 768) return launch_kernel(layernorm_kernel<3>, grid, dim3(kRowThreads), 0, stream, p);
+  if (p.hidden == 1024) return launch_kernel(layernorm_kernel<4>, grid, dim3(kRowThreads), 0, stream, p);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream) {
   const int rows = p.batch * p.seq;
   if (rows < 1) return cudaErrorInvalidValue;
   dim3 grid((rows + kRowThreads / 32 - 1) / (kRowThreads / 32));
-  if (p.hidden == 768) embed_kernel<3><<<grid, kRowThreads, 0, stream>>>(p);
-  else if (p.hidden == 1024) embed_kernel<4><<<grid, kRowThreads, 0, stream>>>(p);
-  else return cudaErrorInvalidValue;
-  return cudaGetLastError();
+  if (p.hidden == 768) return launch_kernel(embed_kernel<3>, grid, dim3(kRowThreads), 0, stream, p);
+  if (p.hidden == 1024) return launch_kernel(embed_kernel<4>, grid, dim3(kRowThreads), 0, stream, p);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream) {
@@ -228,11 +234,10 @@ cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream) {
     return cudaErrorInvalidValue;
   const size_t smem = static_cast<size_t>(kSeqPerCta) * p.hidden * sizeof(float);  // <= 32 KB
   const int chunks = (p.batch + kSeqPerCta - 1) / kSeqPerCta;
-  pooler_kernel<<<dim3(p.hidden / kPoolFeaturesPerCta, p.n_tasks, chunks), kHeadThreads, smem, stream>>>(p);
-  cudaError_t err = cudaGetLastError();
+  cudaError_t err = launch_kernel(pooler_kernel, dim3(p.hidden / kPoolFeaturesPerCta, p.n_tasks, chunks),
+                                  dim3(kHeadThreads), smem, stream, p);
   if (err != cudaSuccess) return err;
-  head_kernel<<<dim3(chunks, p.n_tasks), kHeadThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(head_kernel, dim3(chunks, p.n_tasks), dim3(kHeadThreads), 0, stream, p);
 }
 
 }  // namespace mt
