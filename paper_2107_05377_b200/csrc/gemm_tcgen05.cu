@@ -35,7 +35,7 @@ constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s
 
 constexpr int kStagingBytes = 4096;  // 32 rows x 128 bytes, one epilogue chunk of one warp
-__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 256 ? 4 : 5; }
+__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 128 ? 5 : 4; }
 // staging buffers per epilogue warp: two where shared memory allows (needed to prefetch residuals)
 __host__ __device__ constexpr int gemm_staging_bufs(int bn) { return bn == 256 ? 1 : 2; }
 __host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
@@ -175,7 +175,20 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
-__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+// Exact-form GELU x * Phi(x), Phi(x) = 1/2 erfc(-x / sqrt 2), with erfc evaluated branch-free by the
+// rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7, far below the bf16
+// rounding of the result): erfc(z) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-z^2), t = 1 / (1 + p z),
+// z >= 0.  The negative side uses Phi(x) = 1 - Phi(-x) without cancellation.
+__device__ __forceinline__ float gelu_erf(float x) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float half_erfc = 0.5f * poly * t * __expf(-z * z);   // Phi(-|x|)
+  return x * (x >= 0.0f ? 1.0f - half_erfc : half_erfc);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -199,8 +212,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   constexpr int A_BYTES = gemm_a_bytes();
   constexpr int B_BYTES = gemm_b_bytes(BN);
   constexpr int NBUF = gemm_staging_bufs(BN);
-  constexpr uint32_t TMEM_COLS = 2 * BN;  // 256 or 512: a power of two >= 32
-  static_assert(BN == 128 || BN == 256, "tile widths implemented: 128, 256");
+  constexpr uint32_t TMEM_COLS = BN == 128 ? 256 : 512;  // two accumulators; a power of two >= 32
+  static_assert(BN == 128 || BN == 192 || BN == 256, "tile widths implemented: 128, 192, 256");
   static_assert(EPI != kEpiBiasResidual || NBUF == 2, "the residual epilogue prefetches: two staging buffers");
 
   extern __shared__ uint8_t smem_raw[];
@@ -490,8 +503,8 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
     case kEpiBias: return launch_one<BN, kEpiBias>(p, sm_count, stream);
     case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu>(p, sm_count, stream);
     case kEpiBiasResidual:
-      if constexpr (BN == 128) return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
-      return cudaErrorInvalidValue;  // the residual epilogue exists for 128-wide tiles only
+      if constexpr (BN != 256) return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
+      return cudaErrorInvalidValue;  // no room for two staging buffers beside 256-wide stages
     default: return cudaErrorInvalidValue;
   }
 }
@@ -499,15 +512,19 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
 }  // namespace
 
 int gemm_block_n(int N, int epilogue) {
-  return (epilogue != kEpiBiasResidual && N % 256 == 0 && N >= 2048) ? 256 : 128;
+  if (epilogue != kEpiBiasResidual && N % 256 == 0 && N >= 2048) return 256;
+  return N % 192 == 0 ? 192 : 128;  // 768 = 4 x 192: 128 tiles per 4096 rows, one wave of 148 SMs
 }
 int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
     return cudaErrorInvalidValue;
-  return gemm_block_n(p.N, epilogue) == 256 ? launch_bn<256>(p, epilogue, sm_count, stream)
-                                  : launch_bn<128>(p, epilogue, sm_count, stream);
+  switch (gemm_block_n(p.N, epilogue)) {
+    case 256: return launch_bn<256>(p, epilogue, sm_count, stream);
+    case 192: return launch_bn<192>(p, epilogue, sm_count, stream);
+    default: return launch_bn<128>(p, epilogue, sm_count, stream);
+  }
 }
 
 }  // namespace mt

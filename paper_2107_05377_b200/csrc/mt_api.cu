@@ -275,10 +275,13 @@ bool build_schedule(const mt_model* m, uint64_t mask, Schedule* s) {
       if (j >= 1 && j <= c.branch_layers) s->waves[w - 1].push_back({t, j});
     }
   }
+  // Heads: a task without branch layers pools the trunk state, which lives in a ping-pong buffer, so
+  // its head runs right after the wave that produced that state; every other task keeps its final
+  // state in its own buffer and all of those heads share one launch after the last wave.
   for (int32_t t = 0; t < T; ++t) {
     if (!((mask >> t) & 1)) continue;
     const mt_task_config& c = m->tasks[t].cfg;
-    s->heads[c.fork_depth + c.branch_layers].push_back(t);
+    s->heads[c.branch_layers == 0 ? c.fork_depth : last_wave].push_back(t);
   }
   return true;
 }

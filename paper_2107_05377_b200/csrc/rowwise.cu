@@ -131,14 +131,14 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
 }
 
 // Pooler + head, two launches.
-//   pooler_kernel: one CTA = (64 pooled features, task, chunk of kSeqPerCta sequences).  The
-//     position-0 rows of the chunk are staged in shared memory as fp32; each warp produces 8 features
+//   pooler_kernel: one CTA = (32 pooled features, task, chunk of kSeqPerCta sequences).  The
+//     position-0 rows of the chunk are staged in shared memory as fp32; each warp produces 4 features
 //     for all sequences of the chunk at once (every pooler-matrix row is read once per CTA, 16-byte
 //     loads), applies tanh and writes fp32 pooled vectors to the scratch buffer [task][B][H].
 //   head_kernel: one CTA = (task, chunk); the C_t x chunk logits are warp-level dot products.
 constexpr int kSeqPerCta = 8;
 constexpr int kHeadThreads = 256;
-constexpr int kPoolFeaturesPerCta = 64;
+constexpr int kPoolFeaturesPerCta = 32;
 
 __global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p) {
   extern __shared__ float cls[];  // [kSeqPerCta][H]
@@ -163,28 +163,40 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p
   const int vecs = H / 256;  // 16-byte vectors per lane per row
   float* pooled = p.pooled + static_cast<size_t>(blockIdx.y) * p.batch * H;
   constexpr int kPerWarp = kPoolFeaturesPerCta / (kHeadThreads / 32);
-  for (int i = 0; i < kPerWarp; ++i) {
-    const int j = blockIdx.x * kPoolFeaturesPerCta + warp * kPerWarp + i;
-    float acc[kSeqPerCta];
+  const int j0 = blockIdx.x * kPoolFeaturesPerCta + warp * kPerWarp;
+  float acc[kPerWarp][kSeqPerCta];
 #pragma unroll
-    for (int s = 0; s < kSeqPerCta; ++s) acc[s] = 0.f;
-    for (int v = 0; v < vecs; ++v) {
-      const int col = (v * 32 + lane) * 8;
-      float w[8];
-      unpack8(__ldg(reinterpret_cast<const uint4*>(tk.pool_w + static_cast<size_t>(j) * H + col)), w);
+  for (int i = 0; i < kPerWarp; ++i)
 #pragma unroll
-      for (int s = 0; s < kSeqPerCta; ++s) {
-        const float4 c0 = *reinterpret_cast<const float4*>(cls + s * H + col);
-        const float4 c1 = *reinterpret_cast<const float4*>(cls + s * H + col + 4);
-        acc[s] += w[0] * c0.x + w[1] * c0.y + w[2] * c0.z + w[3] * c0.w + w[4] * c1.x + w[5] * c1.y + w[6] * c1.z +
-                  w[7] * c1.w;
-      }
-    }
-    const float bias = __bfloat162float(tk.pool_b[j]);
+    for (int s = 0; s < kSeqPerCta; ++s) acc[i][s] = 0.f;
+  for (int v = 0; v < vecs; ++v) {
+    const int col = (v * 32 + lane) * 8;
+    // this lane's 8 columns of every staged row, read once for all of the warp's features
+    float c[kSeqPerCta][8];
 #pragma unroll
     for (int s = 0; s < kSeqPerCta; ++s) {
-      const float t = warp_sum(acc[s]);
-      if (lane == 0 && s < nb) pooled[static_cast<size_t>(b0 + s) * H + j] = tanhf(t + bias);
+      const float4 c0 = *reinterpret_cast<const float4*>(cls + s * H + col);
+      const float4 c1 = *reinterpret_cast<const float4*>(cls + s * H + col + 4);
+      c[s][0] = c0.x; c[s][1] = c0.y; c[s][2] = c0.z; c[s][3] = c0.w;
+      c[s][4] = c1.x; c[s][5] = c1.y; c[s][6] = c1.z; c[s][7] = c1.w;
+    }
+#pragma unroll
+    for (int i = 0; i < kPerWarp; ++i) {
+      float w[8];
+      unpack8(__ldg(reinterpret_cast<const uint4*>(tk.pool_w + static_cast<size_t>(j0 + i) * H + col)), w);
+#pragma unroll
+      for (int s = 0; s < kSeqPerCta; ++s)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[i][s] = fmaf(w[k], c[s][k], acc[i][s]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kPerWarp; ++i) {
+    const float bias = __bfloat162float(tk.pool_b[j0 + i]);
+#pragma unroll
+    for (int s = 0; s < kSeqPerCta; ++s) {
+      const float t = warp_sum(acc[i][s]);
+      if (lane == 0 && s < nb) pooled[static_cast<size_t>(b0 + s) * H + j0 + i] = tanhf(t + bias);
     }
   }
 }
