@@ -1,0 +1,137 @@
+"""Serving sweep of the merged multi-task tree (the workloads beside the headline benchmark).
+
+    python -m paper_2107_05377_b200.sweep [--quick]
+
+One JSON line per case:
+  * the 8-task BERT-base tree at batch {1, 4, 16, 64, 256} x seq 128 (all lengths 128) with every
+    task active, a seeded random half of the tasks, and single tasks (the shallowest and the deepest
+    fork), eagerly launched and replayed from a CUDA graph;
+  * eight independent full-depth (12-layer) single-task models over the same inputs, through the same
+    library, to reproduce the paper's sharing saving (Table 2: 96 layers against the merged tree's 24);
+  * the long-sequence variant (16 x 512, lengths in [128, 512]) and the BERT-large-width tree
+    (64 x 128, lengths in [32, 128]).
+Weights are seeded random (timing does not depend on their values; the eight single-task models are
+loaded from one blob into eight separate arenas).  Inputs are resident on the device.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+
+def _dev(batch):
+    return (torch.from_numpy(batch.token_ids).cuda(), torch.from_numpy(batch.segment_ids).cuda(),
+            torch.from_numpy(batch.lengths).cuda())
+
+
+def _time_ms(fn, iters, graph):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(iters):
+            g.replay()
+        end.record()
+    else:
+        start.record()
+        for _ in range(iters):
+            fn()
+        end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / iters
+
+
+def flops_padded(cfg, layers, batch, seq):
+    m = batch * seq
+    return layers * (2.0 * m * (4 * cfg.hidden * cfg.hidden + 2 * cfg.hidden * cfg.ffn) + batch * 4.0 * cfg.hidden * seq * seq)
+
+
+def run_tree(name, cfg, blob, batch, masks, iters, out):
+    B, S = batch.token_ids.shape
+    model = binding.MTModel(cfg, B, S)
+    model.load_weights(blob)
+    tok, seg, lens = _dev(batch)
+    logits = torch.zeros(B, cfg.total_classes, dtype=torch.float32, device="cuda")
+    for label, mask in masks:
+        plan = model.plan_summary(mask)
+        fn = lambda: model.forward(tok, seg, lens, logits, task_mask=mask)  # noqa: E731
+        eager = _time_ms(fn, iters, False)
+        graph = _time_ms(fn, iters, True)
+        assert model.poll_status() == 0
+        fl = flops_padded(cfg, plan["layers"], B, S)
+        out({"case": name, "batch": B, "seq": S, "tasks": label, "mask": mask, "layers": plan["layers"],
+             "waves": plan["waves"], "launches": model.plan_launches(mask), "ms_eager": eager, "ms_graph": graph,
+             "seq_per_s_graph": 1e3 * B / graph, "tflops_padded_graph": fl / graph / 1e9,
+             "valid_fraction": float(batch.lengths.sum()) / (B * S)})
+    model.close()
+    del model
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true", help="batches {1, 32} only and no wide tree")
+    a = ap.parse_args()
+
+    def out(d):
+        print(json.dumps(d), flush=True)
+
+    cfg = synth.config_glue8()
+    weights = synth.make_weights(cfg, seed=0)
+    blob = synth.pack_weights(cfg, weights)
+    half = int(sum(1 << int(t) for t in np.random.default_rng(2).permutation(8)[:4]))
+    masks = [("all 8", 0xFF), (f"random 4 (mask {half:#04x})", half), ("task 6 (fork 4, 3 layers)", 1 << 6),
+             ("task 7 (fork 8, 2 layers)", 1 << 7)]
+    batches = (1, 32) if a.quick else (1, 4, 16, 64, 256)
+
+    # eight independent full-depth single-task models: one blob, eight arenas
+    st_cfg = synth.config_full_depth_single(cfg, 2)
+    st_w = {"emb": weights["emb"], "trunk": weights["trunk"], "tasks": [synth.make_task_weights(st_cfg, 0, seed=0)]}
+    st_blob = synth.pack_weights(st_cfg, st_w)
+
+    for B in batches:
+        batch = synth.make_batch(cfg, B, 128, 128, 128, seed=1)
+        iters = 50 if B <= 64 else 20
+        run_tree("glue8 tree", cfg, blob, batch, masks, iters, out)
+        models = [binding.MTModel(st_cfg, B, 128) for _ in range(8)]
+        for m in models:
+            m.load_weights(st_blob)
+        tok, seg, lens = _dev(batch)
+        lg = torch.zeros(B, 2, dtype=torch.float32, device="cuda")
+
+        def eight():
+            for m in models:
+                m.forward(tok, seg, lens, lg)
+
+        eager, graph = _time_ms(eight, iters, False), _time_ms(eight, iters, True)
+        out({"case": "8 independent 12-layer single-task models", "batch": B, "seq": 128, "layers": 96,
+             "launches": 8 * models[0].plan_launches(1), "ms_eager": eager, "ms_graph": graph,
+             "seq_per_s_graph": 1e3 * B / graph, "tflops_padded_graph": flops_padded(cfg, 96, B, 128) / graph / 1e9})
+        for m in models:
+            m.close()
+        del models
+
+    run_tree("glue8 tree, long sequences", cfg, blob, synth.make_batch(cfg, 16, 512, 128, 512, seed=1),
+             [("all 8", 0xFF)], 20, out)
+    run_tree("glue8 tree, headline shape", cfg, blob, synth.batch_glue8(cfg), [("all 8", 0xFF)], 50, out)
+    if not a.quick:
+        del weights, blob
+        big = synth.config_large8()
+        big_blob = synth.pack_weights(big, synth.make_weights(big, seed=0))
+        run_tree("large-width tree", big, big_blob, synth.make_batch(big, 64, 128, 32, 128, seed=1),
+                 [("all 8", 0xFF)], 20, out)
+
+
+if __name__ == "__main__":
+    main()
