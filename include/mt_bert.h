@@ -160,7 +160,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
  * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
  * mt_workspace_bytes); both must be set before mt_bind_memory.  key "profile" (0/1): see
- * mt_profile_read.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * mt_profile_read.  key "pack_tokens" (0/1, default 1, any time): store
+ * and compute only the valid tokens of every sequence (rows of sequence b follow those of b-1) instead
+ * of batch*seq padded rows; logits agree to rounding either way.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);
@@ -182,7 +184,8 @@ int mt_set_option(mt_model* m, const char* key, int64_t value);
 #define MT_NUM_CLASSES     9
 int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class);
 
-/* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out.
+/* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out (padded
+ * layout, rows at positions >= length are zero; the d_lengths of that forward must still be valid).
  * task = -1: trunk state after `layer` layers (0 = embedding output); task >= 0: state after branch
  * layer `layer` (1-based) of that task.  Requires option debug_capture = 1. */
 int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out_bf16, void* stream);

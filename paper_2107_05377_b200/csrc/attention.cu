@@ -91,11 +91,15 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
   int len = p.lengths[b];
   len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
 
-  const bf16* qkv = p.qkv[g] + static_cast<size_t>(b) * p.seq * ld + head * kHeadDim;
-  bf16* ctx = p.ctx[g] + static_cast<size_t>(b) * p.seq * H + head * kHeadDim;
-  const int rows_here = min(kTileQ, p.seq - q0);
+  const size_t row0 = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b]) : static_cast<size_t>(b) * p.seq;
+  const bf16* qkv = p.qkv[g] + row0 * ld + head * kHeadDim;
+  bf16* ctx = p.ctx[g] + row0 * H + head * kHeadDim;
+  // rows this tile may write: up to the sequence's length when packed (the next sequence follows
+  // immediately), up to the padded length otherwise
+  const int rows_here = min(kTileQ, (p.packed ? len : p.seq) - q0);
 
   if (q0 >= len) {
+    if (p.packed) return;
     // the whole query tile is padding: write zeros
     for (int idx = tid; idx < rows_here * 8; idx += kAttnThreads) {
       const int r = idx >> 3, c = idx & 7;

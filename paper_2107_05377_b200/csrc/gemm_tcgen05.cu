@@ -234,9 +234,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   const int lane = threadIdx.x & 31;
 
   const int n_tiles_n = p.N / BN;
-  const int n_tiles_m = (p.M + kGemmBlockM - 1) / kGemmBlockM;
-  const int tiles_per_group = n_tiles_m * n_tiles_n;
-  const int total_tiles = tiles_per_group * p.n_groups;
   const int k_blocks = p.K / kGemmBlockK;
 
   if (threadIdx.x == 0) {
@@ -261,6 +258,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   // everything above touched no global data; from here on the previous kernel must have completed
   grid_dependency_wait();
   grid_launch_dependents();
+  // rows in use: all M, or fewer when the token layout is packed (a device-side count)
+  int m_rows = p.M;
+  if (p.m_valid != nullptr) m_rows = min(m_rows, *p.m_valid);
+  const int n_tiles_m = (m_rows + kGemmBlockM - 1) / kGemmBlockM;
+  const int tiles_per_group = n_tiles_m * n_tiles_n;
+  const int total_tiles = tiles_per_group * p.n_groups;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -374,7 +377,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag))) break;
       tc_fence_after();
       const bf16* bias = p.group[g].bias;
-      const bool rows_in_range = m0 + quarter * 32 < p.M;
+      const bool rows_in_range = m0 + quarter * 32 < m_rows;
 #pragma unroll 1
       for (int chunk = col_group; chunk < CHUNKS; chunk += COL_GROUPS) {
         const int col = n0 + chunk * CHUNK_COLS;

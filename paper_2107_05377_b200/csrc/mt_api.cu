@@ -159,6 +159,7 @@ struct mt_model {
   // options
   int32_t max_groups;
   bool debug_capture;
+  bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
 
   // device memory (caller-owned)
   uint8_t* d_weights;
@@ -167,7 +168,8 @@ struct mt_model {
   int sm_count;
 
   // workspace layout (byte offsets)
-  size_t ws_status, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0, ws_slot0, ws_dump0;
+  size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
+      ws_slot0, ws_dump0;
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
   size_t state_bytes;  // one hidden state = its bf16 copy (GEMM operand) followed by its fp32 copy (residual)
@@ -177,6 +179,7 @@ struct mt_model {
 
   std::map<std::tuple<uint64_t, int32_t, int32_t>, Plan> plans;
   int32_t last_batch, last_seq;
+  const int32_t* last_lengths;  // device lengths of the last forward (for mt_debug_copy_hidden)
 
   // optional per-launch timing (option "profile"): event pairs recorded around every launch
   bool profile;
@@ -218,6 +221,8 @@ void layout_workspace(mt_model* m) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t at = off; off += pad256(bytes); return at; };
   m->ws_status = take(256);
+  m->ws_rows_valid = take(256);
+  m->ws_row_start = take((static_cast<size_t>(m->max_batch) + 1) * 4);
   m->ws_tok = take(M * 4);
   m->ws_seg = take(M * 4);
   m->ws_len = take(static_cast<size_t>(m->max_batch) * 4);
@@ -306,6 +311,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     memset(g, 0, sizeof(*g));
     g->n_groups = static_cast<int32_t>(count);
     g->M = M; g->N = N; g->K = K;
+    g->m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
     g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   };
   init_gemm(&ck->qkv, 3 * H, H);
@@ -318,6 +324,9 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   ck->attn.n_groups = ck->ln1.n_groups = ck->ln2.n_groups = static_cast<int32_t>(count);
   ck->attn.batch = batch; ck->attn.seq = seq; ck->attn.heads = m->trunk.heads;
   ck->attn.lengths = nullptr;  // patched per call
+  ck->attn.row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
+  ck->attn.packed = m->pack_tokens ? 1 : 0;
+  ck->ln1.rows_valid = ck->ln2.rows_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->ln1.rows = ck->ln2.rows = M;
   ck->ln1.hidden = ck->ln2.hidden = H;
   ck->ln1.eps = ck->ln2.eps = m->trunk.ln_eps;
@@ -376,7 +385,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
 
 cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
   plan->steps.clear();
-  plan->launches = 1;  // embedding
+  plan->launches = 2;  // row starts, embedding
   auto add_heads = [&](const std::vector<int32_t>& tasks) {
     for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
       const size_t count = std::min<size_t>(kMaxGroups, tasks.size() - first);
@@ -387,6 +396,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       st.heads.batch = batch; st.heads.seq = seq; st.heads.hidden = m->trunk.hidden;
       st.heads.logits_stride = m->c_total;
       st.heads.pooled = reinterpret_cast<float*>(m->d_workspace + m->ws_pooled);
+      st.heads.row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
       for (size_t i = 0; i < count; ++i) {
         const int32_t t = tasks[first + i];
         const TaskEntry& te = m->tasks[t];
@@ -451,6 +461,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->max_seq = max_seq;
   m->max_groups = kMaxGroups;
   m->debug_capture = false;
+  m->pack_tokens = true;
+  m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
   m->sm_count = 0;
@@ -513,6 +525,11 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
   if (strcmp(key, "pdl") == 0) {  // process-wide: programmatic dependent launch on or off
     g_use_pdl = value != 0;
+    return MT_OK;
+  }
+  if (strcmp(key, "pack_tokens") == 0) {
+    m->pack_tokens = value != 0;
+    m->plans.clear();
     return MT_OK;
   }
   if (strcmp(key, "profile") == 0) {
@@ -629,7 +646,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
   if (m == nullptr || n_launches == nullptr) return MT_ERR_INVALID_ARG;
   Schedule s;
   if (!build_schedule(m, task_mask, &s)) return fail(m, MT_ERR_INVALID_ARG, "task_mask selects no task");
-  int32_t n = 1;
+  int32_t n = 2;  // row starts, embedding
   for (size_t w = 0; w <= s.waves.size(); ++w) {
     if (w >= 1) n += 7 * static_cast<int32_t>((s.waves[w - 1].size() + m->n_slots - 1) / m->n_slots);
     n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
@@ -692,7 +709,13 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
     }                                                                                        \
   } while (0)
 
+  int32_t* row_start = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_row_start);
+  MT_LAUNCH(launch_row_starts(d_lengths, batch, seq, m->pack_tokens ? 1 : 0, row_start,
+                              reinterpret_cast<int32_t*>(m->d_workspace + m->ws_rows_valid), stream),
+            "row-start kernel");
   EmbedParams ep;
+  ep.row_start = row_start;
+  ep.packed = m->pack_tokens ? 1 : 0;
   ep.token_ids = d_token_ids; ep.segment_ids = d_segment_ids; ep.lengths = d_lengths;
   ep.word = w_ptr(m, m->emb_word); ep.pos = w_ptr(m, m->emb_pos); ep.type = w_ptr(m, m->emb_type);
   ep.gamma = w_ptr(m, m->emb_ln_g); ep.beta = w_ptr(m, m->emb_ln_b);
@@ -729,6 +752,7 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
 #undef MT_LAUNCH
   m->last_batch = batch;
   m->last_seq = seq;
+  m->last_lengths = d_lengths;
   return MT_OK;
 }
 
@@ -803,9 +827,11 @@ int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out, 
   if (task < -1 || task >= T) return fail(m, MT_ERR_INVALID_ARG, "task out of range");
   if (task < 0 ? (layer < 0 || layer > m->trunk.trunk_layers) : (layer < 1 || layer > m->tasks[task].cfg.branch_layers))
     return fail(m, MT_ERR_INVALID_ARG, "layer out of range");
-  const size_t bytes = static_cast<size_t>(m->last_batch) * m->last_seq * m->trunk.hidden * sizeof(bf16);
-  cudaError_t e = cudaMemcpyAsync(d_out, m->d_workspace + m->ws_dump0 + m->act_bytes * dump_slot(m, task, layer), bytes,
-                                  cudaMemcpyDeviceToDevice, as_stream(stream_));
+  // the captured state is in the layout of the forward (packed or padded): hand it back padded
+  cudaError_t e = launch_unpack_rows(
+      reinterpret_cast<const bf16*>(m->d_workspace + m->ws_dump0 + m->act_bytes * dump_slot(m, task, layer)),
+      m->last_lengths, reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start),
+      static_cast<bf16*>(d_out), m->last_batch, m->last_seq, m->trunk.hidden, as_stream(stream_));
   if (e != cudaSuccess) return fail_cuda(m, e, "copying a captured hidden state");
   return MT_OK;
 }
@@ -873,6 +899,8 @@ int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, co
   p.out32 = static_cast<float*>(d_h0_f32);
   p.batch = batch; p.seq = seq; p.hidden = hidden; p.vocab = vocab; p.type_vocab = type_vocab; p.eps = eps;
   p.status = d_status;
+  p.row_start = nullptr;
+  p.packed = 0;
   return launch_embed(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 

@@ -67,7 +67,8 @@ struct alignas(64) GemmParams {
   GemmGroup group[kMaxGroups];
   int32_t n_groups;
   int32_t M, N, K;
-  uint32_t* status;  // sticky device status word (may be null)
+  const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
+  uint32_t* status;        // sticky device status word (may be null)
 };
 
 // Tile width along N chosen for a given N and epilogue (fixed, so results never depend on grouping),
@@ -76,10 +77,15 @@ int gemm_block_n(int N, int epilogue);
 int gemm_out_box_cols(int epilogue);
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
 
+// Token layout.  The rows of sequence b start at row_start[b] (device array of batch + 1 ints written
+// by launch_row_starts: b * seq for the padded layout, the running sum of the lengths for the packed
+// layout, in which only valid tokens exist).  A null row_start means the padded layout.
 struct AttnParams {
-  const bf16* qkv[kMaxGroups];  // [B*S, 3*H] = [Q | K | V]
-  bf16* ctx[kMaxGroups];        // [B*S, H]
+  const bf16* qkv[kMaxGroups];  // [rows, 3*H] = [Q | K | V]
+  bf16* ctx[kMaxGroups];        // [rows, H]
   const int32_t* lengths;       // [B]
+  const int32_t* row_start;     // [B + 1] or null
+  int32_t packed;               // 1: no padded rows exist, nothing is written beyond a sequence's length
   int32_t n_groups, batch, seq, heads;
 };
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
@@ -93,6 +99,7 @@ struct LayerNormParams {
   bf16* y[kMaxGroups];
   float* y32[kMaxGroups];
   int32_t n_groups, rows, hidden;
+  const int32_t* rows_valid;  // device scalar: rows actually in use (<= rows); null = all
   float eps;
 };
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream);
@@ -104,6 +111,8 @@ struct EmbedParams {
   const bf16 *word, *pos, *type, *gamma, *beta;
   bf16* out;
   float* out32;  // may be null
+  const int32_t* row_start;  // [B + 1] or null (padded layout)
+  int32_t packed;            // 1: positions >= length are skipped
   int32_t batch, seq, hidden, vocab, type_vocab;
   float eps;
   uint32_t* status;
@@ -111,7 +120,7 @@ struct EmbedParams {
 cudaError_t launch_embed(const EmbedParams& p, cudaStream_t stream);
 
 struct HeadTask {
-  const bf16* hidden;  // final state of the task, [B*S, H]; row b*S is pooled
+  const bf16* hidden;  // final state of the task, [rows, H]; the first row of every sequence is pooled
   const bf16 *pool_w, *pool_b, *cls_w, *cls_b;
   int32_t num_classes, col0;
 };
@@ -119,8 +128,17 @@ struct HeadParams {
   HeadTask task[kMaxGroups];
   float* logits;
   float* pooled;  // scratch, fp32 [n_tasks][batch][hidden]: tanh pooler outputs between the two launches
+  const int32_t* row_start;  // [B + 1] or null (padded layout: sequence b starts at row b * seq)
   int32_t n_tasks, batch, seq, hidden, logits_stride;
 };
+
+// row_start[b] for b = 0..batch and *rows_valid = row_start[batch]: b * seq (padded) or the running sum
+// of the lengths clamped to [1, seq] (packed).
+cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,
+                              int32_t* rows_valid, cudaStream_t stream);
+// padded[b*seq + pos] = packed[row_start[b] + pos] for pos < length, 0 elsewhere (bf16 rows of `hidden`).
+cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const int32_t* row_start, bf16* padded,
+                               int32_t batch, int32_t seq, int32_t hidden, cudaStream_t stream);
 // Two launches: pooler (tanh features into `pooled`), then head (logits).
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream);
 

@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormP
   const int g = blockIdx.y;
   grid_dependency_wait();
   grid_launch_dependents();
-  if (row >= p.rows) return;
+  if (row >= p.rows || (p.rows_valid != nullptr && row >= *p.rows_valid)) return;
   const float* xin = p.x[g] + static_cast<size_t>(row) * H;
   float x[V][8];
 #pragma unroll
@@ -112,6 +112,13 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
     if (len < 1 || len > p.seq) flags |= kFlagBadLength;
   }
   if (flags != 0 && lane == 0 && p.status != nullptr) atomicOr(p.status, flags);
+  int out_row = row;
+  if (p.row_start != nullptr) {
+    int len = p.lengths[b];
+    len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
+    if (p.packed && pos >= len) return;  // packed layout: padded positions do not exist
+    out_row = p.row_start[b] + pos;
+  }
   const bf16* w = p.word + static_cast<size_t>(tok) * H;
   const bf16* q = p.pos + static_cast<size_t>(pos) * H;
   const bf16* t = p.type + static_cast<size_t>(seg) * H;
@@ -126,8 +133,8 @@ __global__ void __launch_bounds__(kRowThreads) embed_kernel(const EmbedParams p)
 #pragma unroll
     for (int i = 0; i < 8; ++i) x[v][i] = a[i] + c[i] + d[i];
   }
-  float* out32 = p.out32 != nullptr ? p.out32 + static_cast<size_t>(row) * H : nullptr;
-  normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(row) * H, out32, lane, p.eps);
+  float* out32 = p.out32 != nullptr ? p.out32 + static_cast<size_t>(out_row) * H : nullptr;
+  normalise_store<V>(x, p.gamma, p.beta, p.out + static_cast<size_t>(out_row) * H, out32, lane, p.eps);
 }
 
 // Pooler + head, two launches.
@@ -153,8 +160,11 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p
   for (int idx = threadIdx.x; idx < kSeqPerCta * (H / 8); idx += kHeadThreads) {
     const int s = idx / (H / 8), c = idx - s * (H / 8);
     float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (s < nb)
-      unpack8(*reinterpret_cast<const uint4*>(tk.hidden + static_cast<size_t>(b0 + s) * p.seq * H + c * 8), f);
+    if (s < nb) {
+      const size_t row = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b0 + s])
+                                                : static_cast<size_t>(b0 + s) * p.seq;
+      unpack8(*reinterpret_cast<const uint4*>(tk.hidden + row * H + c * 8), f);
+    }
     *reinterpret_cast<float4*>(cls + s * H + c * 8) = make_float4(f[0], f[1], f[2], f[3]);
     *reinterpret_cast<float4*>(cls + s * H + c * 8 + 4) = make_float4(f[4], f[5], f[6], f[7]);
   }
@@ -221,7 +231,70 @@ __global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) 
   }
 }
 
+// One warp: inclusive scan of the clamped lengths in chunks of 32.
+__global__ void row_starts_kernel(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed,
+                                  int32_t* row_start, int32_t* rows_valid) {
+  const int lane = threadIdx.x;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  int carry = 0;
+  for (int base = 0; base < batch; base += 32) {
+    const int b = base + lane;
+    int n = 0;
+    if (b < batch) {
+      n = seq;
+      if (packed) {
+        n = lengths[b];
+        n = n < 1 ? 1 : (n > seq ? seq : n);
+      }
+    }
+    int incl = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (b < batch) row_start[b] = carry + incl - n;
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) {
+    row_start[batch] = carry;
+    *rows_valid = carry;
+  }
+}
+
+// One warp per padded row.
+__global__ void __launch_bounds__(kRowThreads) unpack_rows_kernel(const bf16* packed, const int32_t* lengths,
+                                                                   const int32_t* row_start, bf16* padded, int32_t batch,
+                                                                   int32_t seq, int32_t hidden) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+  if (row >= batch * seq) return;
+  const int b = row / seq, pos = row - b * seq;
+  int len = lengths[b];
+  len = len < 1 ? 1 : (len > seq ? seq : len);
+  const uint4* src = reinterpret_cast<const uint4*>(packed + static_cast<size_t>(row_start[b] + pos) * hidden);
+  uint4* dst = reinterpret_cast<uint4*>(padded + static_cast<size_t>(row) * hidden);
+  for (int c = lane; c < hidden / 8; c += 32) dst[c] = pos < len ? src[c] : make_uint4(0, 0, 0, 0);
+}
+
 }  // namespace
+
+cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,
+                              int32_t* rows_valid, cudaStream_t stream) {
+  if (batch < 1 || seq < 1) return cudaErrorInvalidValue;
+  row_starts_kernel<<<1, 32, 0, stream>>>(lengths, batch, seq, packed, row_start, rows_valid);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const int32_t* row_start, bf16* padded,
+                               int32_t batch, int32_t seq, int32_t hidden, cudaStream_t stream) {
+  const int rows = batch * seq;
+  if (rows < 1 || hidden % 8 != 0) return cudaErrorInvalidValue;
+  unpack_rows_kernel<<<(rows + kRowThreads / 32 - 1) / (kRowThreads / 32), kRowThreads, 0, stream>>>(
+      packed, lengths, row_start, padded, batch, seq, hidden);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1) return cudaErrorInvalidValue;

@@ -16,9 +16,11 @@ HIDDEN_REL_L2 = 1e-2   # tolerance on hidden states (valid rows)
 LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
-def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None):
+def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
+    if pack_tokens is not None:
+        model.set_option("pack_tokens", pack_tokens)
     model.load_weights(blob)
     tok, seg, lens = dev_batch(batch)
     logits = torch.full((B, cfg.total_classes), float("nan") if fill is None else fill, dtype=torch.float32,
@@ -75,6 +77,19 @@ def test_ragged_batch_random_affine_matches_oracle():
                         batch.lengths)
     model, logits = run_model(cfg, blob, batch, debug=True)
     check_against_oracle(cfg, wf, batch, model, logits, rows=range(5))
+
+
+def test_padded_layout_matches_oracle_and_packed_layout():
+    """The same forward with all batch*seq padded rows computed (pack_tokens = 0): parity with the
+    oracle everywhere, and the same logits as the default packed layout."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
+    model, padded = run_model(cfg, blob, batch, debug=True, pack_tokens=0)
+    check_against_oracle(cfg, wf, batch, model, padded, rows=range(6))
+    _, packed = run_model(cfg, blob, batch)
+    assert float((packed - padded).abs().max()) <= 1e-3
 
 
 def test_merged_equals_standalone_students_bit_exact():

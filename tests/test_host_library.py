@@ -71,11 +71,11 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
         assert m.plan_summary(mask)["layers"] == want
     with pytest.raises(binding.MTError):
         m.plan_summary(0)
-    assert m.plan_launches(0xFF) == 1 + 7 * 10 + 2   # embedding, 7 per wave, one pooler + head launch at the end
+    assert m.plan_launches(0xFF) == 2 + 7 * 10 + 2   # row starts + embedding, 7 per wave, pooler + head at the end
     m.close()
     m2 = binding.MTModel(cfg, 32, 128, max_groups=2, bind=False)
     assert m2.plan_summary(0xFF)["layers"] == 24
-    assert m2.plan_launches(0xFF) == 1 + 7 * (1 + 1 + 1 + 1 + 1 + 2 + 3 + 3 + 2 + 1) + 2
+    assert m2.plan_launches(0xFF) == 2 + 7 * (1 + 1 + 1 + 1 + 1 + 2 + 3 + 3 + 2 + 1) + 2
     m2.close()
 
 
