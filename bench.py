@@ -133,6 +133,23 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_throughput(world, sequences_per_rank_step, steps, seconds):
+    """Whole-job sequences/s: every rank processed the same number of sequences (replicas), the job
+    took as long as its slowest rank."""
+    return world * sequences_per_rank_step * steps / seconds
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -259,10 +276,7 @@ def main():
     model.set_option("profile", 0)
     clocks = sampler.stop() if sampler else None
 
-    if distributed:
-        t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_s = float(t[0]), float(t[1])
+    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], device)
 
     if rank == 0:
         peaks = measured_peaks()
@@ -283,7 +297,7 @@ def main():
         valid_flops = gemm_flops + sum(
             plan["layers"] * 4.0 * cfg.hidden * float((batches[i % N_INPUT_BATCHES].lengths.astype(np.float64) ** 2).sum())
             for i in range(args.steps))
-        value = world * BATCH * args.steps / (total_ms * 1e-3)
+        value = aggregate_throughput(world, BATCH, args.steps, total_ms * 1e-3)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -297,7 +311,7 @@ def main():
                        "token_layout": "packed (valid tokens only)",
                        "valid_tokens_per_step": valid_tokens, "padded_tokens_per_step": m_rows},
             "gpu_launches": launches_per_step * args.steps,
-            "e2e": {"value": world * BATCH * args.steps / e2e_s, "unit": UNIT,
+            "e2e": {"value": aggregate_throughput(world, BATCH, args.steps, e2e_s), "unit": UNIT,
                     "h2d_bytes_per_step": 2 * BATCH * SEQ * 4 + BATCH * 4,
                     "d2h_bytes_per_step": BATCH * cfg.total_classes * 4},
             "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches)",

@@ -4,8 +4,9 @@
 // exactly 0 (their K/V rows are never read: zero-filled in shared memory), query rows >= length
 // are written as 0, so padded rows stay finite and deterministic whatever they contained.
 //
-// One CTA = 64 query rows of one (group, sequence, head); 4 warps x 16 rows.  Keys are visited in
-// tiles of 64 with an online softmax (running row maximum and sum in fp32, reduced across the four
+// One CTA = 64 query rows of one (group, sequence, head); 4 warps x 16 rows, five CTAs per SM.  Keys
+// are visited in tiles of 64 (double buffered: tile t+1 is fetched while tile t is used, and V of a
+// tile may still be in flight while its scores are computed) with an online softmax (running row maximum and sum in fp32, reduced across the four
 // lanes that share a row with warp shuffles).  Q, K, V tiles are staged in shared memory with
 // 16-byte cp.async copies into an XOR-swizzled layout and fed to the tensor cores through ldmatrix
 // (mma.sync m16n8k16, bf16 inputs, fp32 accumulate); the probabilities are rounded to bf16 for the
@@ -29,7 +30,8 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool 
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_pending() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -70,11 +72,12 @@ __device__ __forceinline__ void load_tile(uint32_t smem_tile, const bf16* base, 
   }
 }
 
-__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParams p) {
-  __shared__ __align__(128) uint8_t smem[3 * kTileQ * 128];
+__global__ void __launch_bounds__(kAttnThreads, 5) attention_kernel(const AttnParams p) {
+  // Q tile, then two buffers of (K tile, V tile): the keys of tile t+1 are fetched while tile t is used
+  __shared__ __align__(128) uint8_t smem[(kTileQ + 4 * kTileK) * 128];
   const uint32_t sQ = smem_u32(smem);
-  const uint32_t sK = sQ + kTileQ * 128;
-  const uint32_t sV = sK + kTileK * 128;
+  const uint32_t sKV = sQ + kTileQ * 128;
+  constexpr uint32_t kBufBytes = 2 * kTileK * 128;
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -108,7 +111,11 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
     return;
   }
 
+  // copy groups, in order: {Q, K0}, {V0}, then {K(t+1)}, {V(t+1)} issued while tile t is being used
   load_tile(sQ, qkv, ld, q0, len, tid);
+  load_tile(sKV, qkv + H, ld, 0, len, tid);
+  cp_async_commit();
+  load_tile(sKV + kTileK * 128, qkv + 2 * H, ld, 0, len, tid);
   cp_async_commit();
 
   float o[8][4];
@@ -123,12 +130,22 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
   const int n_key_tiles = (len + kTileK - 1) / kTileK;
   for (int kt = 0; kt < n_key_tiles; ++kt) {
     const int k0 = kt * kTileK;
-    if (kt > 0) __syncthreads();  // everyone is done reading the previous K/V tile
-    load_tile(sK, qkv + H, ld, k0, len, tid);
-    load_tile(sV, qkv + 2 * H, ld, k0, len, tid);
-    cp_async_commit();
-    cp_async_wait_all();
+    const uint32_t sK = sKV + (kt & 1) * kBufBytes;
+    const uint32_t sV = sK + kTileK * 128;
+    // K of this tile (and Q) have landed once at most one newer group (this tile's V) is pending;
+    // the barrier also means every warp is done with the previous tile, whose buffer is refilled next
+    cp_async_wait_pending<1>();
     __syncthreads();
+    if (kt + 1 < n_key_tiles) {
+      const uint32_t nK = sKV + ((kt + 1) & 1) * kBufBytes;
+      load_tile(nK, qkv + H, ld, k0 + kTileK, len, tid);
+      cp_async_commit();
+      load_tile(nK + kTileK * 128, qkv + 2 * H, ld, k0 + kTileK, len, tid);
+      cp_async_commit();
+    } else {
+      cp_async_commit();  // empty groups keep the pending-group arithmetic uniform
+      cp_async_commit();
+    }
 
     if (kt == 0) {
       // Q fragments: 16 rows of this warp x 64 dims = four k-steps of 16
@@ -200,6 +217,9 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
       o[n][2] *= corr[1]; o[n][3] *= corr[1];
     }
 
+    // V of this tile has landed once only the two groups of the next tile are pending
+    cp_async_wait_pending<2>();
+    __syncthreads();
     // O += P V : k = keys (four steps of 16), n = 64 dims (eight n-tiles)
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
@@ -224,6 +244,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const AttnParam
   }
   const float inv0 = 1.f / l_run[0];
   const float inv1 = 1.f / l_run[1];
+  cp_async_wait_pending<0>();  // only empty groups can be left
   __syncwarp();
   uint8_t* sQg = smem;
 #pragma unroll
