@@ -4,7 +4,7 @@
 // exactly 0 (their K/V rows are never read: zero-filled in shared memory), query rows >= length
 // are written as 0, so padded rows stay finite and deterministic whatever they contained.
 //
-// One CTA = 64 query rows of one (group, sequence, head); 4 warps x 16 rows, five CTAs per SM.  Keys
+// One CTA = 64 query rows of one (group, sequence, head); 4 warps x 16 rows, four CTAs per SM.  Keys
 // are visited in tiles of 64 (double buffered: tile t+1 is fetched while tile t is used, and V of a
 // tile may still be in flight while its scores are computed) with an online softmax (running row maximum and sum in fp32, reduced across the four
 // lanes that share a row with warp shuffles).  Q, K, V tiles are staged in shared memory with
@@ -72,7 +72,7 @@ __device__ __forceinline__ void load_tile(uint32_t smem_tile, const bf16* base, 
   }
 }
 
-__global__ void __launch_bounds__(kAttnThreads, 5) attention_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kAttnThreads, 4) attention_kernel(const AttnParams p) {
   // Q tile, then two buffers of (K tile, V tile): the keys of tile t+1 are fetched while tile t is used
   __shared__ __align__(128) uint8_t smem[(kTileQ + 4 * kTileK) * 128];
   const uint32_t sQ = smem_u32(smem);
@@ -157,11 +157,20 @@ __global__ void __launch_bounds__(kAttnThreads, 5) attention_kernel(const AttnPa
       }
     }
 
+    // Work is skipped at the granularity of the tensor-core fragments: a warp whose 16 query rows are
+    // all padding computes nothing, n-tiles (8 keys) and k-steps (16 keys) beyond the length are
+    // not multiplied.  All conditions are warp-uniform.
+    const bool warp_has_rows = q0 + warp * 16 < len;
+    const int keys_here = min(kTileK, len - k0);
+    const int n_used = warp_has_rows ? (keys_here + 7) >> 3 : 0;
+    const int ks_used = warp_has_rows ? (keys_here + 15) >> 4 : 0;
+
     // S = Q K^T : 16 x 64 per warp = eight n-tiles of 8 keys
     float s[8][4];
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
       s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+      if (n >= n_used) continue;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         // four 8x8 blocks of K rows (keys n*8..n*8+7), dims half*32 + {0,8,16,24}
@@ -223,6 +232,7 @@ __global__ void __launch_bounds__(kAttnThreads, 5) attention_kernel(const AttnPa
     // O += P V : k = keys (four steps of 16), n = 64 dims (eight n-tiles)
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
+      if (ks >= ks_used) continue;
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         // V rows ks*16 .. +15, dims np*16 .. +15, transposed on load
