@@ -160,7 +160,10 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
  * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
  * mt_workspace_bytes); both must be set before mt_bind_memory.  key "profile" (0/1): see
- * mt_profile_read.  key "pack_tokens" (0/1, default 1, any time): store
+ * mt_profile_read.  key "cls_only_last_layer" (0/1, default 1, any time): the last
+ * layer of every task branch is evaluated for the first token of each sequence only (keys and values
+ * still for all tokens) because the pooler reads nothing else; mt_debug_copy_hidden then returns that
+ * layer's state at position 0 and zeros elsewhere.  key "pack_tokens" (0/1, default 1, any time): store
  * and compute only the valid tokens of every sequence (rows of sequence b follow those of b-1) instead
  * of batch*seq padded rows; logits agree to rounding either way.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's

@@ -278,7 +278,107 @@ __global__ void __launch_bounds__(kAttnThreads, 4) attention_kernel(const AttnPa
   }
 }
 
+// First-token attention: one warp = one (sequence, head).  Lanes split the keys for the scores
+// (each lane a whole 128-byte K row per key), then split the 64 output dimensions for the weighted
+// sum of V rows, the probability of each key being broadcast from the lane that owns it.  fp32
+// throughout; only the output is rounded to bf16.
+constexpr int kClsWarps = 4;
+constexpr int kClsMaxKeysPerLane = 16;  // sequences of up to 512 keys
+
+__global__ void __launch_bounds__(kClsWarps * 32) cls_attention_kernel(const ClsAttnParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int head = blockIdx.x * kClsWarps + warp;
+  const int b = blockIdx.y, g = blockIdx.z;
+  const int H = p.heads * kHeadDim, ld = 3 * H;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  int len = p.lengths[b];
+  len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
+  const size_t row0 = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b]) : static_cast<size_t>(b) * p.seq;
+
+  // the block's share of the residual row: kClsWarps heads x 64 columns
+  {
+    const int col = blockIdx.x * kClsWarps * kHeadDim + threadIdx.x * 2;
+    if (col < H) {
+      const float2 r = *reinterpret_cast<const float2*>(p.in32[g] + row0 * H + col);
+      *reinterpret_cast<float2*>(p.res[g] + static_cast<size_t>(b) * H + col) = r;
+    }
+  }
+  if (head >= p.heads) return;
+
+  const bf16* base = p.qkv[g] + row0 * ld + head * kHeadDim;
+  float q[kHeadDim];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(base) + c);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      q[c * 8 + 2 * i] = __uint_as_float(w[i] << 16);
+      q[c * 8 + 2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  float sc[kClsMaxKeysPerLane];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < kClsMaxKeysPerLane; ++i) {
+    const int j = i * 32 + lane;
+    sc[i] = -INFINITY;
+    if (j < len) {
+      const uint4* krow = reinterpret_cast<const uint4*>(base + static_cast<size_t>(j) * ld + H);
+      float acc = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 u = krow[c];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          acc = fmaf(q[c * 8 + 2 * t], __uint_as_float(w[t] << 16), acc);
+          acc = fmaf(q[c * 8 + 2 * t + 1], __uint_as_float(w[t] & 0xFFFF0000u), acc);
+        }
+      }
+      sc[i] = acc;
+      mx = fmaxf(mx, acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  const float scale_log2 = 0.125f * 1.4426950408889634f;
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < kClsMaxKeysPerLane; ++i) {
+    sc[i] = exp2f((sc[i] - mx) * scale_log2);   // 0 for keys beyond the length
+    sum += sc[i];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+
+  float o0 = 0.f, o1 = 0.f;
+  const bf16* vbase = base + 2 * H + 2 * lane;
+#pragma unroll
+  for (int i = 0; i < kClsMaxKeysPerLane; ++i) {
+    if (i * 32 >= len) break;   // warp-uniform
+    const int n = min(32, len - i * 32);
+    for (int jj = 0; jj < n; ++jj) {
+      const float pj = __shfl_sync(0xffffffffu, sc[i], jj);
+      const uint32_t v = *reinterpret_cast<const uint32_t*>(vbase + static_cast<size_t>(i * 32 + jj) * ld);
+      o0 = fmaf(pj, __uint_as_float(v << 16), o0);
+      o1 = fmaf(pj, __uint_as_float(v & 0xFFFF0000u), o1);
+    }
+  }
+  const float inv = 1.f / sum;
+  *reinterpret_cast<uint32_t*>(p.ctx[g] + static_cast<size_t>(b) * H + head * kHeadDim + 2 * lane) =
+      pack_bf16(o0 * inv, o1 * inv);
+}
+
 }  // namespace
+
+cudaError_t launch_cls_attention(const ClsAttnParams& p, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1 || p.seq > 32 * kClsMaxKeysPerLane)
+    return cudaErrorInvalidValue;
+  dim3 grid((p.heads + kClsWarps - 1) / kClsWarps, p.batch, p.n_groups);
+  return launch_kernel(cls_attention_kernel, grid, dim3(kClsWarps * 32), 0, stream, p);
+}
 
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1) return cudaErrorInvalidValue;

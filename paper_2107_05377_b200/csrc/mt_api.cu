@@ -72,11 +72,26 @@ struct Schedule {
 
 // ---- bound plan (device pointers, tensor maps) --------------------------------------------------
 
-struct Chunk {
-  GemmParams qkv, attn_out, ffn_up, ffn_down;
-  AttnParams attn;
+// Everything of a layer after the QKV projection, for a set of layers that share the row count.
+struct LayerTail {
+  GemmParams attn_out, ffn_up, ffn_down;
   LayerNormParams ln1, ln2;
-  std::vector<std::pair<const bf16*, int32_t>> dumps;  // (layer output, dump slot)
+  int32_t count = 0;
+};
+struct DumpCopy {
+  const bf16* src;
+  int32_t slot;
+  bool compact;  // [B, H]: first tokens only
+};
+// One chunk of a wave: the QKV projection of all its layers in one launch, then the rest of the
+// layer for the layers computed on every token (`full`) and for the last layers of task branches,
+// which are computed for the first token of every sequence only (`cls`).
+struct Chunk {
+  GemmParams qkv;
+  AttnParams attn;
+  ClsAttnParams attn_cls;
+  LayerTail full, cls;
+  std::vector<DumpCopy> dumps;
 };
 struct PlanStep {
   int kind;  // 0 = chunk, 1 = heads
@@ -160,6 +175,7 @@ struct mt_model {
   int32_t max_groups;
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
+  bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
 
   // device memory (caller-owned)
   uint8_t* d_weights;
@@ -235,7 +251,9 @@ void layout_workspace(mt_model* m) {
   off += m->state_bytes * m->tasks.size();
   m->n_slots = std::min<int32_t>(m->max_groups, static_cast<int32_t>(m->tasks.size()) + 1);
   // slot = qkv [M,3H] bf16 + ctx [M,H] bf16 + u [M,H] fp32 + h1 [M,H] bf16 and fp32 + f [M,F] bf16
-  m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2);
+  //        + fp32 residual rows of the first tokens [B,H]
+  m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2) +
+                  pad256(static_cast<size_t>(m->max_batch) * H * 4);
   m->ws_slot0 = off;
   off += m->slot_bytes * m->n_slots;
   m->n_dump = 0;
@@ -302,34 +320,78 @@ float* f32_of(const mt_model* m, bf16* state) {
   return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(state) + m->act_bytes);
 }
 
-cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int32_t batch,
-                        int32_t seq, Chunk* ck) {
-  const int32_t M = batch * seq, H = m->trunk.hidden, F = m->trunk.ffn;
-  const size_t act = m->act_bytes;
-  const size_t qkv_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * 3 * H * 2);
+// True for the last layer of a task branch when only the first token's state is needed downstream.
+bool is_cls_op(const mt_model* m, const OpDesc& op) {
+  return m->cls_only && op.task >= 0 && op.layer == m->tasks[op.task].cfg.branch_layers;
+}
+
+void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid) {
+  const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
+  const int32_t* rows_valid =
+      all_rows_valid ? nullptr : reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K) {
     memset(g, 0, sizeof(*g));
-    g->n_groups = static_cast<int32_t>(count);
-    g->M = M; g->N = N; g->K = K;
-    g->m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
+    g->M = rows; g->N = N; g->K = K;
+    g->m_valid = rows_valid;
     g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   };
-  init_gemm(&ck->qkv, 3 * H, H);
-  init_gemm(&ck->attn_out, H, H);
-  init_gemm(&ck->ffn_up, F, H);
-  init_gemm(&ck->ffn_down, H, F);
+  init_gemm(&t->attn_out, H, H);
+  init_gemm(&t->ffn_up, F, H);
+  init_gemm(&t->ffn_down, H, F);
+  memset(&t->ln1, 0, sizeof(t->ln1));
+  memset(&t->ln2, 0, sizeof(t->ln2));
+  t->ln1.rows_valid = t->ln2.rows_valid = rows_valid;
+  t->ln1.rows = t->ln2.rows = rows;
+  t->ln1.hidden = t->ln2.hidden = H;
+  t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
+  t->count = 0;
+}
+
+// Steps 3-7 of a layer for one group of a tail: u = ctx Wo^T + bo + residual; h1 = LN(u);
+// f = GELU(h1 W1^T + b1); u = f W2^T + b2 + h1; out = LN(u).
+cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo, const bf16* ctx, const float* residual,
+                        float* u, bf16* h1, bf16* f, bf16* out, float* out32) {
+  const int i = t->count;
+  cudaError_t e;
+  if ((e = set_gemm_group(&t->attn_out, i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) !=
+      cudaSuccess)
+    return e;
+  t->ln1.x[i] = u; t->ln1.gamma[i] = w_ptr(m, lo->ln1_g); t->ln1.beta[i] = w_ptr(m, lo->ln1_b);
+  t->ln1.y[i] = h1; t->ln1.y32[i] = f32_of(m, h1);
+  if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
+      cudaSuccess)
+    return e;
+  if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), f32_of(m, h1), u)) !=
+      cudaSuccess)
+    return e;
+  t->ln2.x[i] = u; t->ln2.gamma[i] = w_ptr(m, lo->ln2_g); t->ln2.beta[i] = w_ptr(m, lo->ln2_b);
+  t->ln2.y[i] = out; t->ln2.y32[i] = out32;
+  t->count = i + 1;
+  t->attn_out.n_groups = t->ffn_up.n_groups = t->ffn_down.n_groups = t->ln1.n_groups = t->ln2.n_groups = t->count;
+  return cudaSuccess;
+}
+
+cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int32_t batch,
+                        int32_t seq, Chunk* ck) {
+  const int32_t M = batch * seq, H = m->trunk.hidden;
+  const size_t act = m->act_bytes;
+  const size_t qkv_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * 3 * H * 2);
+  const size_t f_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * m->trunk.ffn * 2);
+  const int32_t* row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
+  memset(&ck->qkv, 0, sizeof(ck->qkv));
+  ck->qkv.n_groups = static_cast<int32_t>(count);
+  ck->qkv.M = M; ck->qkv.N = 3 * H; ck->qkv.K = H;
+  ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
+  ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
+  init_tail(m, &ck->full, M, false);
+  init_tail(m, &ck->cls, batch, true);
   memset(&ck->attn, 0, sizeof(ck->attn));
-  memset(&ck->ln1, 0, sizeof(ck->ln1));
-  memset(&ck->ln2, 0, sizeof(ck->ln2));
-  ck->attn.n_groups = ck->ln1.n_groups = ck->ln2.n_groups = static_cast<int32_t>(count);
-  ck->attn.batch = batch; ck->attn.seq = seq; ck->attn.heads = m->trunk.heads;
-  ck->attn.lengths = nullptr;  // patched per call
-  ck->attn.row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
+  memset(&ck->attn_cls, 0, sizeof(ck->attn_cls));
+  ck->attn.batch = ck->attn_cls.batch = batch;
+  ck->attn.seq = ck->attn_cls.seq = seq;
+  ck->attn.heads = ck->attn_cls.heads = m->trunk.heads;
+  ck->attn.row_start = ck->attn_cls.row_start = row_start;  // lengths are patched per call
   ck->attn.packed = m->pack_tokens ? 1 : 0;
-  ck->ln1.rows_valid = ck->ln2.rows_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
-  ck->ln1.rows = ck->ln2.rows = M;
-  ck->ln1.hidden = ck->ln2.hidden = H;
-  ck->ln1.eps = ck->ln2.eps = m->trunk.ln_eps;
 
   for (size_t i = 0; i < count; ++i) {
     const OpDesc& op = ops[first + i];
@@ -351,36 +413,42 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     float* u = reinterpret_cast<float*>(slot + qkv_bytes + act);
     bf16* h1 = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes);
     bf16* f = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes + m->state_bytes);
+    float* res_cls = reinterpret_cast<float*>(slot + qkv_bytes + act + m->act32_bytes + m->state_bytes + f_bytes);
 
     cudaError_t e;
-    // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv]   (the three matrices and biases are contiguous in the arena)
-    if ((e = set_gemm_group(&ck->qkv, i, kEpiBias, in, w_ptr(m, lo->wq), w_ptr(m, lo->bq), nullptr, qkv)) != cudaSuccess)
+    // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv] on every token (the three matrices and biases are
+    //    contiguous in the arena); keys and values are needed for all tokens even in a `cls` layer
+    if ((e = set_gemm_group(&ck->qkv, static_cast<int>(i), kEpiBias, in, w_ptr(m, lo->wq), w_ptr(m, lo->bq), nullptr,
+                            qkv)) != cudaSuccess)
       return e;
-    // 2. ctx = attention(qkv)
-    ck->attn.qkv[i] = qkv;
-    ck->attn.ctx[i] = ctx;
-    // 3. u = ctx . Wo^T + bo + in   (fp32 residual, fp32 result)
-    if ((e = set_gemm_group(&ck->attn_out, i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), f32_of(m, in),
-                            u)) != cudaSuccess)
-      return e;
-    // 4. h1 = LN(u)
-    ck->ln1.x[i] = u; ck->ln1.gamma[i] = w_ptr(m, lo->ln1_g); ck->ln1.beta[i] = w_ptr(m, lo->ln1_b);
-    ck->ln1.y[i] = h1; ck->ln1.y32[i] = f32_of(m, h1);
-    // 5. f = GELU(h1 . W1^T + b1)
-    if ((e = set_gemm_group(&ck->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
-        cudaSuccess)
-      return e;
-    // 6. u = f . W2^T + b2 + h1
-    if ((e = set_gemm_group(&ck->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), f32_of(m, h1),
-                            u)) != cudaSuccess)
-      return e;
-    // 7. out = LN(u)
-    ck->ln2.x[i] = u; ck->ln2.gamma[i] = w_ptr(m, lo->ln2_g); ck->ln2.beta[i] = w_ptr(m, lo->ln2_b);
-    ck->ln2.y[i] = out; ck->ln2.y32[i] = f32_of(m, out);
-
-    if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer)});
+    const bool cls = is_cls_op(m, op);
+    if (!cls) {
+      // 2. ctx = attention(qkv) for every token; 3-7 on every token
+      const int a = ck->full.count;
+      ck->attn.qkv[a] = qkv;
+      ck->attn.ctx[a] = ctx;
+      ck->attn.n_groups = a + 1;
+      if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f, out, f32_of(m, out))) != cudaSuccess) return e;
+    } else {
+      // 2'. first-token attention into compact [B, H] buffers (the same scratch, B rows used), which
+      //     also gathers the first tokens' fp32 residual; 3-7 on B rows; the task's state becomes [B, H]
+      const int a = ck->cls.count;
+      ck->attn_cls.qkv[a] = qkv;
+      ck->attn_cls.in32[a] = f32_of(m, in);
+      ck->attn_cls.ctx[a] = ctx;
+      ck->attn_cls.res[a] = res_cls;
+      ck->attn_cls.n_groups = a + 1;
+      if ((e = add_to_tail(m, &ck->cls, lo, ctx, res_cls, u, h1, f, out, nullptr)) != cudaSuccess) return e;
+    }
+    if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer), cls});
   }
   return cudaSuccess;
+}
+
+int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count) {
+  size_t n_cls = 0;
+  for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
+  return 1 + (n_cls < count ? 6 : 0) + (n_cls > 0 ? 6 : 0);
 }
 
 cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
@@ -405,6 +473,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         ht.pool_w = w_ptr(m, te.pool_w); ht.pool_b = w_ptr(m, te.pool_b);
         ht.cls_w = w_ptr(m, te.cls_w); ht.cls_b = w_ptr(m, te.cls_b);
         ht.num_classes = te.cfg.num_classes; ht.col0 = te.col0;
+        ht.compact = (m->cls_only && te.cfg.branch_layers > 0) ? 1 : 0;
       }
       plan->steps.push_back(std::move(st));
       plan->launches += 2;
@@ -420,7 +489,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       cudaError_t e = build_chunk(m, ops, first, count, batch, seq, &st.chunk);
       if (e != cudaSuccess) return e;
       plan->steps.push_back(std::move(st));
-      plan->launches += 7;
+      plan->launches += chunk_launches(m, ops, first, count);
     }
     add_heads(s.heads[w]);
   }
@@ -462,6 +531,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->max_groups = kMaxGroups;
   m->debug_capture = false;
   m->pack_tokens = true;
+  m->cls_only = true;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -525,6 +595,11 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
   if (strcmp(key, "pdl") == 0) {  // process-wide: programmatic dependent launch on or off
     g_use_pdl = value != 0;
+    return MT_OK;
+  }
+  if (strcmp(key, "cls_only_last_layer") == 0) {
+    m->cls_only = value != 0;
+    m->plans.clear();
     return MT_OK;
   }
   if (strcmp(key, "pack_tokens") == 0) {
@@ -648,7 +723,11 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
   if (!build_schedule(m, task_mask, &s)) return fail(m, MT_ERR_INVALID_ARG, "task_mask selects no task");
   int32_t n = 2;  // row starts, embedding
   for (size_t w = 0; w <= s.waves.size(); ++w) {
-    if (w >= 1) n += 7 * static_cast<int32_t>((s.waves[w - 1].size() + m->n_slots - 1) / m->n_slots);
+    if (w >= 1) {
+      const std::vector<OpDesc>& ops = s.waves[w - 1];
+      for (size_t first = 0; first < ops.size(); first += m->n_slots)
+        n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
+    }
     n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
   }
   *n_launches = n;
@@ -732,15 +811,22 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
     if (st.kind == 0) {
       Chunk& ck = st.chunk;
       ck.attn.lengths = d_lengths;
+      ck.attn_cls.lengths = d_lengths;
       MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
-      MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
-      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(ck.attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
-      MT_TIMED(MT_CLASS_LN1, launch_layernorm(ck.ln1, stream), "LayerNorm 1");
-      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(ck.ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
-      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(ck.ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
-      MT_TIMED(MT_CLASS_LN2, launch_layernorm(ck.ln2, stream), "LayerNorm 2");
-      for (const auto& d : ck.dumps)
-        MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.second, d.first, act_used,
+      if (ck.full.count > 0) MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
+      if (ck.cls.count > 0)
+        MT_TIMED(MT_CLASS_ATTENTION, launch_cls_attention(ck.attn_cls, stream), "first-token attention kernel");
+      for (LayerTail* t : {&ck.full, &ck.cls}) {
+        if (t->count == 0) continue;
+        MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
+        MT_TIMED(MT_CLASS_LN1, launch_layernorm(t->ln1, stream), "LayerNorm 1");
+        MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
+        MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
+        MT_TIMED(MT_CLASS_LN2, launch_layernorm(t->ln2, stream), "LayerNorm 2");
+      }
+      for (const DumpCopy& d : ck.dumps)
+        MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.slot, d.src,
+                                  d.compact ? static_cast<size_t>(batch) * m->trunk.hidden * sizeof(bf16) : act_used,
                                   cudaMemcpyDeviceToDevice, stream),
                   "debug capture");
     } else {
@@ -831,7 +917,8 @@ int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out, 
   cudaError_t e = launch_unpack_rows(
       reinterpret_cast<const bf16*>(m->d_workspace + m->ws_dump0 + m->act_bytes * dump_slot(m, task, layer)),
       m->last_lengths, reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start),
-      static_cast<bf16*>(d_out), m->last_batch, m->last_seq, m->trunk.hidden, as_stream(stream_));
+      static_cast<bf16*>(d_out), m->last_batch, m->last_seq, m->trunk.hidden,
+      (m->cls_only && task >= 0 && layer == m->tasks[task].cfg.branch_layers) ? 1 : 0, as_stream(stream_));
   if (e != cudaSuccess) return fail_cuda(m, e, "copying a captured hidden state");
   return MT_OK;
 }

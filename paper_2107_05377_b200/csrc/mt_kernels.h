@@ -90,6 +90,20 @@ struct AttnParams {
 };
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
 
+// Attention of the first token of every sequence only (the last layer of a task branch: its head
+// reads nothing but that row).  Writes the context compactly, ctx[b, :], and gathers the fp32
+// residual of that row from the layer input, res[b, :] = in32[row_start[b], :].
+struct ClsAttnParams {
+  const bf16* qkv[kMaxGroups];   // [rows, 3*H]
+  const float* in32[kMaxGroups]; // [rows, H] fp32 layer input
+  bf16* ctx[kMaxGroups];         // [B, H]
+  float* res[kMaxGroups];        // [B, H]
+  const int32_t* lengths;
+  const int32_t* row_start;      // [B + 1] or null (padded layout)
+  int32_t n_groups, batch, seq, heads;
+};
+cudaError_t launch_cls_attention(const ClsAttnParams& p, cudaStream_t stream);
+
 // y = LN(x): x fp32; y is written as bf16 (the next GEMM's operand) and, if y32 is not null, also
 // as fp32 (the residual of the next sub-layer, so the residual stream is never rounded to bf16).
 struct LayerNormParams {
@@ -123,6 +137,7 @@ struct HeadTask {
   const bf16* hidden;  // final state of the task, [rows, H]; the first row of every sequence is pooled
   const bf16 *pool_w, *pool_b, *cls_w, *cls_b;
   int32_t num_classes, col0;
+  int32_t compact;  // 1: `hidden` is [B, H], one row per sequence (last branch layer computed for that row only)
 };
 struct HeadParams {
   HeadTask task[kMaxGroups];
@@ -137,8 +152,9 @@ struct HeadParams {
 cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,
                               int32_t* rows_valid, cudaStream_t stream);
 // padded[b*seq + pos] = packed[row_start[b] + pos] for pos < length, 0 elsewhere (bf16 rows of `hidden`).
+// With compact != 0 the source is [B, H] (first tokens only) and only position 0 of a sequence is filled.
 cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const int32_t* row_start, bf16* padded,
-                               int32_t batch, int32_t seq, int32_t hidden, cudaStream_t stream);
+                               int32_t batch, int32_t seq, int32_t hidden, int32_t compact, cudaStream_t stream);
 // Two launches: pooler (tanh features into `pooled`), then head (logits).
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream);
 

@@ -161,8 +161,9 @@ __global__ void __launch_bounds__(kHeadThreads) pooler_kernel(const HeadParams p
     const int s = idx / (H / 8), c = idx - s * (H / 8);
     float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (s < nb) {
-      const size_t row = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b0 + s])
-                                                : static_cast<size_t>(b0 + s) * p.seq;
+      const size_t row = tk.compact ? static_cast<size_t>(b0 + s)
+                         : p.row_start != nullptr ? static_cast<size_t>(p.row_start[b0 + s])
+                                                  : static_cast<size_t>(b0 + s) * p.seq;
       unpack8(*reinterpret_cast<const uint4*>(tk.hidden + row * H + c * 8), f);
     }
     *reinterpret_cast<float4*>(cls + s * H + c * 8) = make_float4(f[0], f[1], f[2], f[3]);
@@ -266,16 +267,18 @@ __global__ void row_starts_kernel(const int32_t* lengths, int32_t batch, int32_t
 // One warp per padded row.
 __global__ void __launch_bounds__(kRowThreads) unpack_rows_kernel(const bf16* packed, const int32_t* lengths,
                                                                    const int32_t* row_start, bf16* padded, int32_t batch,
-                                                                   int32_t seq, int32_t hidden) {
+                                                                   int32_t seq, int32_t hidden, int32_t compact) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
   if (row >= batch * seq) return;
   const int b = row / seq, pos = row - b * seq;
   int len = lengths[b];
   len = len < 1 ? 1 : (len > seq ? seq : len);
-  const uint4* src = reinterpret_cast<const uint4*>(packed + static_cast<size_t>(row_start[b] + pos) * hidden);
+  const size_t src_row = compact ? static_cast<size_t>(b) : static_cast<size_t>(row_start[b] + pos);
+  const bool present = compact ? pos == 0 : pos < len;
+  const uint4* src = reinterpret_cast<const uint4*>(packed + src_row * hidden);
   uint4* dst = reinterpret_cast<uint4*>(padded + static_cast<size_t>(row) * hidden);
-  for (int c = lane; c < hidden / 8; c += 32) dst[c] = pos < len ? src[c] : make_uint4(0, 0, 0, 0);
+  for (int c = lane; c < hidden / 8; c += 32) dst[c] = present ? src[c] : make_uint4(0, 0, 0, 0);
 }
 
 }  // namespace
@@ -288,11 +291,11 @@ cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq
 }
 
 cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const int32_t* row_start, bf16* padded,
-                               int32_t batch, int32_t seq, int32_t hidden, cudaStream_t stream) {
+                               int32_t batch, int32_t seq, int32_t hidden, int32_t compact, cudaStream_t stream) {
   const int rows = batch * seq;
   if (rows < 1 || hidden % 8 != 0) return cudaErrorInvalidValue;
   unpack_rows_kernel<<<(rows + kRowThreads / 32 - 1) / (kRowThreads / 32), kRowThreads, 0, stream>>>(
-      packed, lengths, row_start, padded, batch, seq, hidden);
+      packed, lengths, row_start, padded, batch, seq, hidden, compact);
   return cudaGetLastError();
 }
 

@@ -16,11 +16,13 @@ HIDDEN_REL_L2 = 1e-2   # tolerance on hidden states (valid rows)
 LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
-def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None):
+def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
     if pack_tokens is not None:
         model.set_option("pack_tokens", pack_tokens)
+    if cls_only is not None:
+        model.set_option("cls_only_last_layer", cls_only)
     model.load_weights(blob)
     tok, seg, lens = dev_batch(batch)
     logits = torch.full((B, cfg.total_classes), float("nan") if fill is None else fill, dtype=torch.float32,
@@ -31,7 +33,9 @@ def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=No
     return model, logits
 
 
-def check_against_oracle(cfg, wf, batch, model, logits, rows, mask=None, check_hidden=True):
+def check_against_oracle(cfg, wf, batch, model, logits, rows, mask=None, check_hidden=True, cls_only=True):
+    """cls_only: the library evaluated the last layer of every branch for the first token only, so
+    that layer's captured state is compared at position 0 alone."""
     B, S = batch.token_ids.shape
     tasks = task_triples(cfg)
     hid = []
@@ -53,7 +57,11 @@ def check_against_oracle(cfg, wf, batch, model, logits, rows, mask=None, check_h
         for i, b in enumerate(rows):
             n = int(batch.lengths[b])
             for key, ref in hid[i].items():
-                err = rel_l2(states[key][b, :n], ref)
+                n_cmp = n
+                if cls_only and key[0] == "task" and key[2] == cfg.tasks[key[1]].branch_layers:
+                    assert np.all(states[key][b, 1:] == 0)
+                    n_cmp = 1
+                err = rel_l2(states[key][b, :n_cmp], ref[:n_cmp])
                 assert err <= HIDDEN_REL_L2, f"hidden {key} row {b}: rel-L2 {err}"
     return worst
 
@@ -77,6 +85,19 @@ def test_ragged_batch_random_affine_matches_oracle():
                         batch.lengths)
     model, logits = run_model(cfg, blob, batch, debug=True)
     check_against_oracle(cfg, wf, batch, model, logits, rows=range(5))
+
+
+def test_every_token_in_last_branch_layers_matches_oracle_and_first_token_only():
+    """cls_only_last_layer = 0 computes the last layer of every branch on all tokens: parity with the
+    oracle on every row, and logits equal (to rounding) to the default first-token-only evaluation."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
+    model, full = run_model(cfg, blob, batch, debug=True, cls_only=0)
+    check_against_oracle(cfg, wf, batch, model, full, rows=range(6), cls_only=False)
+    _, first = run_model(cfg, blob, batch)
+    assert float((first - full).abs().max()) <= 2e-3
 
 
 def test_padded_layout_matches_oracle_and_packed_layout():

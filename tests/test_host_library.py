@@ -71,9 +71,13 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
         assert m.plan_summary(mask)["layers"] == want
     with pytest.raises(binding.MTError):
         m.plan_summary(0)
+    # waves 7, 8, 9 mix layers on all tokens with last branch layers (first token only): 13 launches
+    assert m.plan_launches(0xFF) == 2 + 7 * 4 + 7 + 7 + 13 + 13 + 13 + 7 + 2
+    m.set_option("cls_only_last_layer", 0)
     assert m.plan_launches(0xFF) == 2 + 7 * 10 + 2   # row starts + embedding, 7 per wave, pooler + head at the end
     m.close()
     m2 = binding.MTModel(cfg, 32, 128, max_groups=2, bind=False)
+    m2.set_option("cls_only_last_layer", 0)
     assert m2.plan_summary(0xFF)["layers"] == 24
     assert m2.plan_launches(0xFF) == 2 + 7 * (1 + 1 + 1 + 1 + 1 + 2 + 3 + 3 + 2 + 1) + 2
     m2.close()
