@@ -84,19 +84,24 @@ struct DumpCopy {
   bool compact;  // [B, H]: first tokens only
 };
 // One chunk of a wave: the QKV projection of all its layers in one launch, then the rest of the
-// layer for the layers computed on every token (`full`) and for the last layers of task branches,
-// which are computed for the first token of every sequence only (`cls`).
+// layer for the layers computed on every token (`full`).  The last layers of task branches are
+// needed for the first token of every sequence only: in their wave they get the QKV projection (keys
+// and values of all tokens) and the first-token attention (`attn_cls`, `n_cls` groups); the rest of
+// those layers, a few rows each, is run for all tasks together after the last wave (a `cls tail` step).
 struct Chunk {
   GemmParams qkv;
   AttnParams attn;
   ClsAttnParams attn_cls;
-  LayerTail full, cls;
+  LayerTail full;
+  int32_t n_cls = 0;
   std::vector<DumpCopy> dumps;
 };
 struct PlanStep {
-  int kind;  // 0 = chunk, 1 = heads
+  int kind;  // 0 = chunk, 1 = heads, 2 = cls tail
   Chunk chunk;
   HeadParams heads;
+  LayerTail tail;
+  std::vector<DumpCopy> dumps;
 };
 struct Plan {
   std::vector<PlanStep> steps;
@@ -185,7 +190,8 @@ struct mt_model {
 
   // workspace layout (byte offsets)
   size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
-      ws_slot0, ws_dump0;
+      ws_slot0, ws_cls0, ws_dump0;
+  size_t cls_bytes, cls_h_bytes, cls_h32_bytes;  // per-task first-token scratch and its [B,H] bf16 / fp32 pieces
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
   size_t state_bytes;  // one hidden state = its bf16 copy (GEMM operand) followed by its fp32 copy (residual)
@@ -251,11 +257,16 @@ void layout_workspace(mt_model* m) {
   off += m->state_bytes * m->tasks.size();
   m->n_slots = std::min<int32_t>(m->max_groups, static_cast<int32_t>(m->tasks.size()) + 1);
   // slot = qkv [M,3H] bf16 + ctx [M,H] bf16 + u [M,H] fp32 + h1 [M,H] bf16 and fp32 + f [M,F] bf16
-  //        + fp32 residual rows of the first tokens [B,H]
-  m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2) +
-                  pad256(static_cast<size_t>(m->max_batch) * H * 4);
+  m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2);
   m->ws_slot0 = off;
   off += m->slot_bytes * m->n_slots;
+  // per task, for its last branch layer on first tokens: ctx bf16, residual fp32, u fp32, h1 bf16 + fp32 (all
+  // [B,H]) and f bf16 [B,F]
+  m->cls_h_bytes = pad256(static_cast<size_t>(m->max_batch) * H * 2);
+  m->cls_h32_bytes = pad256(static_cast<size_t>(m->max_batch) * H * 4);
+  m->cls_bytes = 2 * m->cls_h_bytes + 3 * m->cls_h32_bytes + pad256(static_cast<size_t>(m->max_batch) * F * 2);
+  m->ws_cls0 = off;
+  off += m->cls_bytes * m->tasks.size();
   m->n_dump = 0;
   m->ws_dump0 = off;
   if (m->debug_capture) {
@@ -350,18 +361,18 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
 // Steps 3-7 of a layer for one group of a tail: u = ctx Wo^T + bo + residual; h1 = LN(u);
 // f = GELU(h1 W1^T + b1); u = f W2^T + b2 + h1; out = LN(u).
 cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo, const bf16* ctx, const float* residual,
-                        float* u, bf16* h1, bf16* f, bf16* out, float* out32) {
+                        float* u, bf16* h1, float* h1_32, bf16* f, bf16* out, float* out32) {
   const int i = t->count;
   cudaError_t e;
   if ((e = set_gemm_group(&t->attn_out, i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) !=
       cudaSuccess)
     return e;
   t->ln1.x[i] = u; t->ln1.gamma[i] = w_ptr(m, lo->ln1_g); t->ln1.beta[i] = w_ptr(m, lo->ln1_b);
-  t->ln1.y[i] = h1; t->ln1.y32[i] = f32_of(m, h1);
+  t->ln1.y[i] = h1; t->ln1.y32[i] = h1_32;
   if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
       cudaSuccess)
     return e;
-  if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), f32_of(m, h1), u)) !=
+  if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) !=
       cudaSuccess)
     return e;
   t->ln2.x[i] = u; t->ln2.gamma[i] = w_ptr(m, lo->ln2_g); t->ln2.beta[i] = w_ptr(m, lo->ln2_b);
@@ -376,7 +387,6 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   const int32_t M = batch * seq, H = m->trunk.hidden;
   const size_t act = m->act_bytes;
   const size_t qkv_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * 3 * H * 2);
-  const size_t f_bytes = pad256(static_cast<size_t>(m->max_batch) * m->max_seq * m->trunk.ffn * 2);
   const int32_t* row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
   memset(&ck->qkv, 0, sizeof(ck->qkv));
   ck->qkv.n_groups = static_cast<int32_t>(count);
@@ -384,7 +394,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   init_tail(m, &ck->full, M, false);
-  init_tail(m, &ck->cls, batch, true);
+  ck->n_cls = 0;
   memset(&ck->attn, 0, sizeof(ck->attn));
   memset(&ck->attn_cls, 0, sizeof(ck->attn_cls));
   ck->attn.batch = ck->attn_cls.batch = batch;
@@ -413,7 +423,6 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     float* u = reinterpret_cast<float*>(slot + qkv_bytes + act);
     bf16* h1 = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes);
     bf16* f = reinterpret_cast<bf16*>(slot + qkv_bytes + act + m->act32_bytes + m->state_bytes);
-    float* res_cls = reinterpret_cast<float*>(slot + qkv_bytes + act + m->act32_bytes + m->state_bytes + f_bytes);
 
     cudaError_t e;
     // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv] on every token (the three matrices and biases are
@@ -428,19 +437,44 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
       ck->attn.qkv[a] = qkv;
       ck->attn.ctx[a] = ctx;
       ck->attn.n_groups = a + 1;
-      if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f, out, f32_of(m, out))) != cudaSuccess) return e;
+      if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f32_of(m, h1), f, out, f32_of(m, out))) !=
+          cudaSuccess)
+        return e;
+      if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer), false});
     } else {
-      // 2'. first-token attention into compact [B, H] buffers (the same scratch, B rows used), which
-      //     also gathers the first tokens' fp32 residual; 3-7 on B rows; the task's state becomes [B, H]
-      const int a = ck->cls.count;
+      // 2'. first-token attention into the task's compact [B, H] scratch, which also gathers the first
+      //     tokens' fp32 residual; steps 3-7 of these layers follow after the last wave
+      const int a = ck->n_cls;
+      uint8_t* cs = m->d_workspace + m->ws_cls0 + m->cls_bytes * op.task;
       ck->attn_cls.qkv[a] = qkv;
       ck->attn_cls.in32[a] = f32_of(m, in);
-      ck->attn_cls.ctx[a] = ctx;
-      ck->attn_cls.res[a] = res_cls;
-      ck->attn_cls.n_groups = a + 1;
-      if ((e = add_to_tail(m, &ck->cls, lo, ctx, res_cls, u, h1, f, out, nullptr)) != cudaSuccess) return e;
+      ck->attn_cls.ctx[a] = reinterpret_cast<bf16*>(cs);
+      ck->attn_cls.res[a] = reinterpret_cast<float*>(cs + m->cls_h_bytes);
+      ck->attn_cls.n_groups = ck->n_cls = a + 1;
     }
-    if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer), cls});
+  }
+  return cudaSuccess;
+}
+
+// Steps 3-7 of the last branch layers of `tasks` on their first tokens ([B, H] rows), one group per task.
+cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks, size_t first, size_t count,
+                           int32_t batch, PlanStep* st) {
+  init_tail(m, &st->tail, batch, true);
+  for (size_t i = 0; i < count; ++i) {
+    const int32_t t = tasks[first + i];
+    const TaskEntry& te = m->tasks[t];
+    const LayerOffsets* lo = &te.layers[te.cfg.branch_layers - 1];
+    uint8_t* cs = m->d_workspace + m->ws_cls0 + m->cls_bytes * t;
+    bf16* ctx = reinterpret_cast<bf16*>(cs);
+    float* res = reinterpret_cast<float*>(cs + m->cls_h_bytes);
+    float* u = reinterpret_cast<float*>(cs + m->cls_h_bytes + m->cls_h32_bytes);
+    bf16* h1 = reinterpret_cast<bf16*>(cs + m->cls_h_bytes + 2 * m->cls_h32_bytes);
+    float* h1_32 = reinterpret_cast<float*>(cs + 2 * m->cls_h_bytes + 2 * m->cls_h32_bytes);
+    bf16* f = reinterpret_cast<bf16*>(cs + 2 * m->cls_h_bytes + 3 * m->cls_h32_bytes);
+    bf16* out = task_buf(m, t);  // the task's state becomes [B, H]
+    cudaError_t e = add_to_tail(m, &st->tail, lo, ctx, res, u, h1, h1_32, f, out, nullptr);
+    if (e != cudaSuccess) return e;
+    if (m->debug_capture) st->dumps.push_back({out, dump_slot(m, t, te.cfg.branch_layers), true});
   }
   return cudaSuccess;
 }
@@ -448,7 +482,16 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
 int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count) {
   size_t n_cls = 0;
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
-  return 1 + (n_cls < count ? 6 : 0) + (n_cls > 0 ? 6 : 0);
+  return 1 + (n_cls < count ? 6 : 0) + (n_cls > 0 ? 1 : 0);
+}
+// Active tasks whose last branch layer is finished on first tokens after the last wave.
+std::vector<int32_t> cls_tasks(const mt_model* m, const Schedule& s) {
+  std::vector<int32_t> out;
+  for (const auto& wave : s.waves)
+    for (const OpDesc& op : wave)
+      if (is_cls_op(m, op)) out.push_back(op.task);
+  std::sort(out.begin(), out.end());
+  return out;
 }
 
 cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
@@ -490,6 +533,17 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       if (e != cudaSuccess) return e;
       plan->steps.push_back(std::move(st));
       plan->launches += chunk_launches(m, ops, first, count);
+    }
+    if (w == s.waves.size()) {
+      const std::vector<int32_t> tasks = cls_tasks(m, s);
+      for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
+        PlanStep st;
+        st.kind = 2;
+        cudaError_t e = build_cls_tail(m, tasks, first, std::min<size_t>(kMaxGroups, tasks.size() - first), batch, &st);
+        if (e != cudaSuccess) return e;
+        plan->steps.push_back(std::move(st));
+        plan->launches += 5;
+      }
     }
     add_heads(s.heads[w]);
   }
@@ -727,6 +781,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
       const std::vector<OpDesc>& ops = s.waves[w - 1];
       for (size_t first = 0; first < ops.size(); first += m->n_slots)
         n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
+      if (w == s.waves.size()) n += 5 * static_cast<int32_t>((cls_tasks(m, s).size() + kMaxGroups - 1) / kMaxGroups);
     }
     n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
   }
@@ -814,10 +869,10 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
       ck.attn_cls.lengths = d_lengths;
       MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
       if (ck.full.count > 0) MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
-      if (ck.cls.count > 0)
+      if (ck.n_cls > 0)
         MT_TIMED(MT_CLASS_ATTENTION, launch_cls_attention(ck.attn_cls, stream), "first-token attention kernel");
-      for (LayerTail* t : {&ck.full, &ck.cls}) {
-        if (t->count == 0) continue;
+      if (ck.full.count > 0) {
+        LayerTail* t = &ck.full;
         MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
         MT_TIMED(MT_CLASS_LN1, launch_layernorm(t->ln1, stream), "LayerNorm 1");
         MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
@@ -828,6 +883,18 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
         MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.slot, d.src,
                                   d.compact ? static_cast<size_t>(batch) * m->trunk.hidden * sizeof(bf16) : act_used,
                                   cudaMemcpyDeviceToDevice, stream),
+                  "debug capture");
+    } else if (st.kind == 2) {
+      LayerTail* t = &st.tail;
+      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
+      MT_TIMED(MT_CLASS_LN1, launch_layernorm(t->ln1, stream), "LayerNorm 1");
+      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
+      MT_TIMED(MT_CLASS_LN2, launch_layernorm(t->ln2, stream), "LayerNorm 2");
+      for (const DumpCopy& d : st.dumps)
+        MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.slot, d.src,
+                                  static_cast<size_t>(batch) * m->trunk.hidden * sizeof(bf16), cudaMemcpyDeviceToDevice,
+                                  stream),
                   "debug capture");
     } else {
       st.heads.logits = d_logits;

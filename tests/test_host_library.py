@@ -71,8 +71,10 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
         assert m.plan_summary(mask)["layers"] == want
     with pytest.raises(binding.MTError):
         m.plan_summary(0)
-    # waves 7, 8, 9 mix layers on all tokens with last branch layers (first token only): 13 launches
-    assert m.plan_launches(0xFF) == 2 + 7 * 4 + 7 + 7 + 13 + 13 + 13 + 7 + 2
+    # waves 7, 8, 9 mix layers on all tokens (7 launches) with last branch layers, which only add the
+    # first-token attention there; wave 10 holds a last layer alone (projection + first-token attention);
+    # the rest of the eight last layers is one grouped pass of 5 launches before the pooler/head pair
+    assert m.plan_launches(0xFF) == 2 + 7 * 4 + 7 + 7 + 8 + 8 + 8 + 2 + 5 + 2
     m.set_option("cls_only_last_layer", 0)
     assert m.plan_launches(0xFF) == 2 + 7 * 10 + 2   # row starts + embedding, 7 per wave, pooler + head at the end
     m.close()
