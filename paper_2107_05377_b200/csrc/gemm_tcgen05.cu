@@ -57,6 +57,13 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// Adds to the transaction count of the current phase without arriving.
+__device__ __forceinline__ void mbar_add_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -255,15 +262,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // everything above touched no global data; from here on the previous kernel must have completed
+  // Tiles are numbered m-tile outermost: tile = (m_tile * n_groups + g) * n_tiles_n + n_tile, so the
+  // group and the column block of a tile do not depend on the (device-side) number of rows.
+  const int tiles_per_m = p.n_groups * n_tiles_n;
+  // Everything above touched no global data.  The weights do not depend on the previous kernel
+  // either: the producer thread starts the W tiles of this CTA's first tile before it waits for
+  // that kernel, so their trip from HBM overlaps its tail.  From the wait on, the previous kernel
+  // has completed and its writes are visible.
+  int prefetched = 0;   // stages whose W tile is already on its way (producer thread only)
+  if (warp == 0 && lane == 0) {
+    const int rem = static_cast<int>(blockIdx.x) % tiles_per_m;
+    const int g = rem / n_tiles_n;
+    const int n0 = (rem - g * n_tiles_n) * BN;
+    prefetch_tensormap(&p.tmap_x[g]);
+    prefetch_tensormap(&p.tmap_w[g]);
+    prefetched = k_blocks < STAGES ? k_blocks : STAGES;
+    for (int s = 0; s < prefetched; ++s) {
+      mbar_add_tx(bar_full + 8 * s, B_BYTES);
+      tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full + 8 * s);
+    }
+  }
   grid_dependency_wait();
   grid_launch_dependents();
   // rows in use: all M, or fewer when the token layout is packed (a device-side count)
   int m_rows = p.M;
   if (p.m_valid != nullptr) m_rows = min(m_rows, *p.m_valid);
   const int n_tiles_m = (m_rows + kGemmBlockM - 1) / kGemmBlockM;
-  const int tiles_per_group = n_tiles_m * n_tiles_n;
-  const int total_tiles = tiles_per_group * p.n_groups;
+  const int total_tiles = n_tiles_m * tiles_per_m;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -272,16 +297,34 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
+      if (static_cast<int>(blockIdx.x) >= total_tiles) {
+        // no tile for this CTA after all (fewer rows in use than the grid was sized for): let the
+        // early W tiles land before the CTA retires
+        for (int s = 0; s < prefetched; ++s) {
+          mbar_arrive(bar_full + 8 * s);
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(bar_full + 8 * s, 0)) {
+            if (global_timer_ns() - t0 > kWaitLimitNs) break;
+          }
+        }
+      }
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int g = tile / tiles_per_group;
-        const int local = tile - g * tiles_per_group;
-        const int m0 = (local / n_tiles_n) * kGemmBlockM;
-        const int n0 = (local % n_tiles_n) * BN;
+        const int m0 = (tile / tiles_per_m) * kGemmBlockM;
+        const int rem = tile % tiles_per_m;
+        const int g = rem / n_tiles_n;
+        const int n0 = (rem - g * n_tiles_n) * BN;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(bar_full + 8 * stage, A_BYTES + B_BYTES);
-          tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
-          tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+          if (prefetched > 0) {
+            // the W tile of this stage was started before the dependency wait
+            --prefetched;
+            mbar_expect_tx(bar_full + 8 * stage, A_BYTES);
+            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+          } else {
+            mbar_expect_tx(bar_full + 8 * stage, A_BYTES + B_BYTES);
+            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+            tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+          }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -355,10 +398,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
     // (residual epilogue) asks for the residual chunk `chunk` of tile `tile` into staging buffer b
     auto prefetch_residual = [&](int tile, int chunk, int b) {
-      const int g = tile / tiles_per_group;
-      const int local = tile - g * tiles_per_group;
-      const int row0 = (local / n_tiles_n) * kGemmBlockM + quarter * 32;
-      const int col0 = (local % n_tiles_n) * BN + chunk * CHUNK_COLS;
+      const int rem = tile % tiles_per_m;
+      const int g = rem / n_tiles_n;
+      const int row0 = (tile / tiles_per_m) * kGemmBlockM + quarter * 32;
+      const int col0 = (rem - g * n_tiles_n) * BN + chunk * CHUNK_COLS;
       // the store issued last read this very buffer: it must be done with it before TMA refills it
       tma_store_wait_read<0>();
       mbar_expect_tx(my_res_bar + 8 * b, kStagingBytes);
@@ -369,10 +412,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       prefetch_residual(blockIdx.x, col_group, 0);
 
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int g = tile / tiles_per_group;
-      const int local = tile - g * tiles_per_group;
-      const int m0 = (local / n_tiles_n) * kGemmBlockM;
-      const int n0 = (local % n_tiles_n) * BN;
+      const int m0 = (tile / tiles_per_m) * kGemmBlockM;
+      const int rem = tile % tiles_per_m;
+      const int g = rem / n_tiles_n;
+      const int n0 = (rem - g * n_tiles_n) * BN;
       // warp-uniform decisions: the TMEM loads below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag))) break;
       tc_fence_after();
