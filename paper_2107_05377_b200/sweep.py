@@ -97,7 +97,7 @@ def main():
 
     # eight independent full-depth single-task models: one blob, eight arenas
     st_cfg = synth.config_full_depth_single(cfg, 2)
-    st_w = {"emb": weights["emb"], "trunk": weights["trunk"], "tasks": [synth.make_task_weights(st_cfg, 0, seed=0)]}
+    st_w = {"emb": weights["emb"], "trunk": [], "tasks": [synth.make_task_weights(st_cfg, 0, seed=0)]}
     st_blob = synth.pack_weights(st_cfg, st_w)
 
     for B in batches:
@@ -115,7 +115,7 @@ def main():
                 m.forward(tok, seg, lens, lg)
 
         eager, graph = _time_ms(eight, iters, False), _time_ms(eight, iters, True)
-        out({"case": "8 independent 12-layer single-task models", "batch": B, "seq": 128, "layers": 96,
+        out({"case": "8 independent 12-layer single-task models (0,12)", "batch": B, "seq": 128, "layers": 96,
              "launches": 8 * models[0].plan_launches(1), "ms_eager": eager, "ms_graph": graph,
              "seq_per_s_graph": 1e3 * B / graph, "tflops_padded_graph": flops_padded(cfg, 96, B, 128) / graph / 1e9})
         for m in models:

@@ -99,11 +99,12 @@ def config_single_task(base: TreeConfig, task: int) -> TreeConfig:
 
 
 def config_full_depth_single(base: TreeConfig, num_classes: int) -> TreeConfig:
-    """A conventional fully fine-tuned single-task model: the whole trunk depth
-    and a head, nothing shared (Table 2's "12 x 8" baseline is eight of these)."""
-    return TreeConfig(hidden=base.hidden, heads=base.heads, ffn=base.ffn, trunk_layers=base.trunk_layers,
+    """A conventional fully fine-tuned single-task model: every layer is the task's own, nothing
+    is shared - (x, y) = (0, 12) in Table 2's notation; its "12 x 8" baseline is eight of these.
+    No frozen trunk layer is loaded."""
+    return TreeConfig(hidden=base.hidden, heads=base.heads, ffn=base.ffn, trunk_layers=0,
                       vocab_size=base.vocab_size, max_position=base.max_position, type_vocab=base.type_vocab,
-                      ln_eps=base.ln_eps, tasks=(TaskSpec(base.trunk_layers, 0, num_classes),))
+                      ln_eps=base.ln_eps, tasks=(TaskSpec(0, base.trunk_layers, num_classes),))
 
 
 # --------------------------------------------------------------------------
