@@ -1,7 +1,7 @@
 """fp64 CPU oracle of the merged multi-task BERT forward pass.
 
 TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
-CUDA library is judged against.  It shares no code with the CUDA path, imports
+CUDA library is checked against.  It shares no code with the CUDA path, imports
 nothing from it, and must never be called from the product path: only tests,
 the smoke check and the benchmark's CPU-baseline leg use it.
 

@@ -229,6 +229,31 @@ def test_host_entry_point_and_error_paths():
     assert e.value.code == -4
 
 
+def test_production_shaped_tree_with_21_tasks():
+    """App. E serves 21 tasks from one model (8 shared layers, ~1.5 task layers per task).  More tasks
+    than one grouped launch holds: waves, first-token tails and heads are split into chunks."""
+    rng = np.random.default_rng(21)
+    specs = tuple(synth.TaskSpec(int(rng.integers(0, 4)), int(rng.integers(0, 3)), int(rng.integers(1, 5)))
+                  for _ in range(21))
+    cfg = synth.TreeConfig(trunk_layers=3, vocab_size=2000, max_position=64, tasks=specs)
+    w, blob, wf = cached_weights(cfg, 3, random_affine=True)
+    batch = synth.make_batch(cfg, 5, 48, 1, 48, seed=6)
+    model, logits = run_model(cfg, blob, batch, debug=True)
+    assert max(model.plan_summary(model.full_mask())["groups_per_wave"]) > 8
+    check_against_oracle(cfg, wf, batch, model, logits, rows=range(5))
+    # every task alone gives the same bits as inside the merged model
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    for t in (0, 7, 20):
+        _, one = run_model(cfg, blob, batch, mask=1 << t, fill=0.0)
+        assert torch.equal(one[:, offs[t]:offs[t + 1]], logits[:, offs[t]:offs[t + 1]])
+    # a 21-bit mask with the high tasks only
+    mask = sum(1 << t for t in range(12, 21))
+    _, part = run_model(cfg, blob, batch, mask=mask, fill=0.0)
+    for t in range(21):
+        cols = slice(offs[t], offs[t + 1])
+        assert torch.equal(part[:, cols], logits[:, cols]) if (mask >> t) & 1 else torch.all(part[:, cols] == 0)
+
+
 def test_glue8_tree_batch32_seq128_sampled_rows():
     """The 8-task BERT-base tree at 32 x 128 with lengths in [16, 128], in the launch
     configuration the benchmark times; the oracle is evaluated on sampled sequences
