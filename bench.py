@@ -206,14 +206,15 @@ def main():
     from paper_2107_05377_b200 import build as builder
 
     args.warmup = max(args.warmup, 3)
-    if rank == 0 or world == 1:
-        builder.build()
     distributed = world > 1
     if distributed:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        dist.barrier()
+    if rank == 0:
+        builder.build()   # a no-op when the library is up to date
+    if distributed:
+        dist.barrier()    # the other ranks load the library only after rank 0 has (re)built it
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
 

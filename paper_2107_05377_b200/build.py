@@ -31,15 +31,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    tmp = f"{LIB}.{os.getpid()}.tmp"   # built aside and renamed, so a concurrent loader never sees a partial file
     cmd = [nvcc, "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "--threads", "4", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", LIB] + sources()
+           "--threads", "4", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", tmp] + sources()
     if verbose:
         cmd += ["-Xptxas", "-v"]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
     if res.returncode != 0:
+        if os.path.exists(tmp):
+            os.remove(tmp)
         raise RuntimeError("nvcc failed building libmt_bert.so")
+    os.replace(tmp, LIB)
     return LIB
 
 
