@@ -134,6 +134,19 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
                const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
                float* d_logits, void* stream);
 
+/* mt_forward that also tells the caller when each task is done.  task_events: NULL, or an array of
+ * n_tasks entries, each NULL or a cudaEvent_t (passed as void*) owned by the caller; the event of
+ * task t is recorded on `stream` right after the launch that writes that task's logits, so a second
+ * stream (cudaStreamWaitEvent) or the host (cudaEventSynchronize) can pick up task t's columns of
+ * d_logits before the other tasks have finished.  The paper notes that in the merged model no task's
+ * output is available before all are computed (Section 5.2); with option "early_heads" = 1 every task's
+ * head is scheduled right after the wave that completes its branch, so tasks that fork low and have
+ * short branches finish first.  Without that option all heads of tasks with branch layers share one
+ * launch at the end (higher throughput) and their events are recorded together. */
+int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
+                      const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
+                      float* d_logits, void* const* task_events, void* stream);
+
 /* Same computation from HOST buffers: copies the three inputs to the workspace, runs mt_forward,
  * copies the logits back to h_logits ([batch, C_total] fp32) and synchronises the stream.
  * Pinned host buffers make the copies asynchronous with respect to the host. */
@@ -163,7 +176,8 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * mt_profile_read.  key "cls_only_last_layer" (0/1, default 1, any time): the last
  * layer of every task branch is evaluated for the first token of each sequence only (keys and values
  * still for all tokens) because the pooler reads nothing else; mt_debug_copy_hidden then returns that
- * layer's state at position 0 and zeros elsewhere.  key "pack_tokens" (0/1, default 1, any time): store
+ * layer's state at position 0 and zeros elsewhere.  key "early_heads" (0/1, default 0, any time): see mt_forward_events.
+ * key "pack_tokens" (0/1, default 1, any time): store
  * and compute only the valid tokens of every sequence (rows of sequence b follow those of b-1) instead
  * of batch*seq padded rows; logits agree to rounding either way.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's

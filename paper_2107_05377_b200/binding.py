@@ -44,6 +44,7 @@ SIGNATURES = {
     "mt_load_weights": (C.c_int, [_P, _P, _SZ, _P]),
     "mt_load_task_weights": (C.c_int, [_P, _I32, _P, _SZ, _P]),
     "mt_forward": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
+    "mt_forward_events": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, C.POINTER(_P), _P]),
     "mt_forward_host": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
     "mt_poll_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "mt_plan_summary": (C.c_int, [_P, _U64, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32)]),
@@ -93,6 +94,11 @@ def _check(code: int, where: str, model=None) -> None:
 
 def _ptr(t) -> int:
     return 0 if t is None else t.data_ptr()
+
+
+def torch_stream_for_init():
+    import torch
+    return torch.cuda.current_stream()
 
 
 def _stream(stream=None) -> int:
@@ -242,6 +248,21 @@ class MTModel:
         mask = self.full_mask() if task_mask is None else task_mask
         _check(lib().mt_forward(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
                                 _ptr(logits), _stream(stream)), "mt_forward", self.handle)
+
+    def forward_events(self, token_ids, segment_ids, lengths, logits, task_events, task_mask: Optional[int] = None,
+                       stream=None) -> None:
+        """forward() that records ``task_events[t]`` (torch.cuda.Event or None per task) as soon as the
+        launch writing task t's logits has been enqueued."""
+        batch, seq = token_ids.shape
+        mask = self.full_mask() if task_mask is None else task_mask
+        handles = (_P * self.cfg.n_tasks)()
+        for t, ev in enumerate(task_events):
+            if ev is not None:
+                if not ev.cuda_event:       # torch creates the event lazily
+                    ev.record(torch_stream_for_init())
+                handles[t] = ev.cuda_event
+        _check(lib().mt_forward_events(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch,
+                                       seq, _ptr(logits), handles, _stream(stream)), "mt_forward_events", self.handle)
 
     def forward_host(self, token_ids, segment_ids, lengths, logits, task_mask: Optional[int] = None,
                      stream=None) -> None:

@@ -100,6 +100,7 @@ struct PlanStep {
   int kind;  // 0 = chunk, 1 = heads, 2 = cls tail
   Chunk chunk;
   HeadParams heads;
+  std::vector<int32_t> head_tasks;  // tasks of a heads step, in group order
   LayerTail tail;
   std::vector<DumpCopy> dumps;
 };
@@ -181,6 +182,7 @@ struct mt_model {
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
   bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
+  bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
 
   // device memory (caller-owned)
   uint8_t* d_weights;
@@ -311,11 +313,14 @@ bool build_schedule(const mt_model* m, uint64_t mask, Schedule* s) {
   }
   // Heads: a task without branch layers pools the trunk state, which lives in a ping-pong buffer, so
   // its head runs right after the wave that produced that state; every other task keeps its final
-  // state in its own buffer and all of those heads share one launch after the last wave.
+  // state in its own buffer and, for throughput, all of those heads share one launch after the last
+  // wave.  With option early_heads every head runs right after the wave that finishes its task, so
+  // that shallow tasks deliver before the deep ones are done (the latency limitation of Section 5.2).
   for (int32_t t = 0; t < T; ++t) {
     if (!((mask >> t) & 1)) continue;
     const mt_task_config& c = m->tasks[t].cfg;
-    s->heads[c.branch_layers == 0 ? c.fork_depth : last_wave].push_back(t);
+    const bool now = c.branch_layers == 0 || m->early_heads;
+    s->heads[now ? c.fork_depth + c.branch_layers : last_wave].push_back(t);
   }
   return true;
 }
@@ -484,12 +489,15 @@ int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
   return 1 + (n_cls < count ? 6 : 0) + (n_cls > 0 ? 1 : 0);
 }
-// Active tasks whose last branch layer is finished on first tokens after the last wave.
-std::vector<int32_t> cls_tasks(const mt_model* m, const Schedule& s) {
+// Active tasks whose last branch layer is finished on first tokens right after wave w (1-based):
+// those whose last layer is in wave w with option early_heads, otherwise all of them after the last wave.
+std::vector<int32_t> cls_tasks_after_wave(const mt_model* m, const Schedule& s, size_t w) {
   std::vector<int32_t> out;
-  for (const auto& wave : s.waves)
-    for (const OpDesc& op : wave)
+  for (size_t v = 1; v <= s.waves.size(); ++v) {
+    if (m->early_heads ? v != w : w != s.waves.size()) continue;
+    for (const OpDesc& op : s.waves[v - 1])
       if (is_cls_op(m, op)) out.push_back(op.task);
+  }
   std::sort(out.begin(), out.end());
   return out;
 }
@@ -517,6 +525,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         ht.cls_w = w_ptr(m, te.cls_w); ht.cls_b = w_ptr(m, te.cls_b);
         ht.num_classes = te.cfg.num_classes; ht.col0 = te.col0;
         ht.compact = (m->cls_only && te.cfg.branch_layers > 0) ? 1 : 0;
+        st.head_tasks.push_back(t);
       }
       plan->steps.push_back(std::move(st));
       plan->launches += 2;
@@ -534,8 +543,9 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       plan->steps.push_back(std::move(st));
       plan->launches += chunk_launches(m, ops, first, count);
     }
-    if (w == s.waves.size()) {
-      const std::vector<int32_t> tasks = cls_tasks(m, s);
+    {
+      // first-token tails: of the tasks finishing in this wave (early_heads), or of all tasks after the last wave
+      const std::vector<int32_t> tasks = cls_tasks_after_wave(m, s, w);
       for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
         PlanStep st;
         st.kind = 2;
@@ -586,6 +596,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->debug_capture = false;
   m->pack_tokens = true;
   m->cls_only = true;
+  m->early_heads = false;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -649,6 +660,11 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
   if (strcmp(key, "pdl") == 0) {  // process-wide: programmatic dependent launch on or off
     g_use_pdl = value != 0;
+    return MT_OK;
+  }
+  if (strcmp(key, "early_heads") == 0) {
+    m->early_heads = value != 0;
+    m->plans.clear();
     return MT_OK;
   }
   if (strcmp(key, "cls_only_last_layer") == 0) {
@@ -781,7 +797,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
       const std::vector<OpDesc>& ops = s.waves[w - 1];
       for (size_t first = 0; first < ops.size(); first += m->n_slots)
         n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
-      if (w == s.waves.size()) n += 5 * static_cast<int32_t>((cls_tasks(m, s).size() + kMaxGroups - 1) / kMaxGroups);
+      n += 5 * static_cast<int32_t>((cls_tasks_after_wave(m, s, w).size() + kMaxGroups - 1) / kMaxGroups);
     }
     n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
   }
@@ -791,6 +807,12 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
 
 int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
                uint64_t task_mask, int32_t batch, int32_t seq, float* d_logits, void* stream_) {
+  return mt_forward_events(m, d_token_ids, d_segment_ids, d_lengths, task_mask, batch, seq, d_logits, nullptr, stream_);
+}
+
+int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
+                      uint64_t task_mask, int32_t batch, int32_t seq, float* d_logits, void* const* task_events,
+                      void* stream_) {
   if (m == nullptr) return MT_ERR_INVALID_ARG;
   if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr || d_logits == nullptr)
     return fail(m, MT_ERR_INVALID_ARG, "null input or output pointer");
@@ -899,6 +921,10 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
     } else {
       st.heads.logits = d_logits;
       MT_TIMED(MT_CLASS_HEAD, launch_pooler_head(st.heads, stream), "pooler/head kernel");
+      if (task_events != nullptr)
+        for (int32_t t : st.head_tasks)
+          if (task_events[t] != nullptr)
+            MT_LAUNCH(cudaEventRecord(reinterpret_cast<cudaEvent_t>(task_events[t]), stream), "recording a task event");
     }
   }
 #undef MT_TIMED

@@ -125,6 +125,32 @@ def main():
     run_tree("glue8 tree, long sequences", cfg, blob, synth.make_batch(cfg, 16, 512, 128, 512, seed=1),
              [("all 8", 0xFF)], 20, out)
     run_tree("glue8 tree, headline shape", cfg, blob, synth.batch_glue8(cfg), [("all 8", 0xFF)], 50, out)
+    # time to each task's logits with heads scheduled as early as possible (the latency limitation of Section 5.2)
+    hb = synth.batch_glue8(cfg)
+    for early in (0, 1):
+        model = binding.MTModel(cfg, 32, 128)
+        model.set_option("early_heads", early)
+        model.load_weights(blob)
+        tok, seg, lens = _dev(hb)
+        logits = torch.zeros(32, cfg.total_classes, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            model.forward(tok, seg, lens, logits)
+        torch.cuda.synchronize()
+        acc, total, reps = [0.0] * 8, 0.0, 20
+        for _ in range(reps):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record()
+            model.forward_events(tok, seg, lens, logits, ev)
+            s1.record()
+            torch.cuda.synchronize()
+            acc = [x + s0.elapsed_time(e) for x, e in zip(acc, ev)]
+            total += s0.elapsed_time(s1)
+        out({"case": "glue8 tree, headline shape, per-task completion", "batch": 32, "seq": 128, "early_heads": early,
+             "launches": model.plan_launches(0xFF), "ms_total": total / reps,
+             "ms_to_task_logits": [x / reps for x in acc],
+             "task_finish_wave": [t.fork_depth + t.branch_layers for t in cfg.tasks]})
+        model.close()
     if not a.quick:
         del weights, blob
         big = synth.config_large8()

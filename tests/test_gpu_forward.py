@@ -229,6 +229,43 @@ def test_host_entry_point_and_error_paths():
     assert e.value.code == -4
 
 
+def test_early_heads_deliver_shallow_tasks_first_with_the_same_bits():
+    """Section 5.2 names the latency limitation of the merged model (no output before all tasks are
+    done).  With early_heads every task's head follows the wave that completes it and its event fires
+    then; the logits are bit-identical to the throughput-oriented schedule."""
+    cfg = synth.config_glue8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_glue8(cfg)
+    _, base = run_model(cfg, blob, batch)
+    model = mt.MTModel(cfg, 32, 128)
+    model.set_option("early_heads", 1)
+    model.load_weights(blob)
+    tok, seg, lens = dev_batch(batch)
+    logits = torch.zeros_like(base)
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    model.forward(tok, seg, lens, logits)           # builds the plan
+    torch.cuda.synchronize()
+    start.record()
+    model.forward_events(tok, seg, lens, logits, events)
+    end.record()
+    torch.cuda.synchronize()
+    assert torch.equal(logits, base)
+    done = [start.elapsed_time(e) for e in events]
+    total = start.elapsed_time(end)
+    finish_wave = [t.fork_depth + t.branch_layers for t in cfg.tasks]     # 9 8 9 8 7 8 7 10
+    order = sorted(range(8), key=lambda t: done[t])
+    assert [finish_wave[t] for t in order] == sorted(finish_wave)
+    assert min(done) < 0.85 * total, f"first task at {min(done):.3f} ms of {total:.3f} ms"
+    # events are optional per task, and also work with the default schedule (all at the end)
+    model.set_option("early_heads", 0)
+    some = [None] * 8
+    some[3] = torch.cuda.Event(enable_timing=True)
+    model.forward_events(tok, seg, lens, logits, some)
+    some[3].synchronize()
+    assert torch.equal(logits, base)
+
+
 def test_production_shaped_tree_with_21_tasks():
     """App. E serves 21 tasks from one model (8 shared layers, ~1.5 task layers per task).  More tasks
     than one grouped launch holds: waves, first-token tails and heads are split into chunks."""

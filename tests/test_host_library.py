@@ -77,6 +77,12 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     assert m.plan_launches(0xFF) == 2 + 7 * 4 + 7 + 7 + 8 + 8 + 8 + 2 + 5 + 2
     m.set_option("cls_only_last_layer", 0)
     assert m.plan_launches(0xFF) == 2 + 7 * 10 + 2   # row starts + embedding, 7 per wave, pooler + head at the end
+    # early_heads: tasks finish after waves 7 (2 tasks), 8 (3), 9 (2), 10 (1): four pooler + head pairs, and
+    # with first-token-only last layers four grouped tails of 5 launches instead of one
+    m.set_option("early_heads", 1)
+    assert m.plan_launches(0xFF) == 2 + 7 * 10 + 2 * 4
+    m.set_option("cls_only_last_layer", 1)
+    assert m.plan_launches(0xFF) == 2 + 7 * 4 + 7 + 7 + 8 + 8 + 8 + 2 + 5 * 4 + 2 * 4
     m.close()
     m2 = binding.MTModel(cfg, 32, 128, max_groups=2, bind=False)
     m2.set_option("cls_only_last_layer", 0)
