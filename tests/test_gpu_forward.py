@@ -316,6 +316,18 @@ def test_glue8_tree_batch32_seq128_sampled_rows():
                 assert torch.equal(part[:, offs[t]:offs[t + 1]], logits[:, offs[t]:offs[t + 1]])
 
 
+def test_glue8_tree_batch256_sampled_rows():
+    """Largest batch of the serving sweep (256 x 128 = 32768 padded rows, lengths from 1)."""
+    cfg = synth.config_glue8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 256, 128, 1, 128, seed=8)
+    model, logits = run_model(cfg, blob, batch)
+    order = np.argsort(batch.lengths)
+    check_against_oracle(cfg, wf, batch, model, logits, rows=[int(order[0]), int(order[128]), int(order[-1]), 255],
+                         check_hidden=False)
+    assert torch.isfinite(logits).all()
+
+
 def test_glue8_tree_long_sequences_sampled_rows():
     cfg = synth.config_glue8()
     w, blob, wf = cached_weights(cfg, 0)
