@@ -35,15 +35,16 @@ constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;  // 4 s
 
 constexpr int kStagingBytes = 4096;  // 32 rows x 128 bytes, one epilogue chunk of one warp
-__host__ __device__ constexpr int gemm_stages(int bn) { return bn == 128 ? 5 : 4; }
+// A CTA of a pair stages only its half of the W tile, which leaves room for more stages.
+__host__ __device__ constexpr int gemm_stages(int bn, bool pair) { return pair ? 5 : (bn == 128 ? 5 : 4); }
 // staging buffers per epilogue warp: two where shared memory allows (needed to prefetch residuals)
-__host__ __device__ constexpr int gemm_staging_bufs(int bn) { return bn == 256 ? 1 : 2; }
+__host__ __device__ constexpr int gemm_staging_bufs(int bn, bool pair) { return (bn == 256 && !pair) ? 1 : 2; }
 __host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
-__host__ __device__ constexpr int gemm_b_bytes(int bn) { return bn * kGemmBlockK * 2; }
-__host__ __device__ constexpr int gemm_smem_bytes(int bn) {
+__host__ __device__ constexpr int gemm_b_bytes(int bn, bool pair) { return (pair ? bn / 2 : bn) * kGemmBlockK * 2; }
+__host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair) {
   // stages + staging + barriers/bookkeeping + slack for manual 1024-byte alignment
-  return gemm_stages(bn) * (gemm_a_bytes() + gemm_b_bytes(bn)) +
-         kNumEpilogueWarps * gemm_staging_bufs(bn) * kStagingBytes + 512 + 1024;
+  return gemm_stages(bn, pair) * (gemm_a_bytes() + gemm_b_bytes(bn, pair)) +
+         kNumEpilogueWarps * gemm_staging_bufs(bn, pair) * kStagingBytes + 512 + 1024;
 }
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -123,6 +124,61 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 // Makes this thread's shared-memory writes visible to the TMA unit.
 __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster work on one 256-row tile ------------------
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Shared-memory address of `addr` (an address of this CTA) in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// All threads of both CTAs.  Only used where every thread is known to arrive (set-up and exit).
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Tile load of a CTA pair: data lands in this CTA, the bytes are counted on the barrier `bar_cluster`,
+// which may live in the other CTA of the pair (no multicast: every CTA fetches its own part).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar_cluster)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D (+)= A . B^T over the pair: 256 x N x 16; each CTA holds 128 rows of A and D and N/2 rows of B.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// One arrival on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued
+// so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(static_cast<uint16_t>(3))
+      : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -213,12 +269,19 @@ __device__ __forceinline__ uint32_t staging_off(int r, int c) {
   return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4));
 }
 
-template <int BN, int EPI>
+// PAIR: the kernel runs as clusters of two CTAs that share 256 x BN tiles (tcgen05 cta_group::2).
+// CTA `rank` of a pair owns rows rank*128.. of the tile (its A rows, its accumulator, its epilogue)
+// and stages half of the W tile; the MMA, issued by rank 0, reads both halves.  Per 128 x BN x 64
+// of tensor work a CTA then pulls 16 KB + BN/2 x 128 B from L2 instead of 16 KB + BN x 128 B, which
+// is what bounds the single-CTA kernel (an SM takes in roughly 64 bytes per clock).
+template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __grid_constant__ GemmParams p) {
-  constexpr int STAGES = gemm_stages(BN);
+  constexpr int STAGES = gemm_stages(BN, PAIR);
   constexpr int A_BYTES = gemm_a_bytes();
-  constexpr int B_BYTES = gemm_b_bytes(BN);
-  constexpr int NBUF = gemm_staging_bufs(BN);
+  constexpr int B_BYTES = gemm_b_bytes(BN, PAIR);   // this CTA's part of the W tile
+  constexpr int NBUF = gemm_staging_bufs(BN, PAIR);
+  constexpr int TILE_M = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
+  constexpr int ACC_ARRIVALS = PAIR ? 2 * kNumEpilogueWarps : kNumEpilogueWarps;
   constexpr uint32_t TMEM_COLS = BN == 128 ? 256 : 512;  // two accumulators; a power of two >= 32
   static_assert(BN == 128 || BN == 192 || BN == 256, "tile widths implemented: 128, 192, 256");
   static_assert(EPI != kEpiBiasResidual || NBUF == 2, "the residual epilogue prefetches: two staging buffers");
@@ -239,6 +302,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_cta_rank() : 0u;           // 0 = the CTA that issues the MMAs
+  const int worker = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
   const int n_tiles_n = p.N / BN;
   const int k_blocks = p.K / kGemmBlockK;
@@ -250,18 +316,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_acc_full + 8 * a, 1);
-      mbar_init(bar_acc_empty + 8 * a, kNumEpilogueWarps);
+      mbar_init(bar_acc_empty + 8 * a, ACC_ARRIVALS);
     }
     for (int i = 0; i < 2 * kNumEpilogueWarps; ++i) mbar_init(bar_res + 8 * i, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  if (warp == 1) {
+    if (PAIR) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS); else tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  }
   tc_fence_before();
-  __syncthreads();
+  // the partner's barriers must exist before anything of this CTA can signal them
+  __syncwarp();
+  if (PAIR) cluster_sync_all(); else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // where the "stage full" barriers are counted: in rank 0 of a pair
+  const uint32_t bar_full_count = PAIR ? map_to_cta(bar_full, 0) : bar_full;
   // Tiles are numbered m-tile outermost: tile = (m_tile * n_groups + g) * n_tiles_n + n_tile, so the
   // group and the column block of a tile do not depend on the (device-side) number of rows.
   const int tiles_per_m = p.n_groups * n_tiles_n;
@@ -271,15 +343,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   // has completed and its writes are visible.
   int prefetched = 0;   // stages whose W tile is already on its way (producer thread only)
   if (warp == 0 && lane == 0) {
-    const int rem = static_cast<int>(blockIdx.x) % tiles_per_m;
+    const int rem = worker % tiles_per_m;
     const int g = rem / n_tiles_n;
-    const int n0 = (rem - g * n_tiles_n) * BN;
+    const int n0 = (rem - g * n_tiles_n) * BN + static_cast<int>(rank) * (PAIR ? BN / 2 : 0);
     prefetch_tensormap(&p.tmap_x[g]);
     prefetch_tensormap(&p.tmap_w[g]);
     prefetched = k_blocks < STAGES ? k_blocks : STAGES;
     for (int s = 0; s < prefetched; ++s) {
-      mbar_add_tx(bar_full + 8 * s, B_BYTES);
-      tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full + 8 * s);
+      if (PAIR) {
+        // rank 0 announces the bytes of both CTAs' W parts on its barrier; either CTA's copy may land first
+        if (rank == 0) mbar_add_tx(bar_full + 8 * s, 2 * B_BYTES);
+        tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full_count + 8 * s);
+      } else {
+        mbar_add_tx(bar_full + 8 * s, B_BYTES);
+        tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full + 8 * s);
+      }
     }
   }
   grid_dependency_wait();
@@ -287,7 +365,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   // rows in use: all M, or fewer when the token layout is packed (a device-side count)
   int m_rows = p.M;
   if (p.m_valid != nullptr) m_rows = min(m_rows, *p.m_valid);
-  const int n_tiles_m = (m_rows + kGemmBlockM - 1) / kGemmBlockM;
+  const int n_tiles_m = (m_rows + TILE_M - 1) / TILE_M;
   const int total_tiles = n_tiles_m * tiles_per_m;
 
   if (warp == 0) {
@@ -297,9 +375,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
-      if (static_cast<int>(blockIdx.x) >= total_tiles) {
-        // no tile for this CTA after all (fewer rows in use than the grid was sized for): let the
-        // early W tiles land before the CTA retires
+      if (worker >= total_tiles && rank == 0) {
+        // no tile for this CTA (pair) after all (fewer rows in use than the grid was sized for): let
+        // the early W tiles land before the CTA retires (in a pair, rank 1 is held by the exit barrier)
         for (int s = 0; s < prefetched; ++s) {
           mbar_arrive(bar_full + 8 * s);
           const unsigned long long t0 = global_timer_ns();
@@ -308,28 +386,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           }
         }
       }
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / tiles_per_m) * kGemmBlockM;
+      for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+        const int m0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM;
         const int rem = tile % tiles_per_m;
         const int g = rem / n_tiles_n;
-        const int n0 = (rem - g * n_tiles_n) * BN;
+        const int n0 = (rem - g * n_tiles_n) * BN + static_cast<int>(rank) * (PAIR ? BN / 2 : 0);
         for (int kb = 0; kb < k_blocks; ++kb) {
+          // this CTA's stage is free once the MMAs that read it (in both CTAs of a pair) are done
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          if (prefetched > 0) {
-            // the W tile of this stage was started before the dependency wait
-            --prefetched;
-            mbar_expect_tx(bar_full + 8 * stage, A_BYTES);
-            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+          const bool w_on_its_way = prefetched > 0;
+          if (w_on_its_way) --prefetched;
+          if (PAIR) {
+            if (rank == 0)
+              mbar_expect_tx(bar_full + 8 * stage, 2 * A_BYTES + (w_on_its_way ? 0 : 2 * B_BYTES));
+            tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full_count + 8 * stage);
+            if (!w_on_its_way)
+              tma_load_2d_pair(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full_count + 8 * stage);
           } else {
-            mbar_expect_tx(bar_full + 8 * stage, A_BYTES + B_BYTES);
+            mbar_expect_tx(bar_full + 8 * stage, A_BYTES + (w_on_its_way ? 0 : B_BYTES));
             tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
-            tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+            if (!w_on_its_way)
+              tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
           }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
+      if (!ok && rank == 0) {
         // Aborting: wait (bounded) until the copies still in flight have landed, so that the
         // CTA does not retire underneath them.  The last min(issued, STAGES) fills are the ones
         // that may be pending; walk back over them.
@@ -348,14 +431,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kGemmBlockM, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(TILE_M, BN);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+        // the epilogue warps (of both CTAs of a pair) have drained this accumulator
         if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -367,13 +451,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 #pragma unroll
           for (int k = 0; k < kGemmBlockK / 16; ++k) {
             // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the address field
-            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if (PAIR) umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit(bar_empty + 8 * stage);
+          if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(bar_acc_full + 8 * acc);
+        if (PAIR) umma_commit_pair(bar_acc_full + 8 * acc); else umma_commit(bar_acc_full + 8 * acc);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -400,7 +485,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     auto prefetch_residual = [&](int tile, int chunk, int b) {
       const int rem = tile % tiles_per_m;
       const int g = rem / n_tiles_n;
-      const int row0 = (tile / tiles_per_m) * kGemmBlockM + quarter * 32;
+      const int row0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM + quarter * 32;
       const int col0 = (rem - g * n_tiles_n) * BN + chunk * CHUNK_COLS;
       // the store issued last read this very buffer: it must be done with it before TMA refills it
       tma_store_wait_read<0>();
@@ -408,11 +493,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       tma_load_2d(my_stage + b * kStagingBytes, &p.tmap_res[g], col0, row0, my_res_bar + 8 * b);
     };
 
-    if (EPI == kEpiBiasResidual && lane == 0 && static_cast<int>(blockIdx.x) < total_tiles)
-      prefetch_residual(blockIdx.x, col_group, 0);
+    if (EPI == kEpiBiasResidual && lane == 0 && worker < total_tiles) prefetch_residual(worker, col_group, 0);
+    // a pair's accumulator is free again when the epilogue warps of both CTAs are done with it
+    const uint32_t bar_acc_empty_count = (PAIR && rank != 0) ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;
 
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int m0 = (tile / tiles_per_m) * kGemmBlockM;
+    for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+      const int m0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM;
       const int rem = tile % tiles_per_m;
       const int g = rem / n_tiles_n;
       const int n0 = (rem - g * n_tiles_n) * BN;
@@ -432,7 +518,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           // chunk of this CTA's next tile) into the other buffer
           if (lane == 0) {
             int nt = tile, nc = chunk + COL_GROUPS;
-            if (nc >= CHUNKS) { nt = tile + gridDim.x; nc = col_group; }
+            if (nc >= CHUNKS) { nt = tile + n_workers; nc = col_group; }
             if (nt < total_tiles) prefetch_residual(nt, nc, buf ^ 1);
           }
           __syncwarp();
@@ -504,7 +590,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+      if (lane == 0) {
+        if (PAIR && rank != 0) mbar_arrive_cluster(bar_acc_empty_count + 8 * acc);
+        else mbar_arrive(bar_acc_empty + 8 * acc);
+      }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
     // shared memory must outlive the stores that still read it
@@ -514,44 +603,60 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
   // ------------------------------ teardown ------------------------------------
   tc_fence_before();
-  __syncthreads();
+  // In a pair neither CTA may retire (or free tensor memory) while the other can still signal its
+  // barriers or while MMAs that read its shared memory may be in flight: every thread of both CTAs
+  // gets here (all waits above are bounded), so this barrier completes.
+  __syncwarp();
+  if (PAIR) cluster_sync_all(); else __syncthreads();
   if (threadIdx.x == 0 && *abort_flag && p.status != nullptr) atomicOr(p.status, kFlagWaitTimeout);
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool PAIR>
 cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
-  auto kernel = gemm_bf16_tcgen05<BN, EPI>;
+  auto kernel = gemm_bf16_tcgen05<BN, EPI, PAIR>;
   static bool configured = false;  // per instantiation; the attribute is per function and per device
   static int configured_device = -1;
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (!configured || configured_device != dev) {
-    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN));
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN, PAIR));
     if (err != cudaSuccess) return err;
     configured = true;
     configured_device = dev;
   }
-  const int tiles = ((p.M + kGemmBlockM - 1) / kGemmBlockM) * (p.N / BN) * p.n_groups;
-  const int grid = tiles < sm_count ? tiles : sm_count;
-  if (grid <= 0) return cudaSuccess;
-  return launch_kernel(kernel, dim3(grid), dim3(kGemmThreads), gemm_smem_bytes(BN), stream, p);
+  constexpr int tile_m = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
+  const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN) * p.n_groups;
+  const int workers_max = PAIR ? sm_count / 2 : sm_count;
+  const int workers = tiles < workers_max ? tiles : workers_max;
+  if (workers <= 0) return cudaSuccess;
+  return launch_kernel(kernel, dim3(PAIR ? 2 * workers : workers), dim3(kGemmThreads), gemm_smem_bytes(BN, PAIR), stream,
+                       p, PAIR ? 2u : 1u);
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   switch (epilogue) {
-    case kEpiBias: return launch_one<BN, kEpiBias>(p, sm_count, stream);
-    case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu>(p, sm_count, stream);
+    case kEpiBias: return launch_one<BN, kEpiBias, PAIR>(p, sm_count, stream);
+    case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu, PAIR>(p, sm_count, stream);
     case kEpiBiasResidual:
-      if constexpr (BN != 256) return launch_one<BN, kEpiBiasResidual>(p, sm_count, stream);
-      return cudaErrorInvalidValue;  // no room for two staging buffers beside 256-wide stages
+      if constexpr (BN != 256) return launch_one<BN, kEpiBiasResidual, PAIR>(p, sm_count, stream);
+      return cudaErrorInvalidValue;  // 256-wide tiles are not used with the residual epilogue
     default: return cudaErrorInvalidValue;
+  }
+}
+
+template <bool PAIR>
+cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
+  switch (gemm_block_n(p.N, epilogue)) {
+    case 256: return launch_bn<256, PAIR>(p, epilogue, sm_count, stream);
+    case 192: return launch_bn<192, PAIR>(p, epilogue, sm_count, stream);
+    default: return launch_bn<128, PAIR>(p, epilogue, sm_count, stream);
   }
 }
 
@@ -562,15 +667,13 @@ int gemm_block_n(int N, int epilogue) {
   return N % 192 == 0 ? 192 : 128;  // 768 = 4 x 192: 128 tiles per 4096 rows, one wave of 148 SMs
 }
 int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
+bool g_gemm_pair = true;
+int gemm_w_box_rows(int N, int epilogue) { return gemm_block_n(N, epilogue) / (g_gemm_pair ? 2 : 1); }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
     return cudaErrorInvalidValue;
-  switch (gemm_block_n(p.N, epilogue)) {
-    case 256: return launch_bn<256>(p, epilogue, sm_count, stream);
-    case 192: return launch_bn<192>(p, epilogue, sm_count, stream);
-    default: return launch_bn<128>(p, epilogue, sm_count, stream);
-  }
+  return g_gemm_pair ? launch_any<true>(p, epilogue, sm_count, stream) : launch_any<false>(p, epilogue, sm_count, stream);
 }
 
 }  // namespace mt

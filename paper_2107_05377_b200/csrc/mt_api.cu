@@ -157,7 +157,7 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
   const bool res = epilogue == kEpiBiasResidual;
   cudaError_t e;
   if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
-  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_block_n(N, epilogue), kGemmBlockK, false)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_w_box_rows(N, epilogue), kGemmBlockK, false)) != cudaSuccess) return e;
   if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), res)) != cudaSuccess) return e;
   if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
   g->group[i].bias = bias;
@@ -658,6 +658,11 @@ const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c
 
 int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
+  if (strcmp(key, "gemm_pair") == 0) {  // process-wide; plans hold tensor maps sized for one mode
+    g_gemm_pair = value != 0;
+    m->plans.clear();
+    return MT_OK;
+  }
   if (strcmp(key, "pdl") == 0) {  // process-wide: programmatic dependent launch on or off
     g_use_pdl = value != 0;
     return MT_OK;

@@ -32,19 +32,31 @@ extern bool g_use_pdl;
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// cluster_x > 1 launches the grid as thread-block clusters of that many CTAs along x.
 template <typename Param>
 cudaError_t launch_kernel(void (*kernel)(Param), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                          const Param& param) {
+                          const Param& param, unsigned cluster_x = 1) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (g_use_pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = g_use_pdl ? 1 : 0;
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, param);
 }
 #endif
@@ -75,6 +87,10 @@ struct alignas(64) GemmParams {
 // and the width in elements of the 128-byte output box (64 bf16 or 32 fp32 columns; 32 rows).
 int gemm_block_n(int N, int epilogue);
 int gemm_out_box_cols(int epilogue);
+// g_gemm_pair: run the GEMM as pairs of CTAs sharing 256-row tiles (each CTA stages half of a W
+// tile); gemm_w_box_rows is the number of W rows one TMA box fetches (the tile width or half of it).
+extern bool g_gemm_pair;
+int gemm_w_box_rows(int N, int epilogue);
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
 
 // Token layout.  The rows of sequence b start at row_start[b] (device array of batch + 1 ints written
