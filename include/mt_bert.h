@@ -179,9 +179,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * layer's state at position 0 and zeros elsewhere.  key "early_heads" (0/1, default 0, any time): see mt_forward_events.
  * key "pack_tokens" (0/1, default 1, any time): store
  * and compute only the valid tokens of every sequence (rows of sequence b follow those of b-1) instead
- * of batch*seq padded rows; logits agree to rounding either way.  key "gemm_pair" (0/1, default 1, whole process; set it before
- * the first forward of every model in the process): run the GEMMs as pairs of CTAs on 256-row tiles
- * (tcgen05 cta_group::2) instead of single CTAs on 128-row tiles.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * of batch*seq padded rows; logits agree to rounding either way.  key "gemm_pair" (0/1, default 0, any time): run the GEMMs as pairs of
+ * CTAs on 256-row tiles (tcgen05 cta_group::2, each CTA stages half of a weight tile) instead of single
+ * CTAs on 128-row tiles; about 3 % faster on large problems, no gain at the 32 x 128 workload.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);
@@ -217,9 +217,10 @@ const char* mt_last_error_string(const mt_model* m);
 /* Y[M,N] = epilogue(X[M,K] . W[N,K]^T + bias[N]) on tcgen05 tensor cores (X, W, bias bf16; fp32
  * accumulate).  epilogue 0: +bias, Y bf16; 1: +bias then erf-GELU, Y bf16; 2: +bias +residual with
  * residual fp32 [M,N] and Y fp32 [M,N] (the LayerNorm input).  K % 64 == 0, N % 128 == 0, all
- * pointers 16-byte aligned.  This is one linear map of the layer above. */
+ * pointers 16-byte aligned.  cta_pair != 0 runs it as pairs of CTAs (see option "gemm_pair").  This is
+ * one linear map of the layer above. */
 int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
-                     void* d_y, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                     void* d_y, int32_t M, int32_t N, int32_t K, int32_t epilogue, int32_t cta_pair,
                      uint32_t* d_status, void* stream);
 
 /* ctx[B*S, heads*64] = softmax(QK^T/8 masked to keys < length) V per (sequence, head), from the

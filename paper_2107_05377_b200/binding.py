@@ -53,7 +53,7 @@ SIGNATURES = {
     "mt_debug_copy_hidden": (C.c_int, [_P, _I32, _I32, _P, _P]),
     "mt_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "mt_last_error_string": (C.c_char_p, [_P]),
-    "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
@@ -110,11 +110,11 @@ def _stream(stream=None) -> int:
 # single steps (device tensors in, device tensors out)
 # ---------------------------------------------------------------------------
 
-def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream=None) -> None:
+def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream=None, cta_pair: bool = False) -> None:
     M, K = x.shape
     N = w.shape[0]
     _check(lib().mt_kernel_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), M, N, K, epilogue,
-                                  _ptr(status), _stream(stream)), "mt_kernel_linear")
+                                  1 if cta_pair else 0, _ptr(status), _stream(stream)), "mt_kernel_linear")
 
 
 def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None) -> None:

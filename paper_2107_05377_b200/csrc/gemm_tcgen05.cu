@@ -667,13 +667,12 @@ int gemm_block_n(int N, int epilogue) {
   return N % 192 == 0 ? 192 : 128;  // 768 = 4 x 192: 128 tiles per 4096 rows, one wave of 148 SMs
 }
 int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
-bool g_gemm_pair = true;
-int gemm_w_box_rows(int N, int epilogue) { return gemm_block_n(N, epilogue) / (g_gemm_pair ? 2 : 1); }
+int gemm_w_box_rows(int N, int epilogue, bool pair) { return gemm_block_n(N, epilogue) / (pair ? 2 : 1); }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
     return cudaErrorInvalidValue;
-  return g_gemm_pair ? launch_any<true>(p, epilogue, sm_count, stream) : launch_any<false>(p, epilogue, sm_count, stream);
+  return p.pair ? launch_any<true>(p, epilogue, sm_count, stream) : launch_any<false>(p, epilogue, sm_count, stream);
 }
 
 }  // namespace mt

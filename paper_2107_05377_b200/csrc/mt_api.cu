@@ -157,7 +157,7 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
   const bool res = epilogue == kEpiBiasResidual;
   cudaError_t e;
   if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
-  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_w_box_rows(N, epilogue), kGemmBlockK, false)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_w_box_rows(N, epilogue, g->pair != 0), kGemmBlockK, false)) != cudaSuccess) return e;
   if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), res)) != cudaSuccess) return e;
   if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
   g->group[i].bias = bias;
@@ -182,6 +182,7 @@ struct mt_model {
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
   bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
+  bool gemm_pair;    // GEMMs as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2)
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
 
   // device memory (caller-owned)
@@ -348,6 +349,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K) {
     memset(g, 0, sizeof(*g));
     g->M = rows; g->N = N; g->K = K;
+    g->pair = m->gemm_pair ? 1 : 0;
     g->m_valid = rows_valid;
     g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   };
@@ -396,6 +398,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   memset(&ck->qkv, 0, sizeof(ck->qkv));
   ck->qkv.n_groups = static_cast<int32_t>(count);
   ck->qkv.M = M; ck->qkv.N = 3 * H; ck->qkv.K = H;
+  ck->qkv.pair = m->gemm_pair ? 1 : 0;
   ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   init_tail(m, &ck->full, M, false);
@@ -597,6 +600,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->pack_tokens = true;
   m->cls_only = true;
   m->early_heads = false;
+  m->gemm_pair = false;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -658,8 +662,8 @@ const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c
 
 int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
-  if (strcmp(key, "gemm_pair") == 0) {  // process-wide; plans hold tensor maps sized for one mode
-    g_gemm_pair = value != 0;
+  if (strcmp(key, "gemm_pair") == 0) {
+    m->gemm_pair = value != 0;
     m->plans.clear();
     return MT_OK;
   }
@@ -1024,7 +1028,7 @@ int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out, 
 // ---- single steps ------------------------------------------------------------------------------
 
 int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual, void* d_y, int32_t M,
-                     int32_t N, int32_t K, int32_t epilogue, uint32_t* d_status, void* stream) {
+                     int32_t N, int32_t K, int32_t epilogue, int32_t cta_pair, uint32_t* d_status, void* stream) {
   if (d_x == nullptr || d_w == nullptr || d_bias == nullptr || d_y == nullptr || M < 1 || N < 128 || N % 128 != 0 ||
       K < 64 || K % 64 != 0 || epilogue < 0 || epilogue > 2 || (epilogue == 2 && d_residual == nullptr))
     return MT_ERR_INVALID_ARG;
@@ -1035,6 +1039,7 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
+  p.pair = cta_pair != 0 ? 1 : 0;
   if (set_gemm_group(&p, 0, epilogue, d_x, d_w, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
                      d_y) != cudaSuccess)
     return MT_ERR_CUDA;

@@ -80,6 +80,7 @@ struct alignas(64) GemmParams {
   int32_t n_groups;
   int32_t M, N, K;
   const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
+  int32_t pair;            // 1: run as pairs of CTAs on 256-row tiles (the W maps then fetch half a tile's rows)
   uint32_t* status;        // sticky device status word (may be null)
 };
 
@@ -87,10 +88,9 @@ struct alignas(64) GemmParams {
 // and the width in elements of the 128-byte output box (64 bf16 or 32 fp32 columns; 32 rows).
 int gemm_block_n(int N, int epilogue);
 int gemm_out_box_cols(int epilogue);
-// g_gemm_pair: run the GEMM as pairs of CTAs sharing 256-row tiles (each CTA stages half of a W
-// tile); gemm_w_box_rows is the number of W rows one TMA box fetches (the tile width or half of it).
-extern bool g_gemm_pair;
-int gemm_w_box_rows(int N, int epilogue);
+// Rows of W one TMA box fetches: the tile width, or half of it when the GEMM runs as CTA pairs
+// (each CTA of a pair stages half of the W tile).
+int gemm_w_box_rows(int N, int epilogue, bool pair);
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
 
 // Token layout.  The rows of sequence b start at row_start[b] (device array of batch + 1 ints written

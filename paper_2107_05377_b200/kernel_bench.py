@@ -22,6 +22,7 @@ from . import binding as mt
 
 L2_FLUSH_BYTES = 256 << 20
 USE_GRAPH = False
+CTA_PAIR = False
 
 
 def _time(fn, iters, warmup, flush):
@@ -71,7 +72,7 @@ def bench_linear(m, n, k, epilogue, iters, warmup, flush):
     b = (0.02 * torch.randn(n, device="cuda")).to(torch.bfloat16)
     r = torch.randn(m, n, device="cuda") if epilogue == 2 else None
     y = torch.empty(m, n, device="cuda", dtype=torch.float32 if epilogue == 2 else torch.bfloat16)
-    ms = _time(lambda: mt.mt_kernel_linear(x, w, b, r, y, epilogue), iters, warmup, flush)
+    ms = _time(lambda: mt.mt_kernel_linear(x, w, b, r, y, epilogue, cta_pair=CTA_PAIR), iters, warmup, flush)
     flops = 2.0 * m * n * k
     bytes_ = 2.0 * (m * k + n * k) + (8.0 if epilogue == 2 else 2.0) * m * n
     return {"kernel": "linear", "M": m, "N": n, "K": k, "epilogue": epilogue, "us": 1e3 * ms,
@@ -119,9 +120,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--flush", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
+    ap.add_argument("--pair", action="store_true", help="linear: pairs of CTAs on 256-row tiles (cta_group::2)")
     a = ap.parse_args()
-    global USE_GRAPH
+    global USE_GRAPH, CTA_PAIR
     USE_GRAPH = a.graph
+    CTA_PAIR = a.pair
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))

@@ -16,9 +16,12 @@ HIDDEN_REL_L2 = 1e-2   # tolerance on hidden states (valid rows)
 LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
-def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None):
+def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None,
+              gemm_pair=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
+    if gemm_pair is not None:
+        model.set_option("gemm_pair", gemm_pair)
     if pack_tokens is not None:
         model.set_option("pack_tokens", pack_tokens)
     if cls_only is not None:
@@ -98,6 +101,26 @@ def test_every_token_in_last_branch_layers_matches_oracle_and_first_token_only()
     check_against_oracle(cfg, wf, batch, model, full, rows=range(6), cls_only=False)
     _, first = run_model(cfg, blob, batch)
     assert float((first - full).abs().max()) <= 2e-3
+
+
+def test_cta_pair_gemms_match_oracle_and_single_cta_bits():
+    """GEMMs run as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2): parity with the oracle on
+    every hidden state; every output element is still one fixed-order sum over K, so the logits are
+    bit-identical to the single-CTA tiles."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
+    model, paired = run_model(cfg, blob, batch, debug=True, gemm_pair=1)
+    check_against_oracle(cfg, wf, batch, model, paired, rows=range(6))
+    _, single = run_model(cfg, blob, batch)
+    assert torch.equal(paired, single)
+    big = synth.config_glue8()
+    w8, blob8, wf8 = cached_weights(big, 0)
+    b8 = synth.batch_glue8(big)
+    _, p8 = run_model(big, blob8, b8, gemm_pair=1)
+    _, s8 = run_model(big, blob8, b8)
+    assert torch.equal(p8, s8)
 
 
 def test_padded_layout_matches_oracle_and_packed_layout():

@@ -32,7 +32,8 @@ def bf16_round_tol(want):
     (1000, 1024, 4096, 2),    # BERT-large width
     (520, 4096, 1024, 1),
 ])
-def test_linear_matches_oracle(M, N, K, epi):
+@pytest.mark.parametrize("pair", [False, True], ids=["single_cta", "cta_pair"])
+def test_linear_matches_oracle(M, N, K, epi, pair):
     xb, x = rand_bf16(11, f"x{M}.{N}.{K}", (M, K), 1.0)
     wb, w = rand_bf16(12, f"w{M}.{N}.{K}", (N, K), 0.05)
     bb, b = rand_bf16(13, f"b{M}.{N}.{K}", (N,), 0.5)
@@ -41,7 +42,7 @@ def test_linear_matches_oracle(M, N, K, epi):
     y = torch.full((M + 8, N), float("nan"), dtype=out_dtype, device="cuda")   # 8 guard rows
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     mt.mt_kernel_linear(to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(bb),
-                        torch.from_numpy(r32).cuda() if epi == 2 else None, y[:M], epi, status=status)
+                        torch.from_numpy(r32).cuda() if epi == 2 else None, y[:M], epi, status=status, cta_pair=pair)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     want = orc.linear(x, w, b)
