@@ -179,9 +179,10 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * layer's state at position 0 and zeros elsewhere.  key "early_heads" (0/1, default 0, any time): see mt_forward_events.
  * key "pack_tokens" (0/1, default 1, any time): store
  * and compute only the valid tokens of every sequence (rows of sequence b follow those of b-1) instead
- * of batch*seq padded rows; logits agree to rounding either way.  key "gemm_pair" (0/1, default 0, any time): run the GEMMs as pairs of
- * CTAs on 256-row tiles (tcgen05 cta_group::2, each CTA stages half of a weight tile) instead of single
- * CTAs on 128-row tiles; about 3 % faster on large problems, no gain at the 32 x 128 workload.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * of batch*seq padded rows; logits agree to rounding either way.  key "gemm_pair" (0 never, 1 always, 2 = by launch size, the default; any
+ * time): run GEMM launches as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2, each CTA stages half
+ * of a weight tile) instead of single CTAs on 128-row tiles; faster on large launches (+11 % at 8192^3),
+ * slower on small ones; the results are bit-identical.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);

@@ -182,7 +182,7 @@ struct mt_model {
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
   bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
-  bool gemm_pair;    // GEMMs as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2)
+  int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
 
   // device memory (caller-owned)
@@ -342,14 +342,22 @@ bool is_cls_op(const mt_model* m, const OpDesc& op) {
   return m->cls_only && op.task >= 0 && op.layer == m->tasks[op.task].cfg.branch_layers;
 }
 
-void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid) {
+// Whether a grouped GEMM launch of `groups` problems of `rows` (padded) rows runs as CTA pairs.  Pairs
+// stage half as many weight bytes per CTA but tile rows by 256: measured faster from about three
+// layers' worth of the 32 x 128 batch per launch, slower below.  The result is the same bits either way.
+int32_t use_pair(const mt_model* m, int64_t rows, int64_t groups) {
+  if (m->gemm_pair != 2) return m->gemm_pair;
+  return rows * groups >= 12288 ? 1 : 0;
+}
+
+void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
   const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
   const int32_t* rows_valid =
       all_rows_valid ? nullptr : reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K) {
     memset(g, 0, sizeof(*g));
     g->M = rows; g->N = N; g->K = K;
-    g->pair = m->gemm_pair ? 1 : 0;
+    g->pair = use_pair(m, rows, groups);
     g->m_valid = rows_valid;
     g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   };
@@ -398,10 +406,12 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   memset(&ck->qkv, 0, sizeof(ck->qkv));
   ck->qkv.n_groups = static_cast<int32_t>(count);
   ck->qkv.M = M; ck->qkv.N = 3 * H; ck->qkv.K = H;
-  ck->qkv.pair = m->gemm_pair ? 1 : 0;
+  ck->qkv.pair = use_pair(m, M, static_cast<int64_t>(count));
   ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
-  init_tail(m, &ck->full, M, false);
+  int32_t n_full = 0;
+  for (size_t i = 0; i < count; ++i) n_full += is_cls_op(m, ops[first + i]) ? 0 : 1;
+  init_tail(m, &ck->full, M, false, n_full);
   ck->n_cls = 0;
   memset(&ck->attn, 0, sizeof(ck->attn));
   memset(&ck->attn_cls, 0, sizeof(ck->attn_cls));
@@ -467,7 +477,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
 // Steps 3-7 of the last branch layers of `tasks` on their first tokens ([B, H] rows), one group per task.
 cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks, size_t first, size_t count,
                            int32_t batch, PlanStep* st) {
-  init_tail(m, &st->tail, batch, true);
+  init_tail(m, &st->tail, batch, true, static_cast<int32_t>(count));
   for (size_t i = 0; i < count; ++i) {
     const int32_t t = tasks[first + i];
     const TaskEntry& te = m->tasks[t];
@@ -600,7 +610,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->pack_tokens = true;
   m->cls_only = true;
   m->early_heads = false;
-  m->gemm_pair = false;
+  m->gemm_pair = 2;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -663,7 +673,8 @@ const char* mt_last_error_string(const mt_model* m) { return m ? m->last_error.c
 int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (m == nullptr || key == nullptr) return MT_ERR_INVALID_ARG;
   if (strcmp(key, "gemm_pair") == 0) {
-    m->gemm_pair = value != 0;
+    if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "gemm_pair must be 0, 1 or 2");
+    m->gemm_pair = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
   }

@@ -113,14 +113,16 @@ def test_cta_pair_gemms_match_oracle_and_single_cta_bits():
     batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
     model, paired = run_model(cfg, blob, batch, debug=True, gemm_pair=1)
     check_against_oracle(cfg, wf, batch, model, paired, rows=range(6))
-    _, single = run_model(cfg, blob, batch)
+    _, single = run_model(cfg, blob, batch, gemm_pair=0)
     assert torch.equal(paired, single)
     big = synth.config_glue8()
     w8, blob8, wf8 = cached_weights(big, 0)
     b8 = synth.batch_glue8(big)
     _, p8 = run_model(big, blob8, b8, gemm_pair=1)
-    _, s8 = run_model(big, blob8, b8)
+    _, s8 = run_model(big, blob8, b8, gemm_pair=0)
     assert torch.equal(p8, s8)
+    _, auto8 = run_model(big, blob8, b8)          # default: pairs for the large grouped launches only
+    assert torch.equal(auto8, s8)
 
 
 def test_padded_layout_matches_oracle_and_packed_layout():
