@@ -225,9 +225,13 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
                      uint32_t* d_status, void* stream);
 
 /* ctx[B*S, heads*64] = softmax(QK^T/8 masked to keys < length) V per (sequence, head), from the
- * packed projection qkv[B*S, 3*heads*64] = [Q | K | V].  Rows at positions >= length are written as 0. */
+ * packed projection qkv[B*S, 3*heads*64] = [Q | K | V].  Rows at positions >= length are written as 0.
+ * tensor_memory != 0 (seq <= 128 only, else MT_ERR_INVALID_ARG) selects the tcgen05 kernel, whose
+ * score and output accumulators live in tensor memory; 0 the mma.sync kernel, which takes any seq
+ * (see option "attention_tc").  d_status (device, may be NULL) receives MT_FLAG_WAIT_TIMEOUT. */
 int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx,
-                        int32_t batch, int32_t seq, int32_t heads, void* stream);
+                        int32_t batch, int32_t seq, int32_t heads, int32_t tensor_memory,
+                        uint32_t* d_status, void* stream);
 
 /* y[rows, hidden] = LayerNorm(x) * gamma + beta (fp32 statistics, biased variance) for fp32 x;
  * written as bf16 to d_y and, when d_y_f32 is not NULL, as fp32 too.  hidden in {768, 1024}. */

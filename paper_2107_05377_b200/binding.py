@@ -54,7 +54,7 @@ SIGNATURES = {
     "mt_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "mt_last_error_string": (C.c_char_p, [_P]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
-    "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _P]),
+    "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
                                   _P]),
@@ -117,9 +117,10 @@ def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream
                                   1 if cta_pair else 0, _ptr(status), _stream(stream)), "mt_kernel_linear")
 
 
-def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None) -> None:
-    _check(lib().mt_kernel_attention(_ptr(qkv), _ptr(lengths), _ptr(ctx), batch, seq, heads, _stream(stream)),
-           "mt_kernel_attention")
+def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None,
+                        tensor_memory: bool = False, status=None) -> None:
+    _check(lib().mt_kernel_attention(_ptr(qkv), _ptr(lengths), _ptr(ctx), batch, seq, heads,
+                                     1 if tensor_memory else 0, _ptr(status), _stream(stream)), "mt_kernel_attention")
 
 
 def mt_kernel_layernorm(x, gamma, beta, y, eps: float, y_f32=None, stream=None) -> None:

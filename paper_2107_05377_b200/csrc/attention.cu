@@ -72,7 +72,7 @@ __device__ __forceinline__ void load_tile(uint32_t smem_tile, const bf16* base, 
   }
 }
 
-__global__ void __launch_bounds__(kAttnThreads, 4) attention_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(kAttnThreads, 4) attention_kernel(const __grid_constant__ AttnParams p) {
   // Q tile, then two buffers of (K tile, V tile): the keys of tile t+1 are fetched while tile t is used
   __shared__ __align__(128) uint8_t smem[(kTileQ + 4 * kTileK) * 128];
   const uint32_t sQ = smem_u32(smem);
@@ -382,6 +382,7 @@ cudaError_t launch_cls_attention(const ClsAttnParams& p, cudaStream_t stream) {
 
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1) return cudaErrorInvalidValue;
+  if (p.tensor_memory) return launch_attention_tc(p, stream);
   dim3 grid((p.seq + kTileQ - 1) / kTileQ, p.heads, p.batch * p.n_groups);
   return launch_kernel(attention_kernel, grid, dim3(kAttnThreads), 0, stream, p);
 }

@@ -1,0 +1,257 @@
+// Masked self-attention of the encoder layer on the tcgen05 tensor cores, for sequences of at most
+// 128 tokens (the length the throughput configurations use):
+//   ctx[i, head] = softmax_j( q_i . k_j / sqrt(64),  j < length ) . V        per (sequence, head)
+// from the packed projection qkv[rows, 3H] = [Q | K | V].
+//
+// One CTA of 128 threads = one (layer of the wave, sequence, head); thread t owns query row t, which
+// is lane t of tensor memory.  Steps:
+//   1. one thread fetches the 128 x 64 Q, K and V tiles with three TMA loads (128-byte swizzle; rows
+//      past the end of the buffer arrive as zeros, rows past the sequence's length are another
+//      sequence's finite data or stale memory and are masked: V rows >= length are overwritten with
+//      zeros in shared memory, score columns >= length never enter the softmax)
+//   2. S = Q . K^T: four tcgen05.mma 128 x N x 16 (N = 64 when length <= 64, else 128) into tensor
+//      memory columns [0, N)
+//   3. every thread reads its row of S twice with tcgen05.ld (maximum; then exponentials and their
+//      fp32 sum), rounds the probabilities to bf16 and stores them K-major, 128-byte swizzled, over
+//      the Q and K tiles, which are no longer needed
+//   4. O = P . V: V is the MN-major B operand (its rows are keys = the K dimension), accumulated over
+//      the S columns already consumed
+//   5. O / sum, rounded to bf16, goes through shared memory and leaves as full 128-byte row segments.
+// 50 KB of shared memory and 128 columns of tensor memory per CTA: four CTAs per SM.
+//
+// Both waits are bounded; a wait that runs out raises the timeout flag of the status word, the
+// copies still in flight are given the same limit to land, tensor memory is freed and the CTA returns.
+
+#include "tc_ptx.cuh"
+
+namespace mt {
+namespace {
+
+constexpr int kTcThreads = 128;
+constexpr int kTcRows = kAttnTensorMemoryMaxSeq;  // queries and keys one CTA covers
+constexpr int kTcTileBytes = kTcRows * 128;  // 128 rows of 64 bf16
+constexpr uint32_t kTcTmemCols = 128;
+constexpr int kTcSmemBytes = 3 * kTcTileBytes + 64 + 1024;  // Q, K, V + bookkeeping + alignment slack
+
+// B operand in MN-major form (bit 16): the shared-memory rows of the tile run along K.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_b_mn(int m, int n) { return umma_idesc_bf16(m, n) | (1u << 16); }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __grid_constant__ AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sQ = smem_u32(smem);
+  const uint32_t sK = sQ + kTcTileBytes;
+  const uint32_t sV = sK + kTcTileBytes;
+  uint8_t* book = smem + 3 * kTcTileBytes;
+  const uint32_t bar_load = smem_u32(book);
+  const uint32_t bar_mma = bar_load + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(book + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(book + 20);
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int head = blockIdx.x;
+  const int b = blockIdx.y;
+  const int g = blockIdx.z;
+  const int H = p.heads * kHeadDim;
+
+  if (tid == 0) {
+    mbar_init(bar_load, 1);
+    mbar_init(bar_mma, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_shared();
+    prefetch_tensormap(&p.tmap_qkv[g]);
+  }
+  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTcTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  grid_dependency_wait();
+  grid_launch_dependents();
+
+  int len = p.lengths[b];
+  len = len < 0 ? 0 : (len > p.seq ? p.seq : len);
+  const int row0 = p.row_start != nullptr ? p.row_start[b] : b * p.seq;
+  const int rows_out = p.packed ? len : p.seq;   // the padded layout also gets its rows >= length, as zeros
+  bf16* ctx = p.ctx[g];
+
+  bool ok = true;
+  bool loads_in_flight = false;
+  if (len > 0) {
+    if (tid == 0) {
+      mbar_expect_tx(bar_load, 3 * kTcTileBytes);
+      tma_load_2d(sQ, &p.tmap_qkv[g], head * kHeadDim, row0, bar_load);
+      tma_load_2d(sK, &p.tmap_qkv[g], H + head * kHeadDim, row0, bar_load);
+      tma_load_2d(sV, &p.tmap_qkv[g], 2 * H + head * kHeadDim, row0, bar_load);
+    }
+    ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag)) != 0;
+    loads_in_flight = !ok;
+  }
+
+  if (ok && len > 0) {
+    // keys >= length take no part: their probabilities are exactly 0, and 0 * V must stay finite
+    if (tid >= len) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(smem + 2 * kTcTileBytes + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+    }
+    fence_async_shared();
+    __syncthreads();
+
+    const int key_tiles = len > 64 ? 2 : 1;   // 64 keys each
+    if (tid == 0) {
+      tc_fence_after();
+      const uint64_t dq = smem_desc_sw128(sQ);
+      const uint64_t dk = smem_desc_sw128(sK);
+      const uint32_t idesc = umma_idesc_bf16(kTcRows, 64 * key_tiles);
+#pragma unroll
+      for (int k = 0; k < kHeadDim / 16; ++k) umma_bf16(tmem_base, dq + 2 * k, dk + 2 * k, idesc, k > 0 ? 1u : 0u);
+      umma_commit(bar_mma);
+    }
+    ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag)) != 0;
+  }
+
+  if (ok && len > 0) {
+    tc_fence_after();
+    const int key_tiles = len > 64 ? 2 : 1;
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    const bool row_valid = tid < len;
+    float row_max = -INFINITY;
+    for (int c = 0; c < 2 * key_tiles; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(t_row + c * 32, v);
+      tmem_ld_wait();
+      if (!row_valid) continue;
+      if ((c + 1) * 32 <= len) {   // all 32 keys of the chunk are valid: no per-key test
+#pragma unroll
+        for (int j = 0; j < 32; ++j) row_max = fmaxf(row_max, __uint_as_float(v[j]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (c * 32 + j < len) row_max = fmaxf(row_max, __uint_as_float(v[j]));
+      }
+    }
+    // exp((s - max) / 8) = 2^((s - max) * log2(e) / 8); the exponent is <= 0, so ex2.approx is in range
+    const float k2 = 0.125f * 1.4426950408889634f;
+    const float shift = row_max * k2;
+    float row_sum = 0.0f;
+    for (int c = 0; c < 2 * key_tiles; ++c) {
+      uint32_t v[32];
+      tmem_ld_32x32(t_row + c * 32, v);
+      tmem_ld_wait();
+      uint8_t* p_tile = smem + (c >> 1) * kTcTileBytes;   // probabilities replace the Q tile, then the K tile
+      const bool chunk_full = (c + 1) * 32 <= len;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (row_valid) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int key = c * 32 + q * 8 + 2 * j;
+            float e0 = ex2_approx(fmaf(__uint_as_float(v[q * 8 + 2 * j]), k2, -shift));
+            float e1 = ex2_approx(fmaf(__uint_as_float(v[q * 8 + 2 * j + 1]), k2, -shift));
+            if (!chunk_full) {
+              e0 = key < len ? e0 : 0.0f;
+              e1 = key + 1 < len ? e1 : 0.0f;
+            }
+            row_sum += e0 + e1;
+            w[j] = pack_bf16(e0, e1);
+          }
+        }
+        *reinterpret_cast<uint4*>(p_tile + staging_off(tid, (c & 1) * 4 + q)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+    const float inv_sum = row_valid ? 1.0f / row_sum : 0.0f;
+    fence_async_shared();
+    tc_fence_before();
+    __syncthreads();
+
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t idesc = umma_idesc_bf16_b_mn(kTcRows, kHeadDim);
+      for (int t = 0; t < key_tiles; ++t) {
+        const uint64_t dp = smem_desc_sw128(sQ + t * kTcTileBytes);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          // sixteen keys = sixteen 128-byte rows of the V tile: two groups of eight rows, 1024 bytes apart
+          const uint64_t dv = smem_desc_sw128(sV + (t * 64 + k * 16) * 128);
+          umma_bf16(tmem_base, dp + 2 * k, dv, idesc, (t | k) != 0 ? 1u : 0u);
+        }
+      }
+      umma_commit(bar_mma);
+    }
+    ok = __syncthreads_and(mbar_wait(bar_mma, 1, abort_flag)) != 0;
+
+    if (ok) {
+      tc_fence_after();
+      // O / sum -> bf16 -> the V tile's place (both products have completed), then out row by row
+      uint8_t* o_tile = smem + 2 * kTcTileBytes;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t v[32];
+        tmem_ld_32x32(t_row + half * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            w[j] = pack_bf16(__uint_as_float(v[q * 8 + 2 * j]) * inv_sum, __uint_as_float(v[q * 8 + 2 * j + 1]) * inv_sum);
+          *reinterpret_cast<uint4*>(o_tile + staging_off(tid, half * 4 + q)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      __syncthreads();
+      const int chunk = tid & 7;
+      for (int r = tid >> 3; r < rows_out; r += kTcThreads / 8) {
+        const uint4 val = *reinterpret_cast<const uint4*>(o_tile + staging_off(r, chunk));
+        *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(row0 + r) * H + head * kHeadDim + chunk * 8) = val;
+      }
+    }
+  } else if (ok && len == 0) {
+    // an empty sequence has rows only in the padded layout: zeros
+    const int chunk = tid & 7;
+    for (int r = tid >> 3; r < rows_out; r += kTcThreads / 8)
+      *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(row0 + r) * H + head * kHeadDim + chunk * 8) = make_uint4(0, 0, 0, 0);
+  }
+
+  if (!ok && tid == 0) {
+    if (loads_in_flight) {
+      // shared memory must not be handed to another CTA while copies may still land in it
+      const unsigned long long t0 = global_timer_ns();
+      while (!mbar_try_wait(bar_load, 0)) {
+        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      }
+    }
+    if (p.status != nullptr) atomicOr(p.status, kFlagWaitTimeout);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, kTcTmemCols);
+}
+
+}  // namespace
+
+cudaError_t launch_attention_tc(const AttnParams& p, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1 || p.seq > kTcRows) return cudaErrorInvalidValue;
+  static int configured_device = -1;   // the attribute is per function and per device
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (configured_device != dev) {
+    e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured_device = dev;
+  }
+  dim3 grid(p.heads, p.batch, p.n_groups);
+  return launch_kernel(attention_tc_kernel, grid, dim3(kTcThreads), kTcSmemBytes, stream, p);
+}
+
+}  // namespace mt

@@ -182,6 +182,7 @@ struct mt_model {
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
   bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
+  bool attention_tc;  // attention on tcgen05 with tensor-memory accumulators when seq <= 128 (else mma.sync)
   int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
 
@@ -420,6 +421,8 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   ck->attn.heads = ck->attn_cls.heads = m->trunk.heads;
   ck->attn.row_start = ck->attn_cls.row_start = row_start;  // lengths are patched per call
   ck->attn.packed = m->pack_tokens ? 1 : 0;
+  ck->attn.tensor_memory = (m->attention_tc && seq <= kAttnTensorMemoryMaxSeq) ? 1 : 0;
+  ck->attn.status = ck->qkv.status;
 
   for (size_t i = 0; i < count; ++i) {
     const OpDesc& op = ops[first + i];
@@ -455,6 +458,9 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
       ck->attn.qkv[a] = qkv;
       ck->attn.ctx[a] = ctx;
       ck->attn.n_groups = a + 1;
+      if (ck->attn.tensor_memory &&
+          (e = make_tmap(&ck->attn.tmap_qkv[a], qkv, M, 3 * H, kAttnTensorMemoryMaxSeq, kHeadDim, false)) != cudaSuccess)
+        return e;
       if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f32_of(m, h1), f, out, f32_of(m, out))) !=
           cudaSuccess)
         return e;
@@ -611,6 +617,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->cls_only = true;
   m->early_heads = false;
   m->gemm_pair = 2;
+  m->attention_tc = true;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -675,6 +682,11 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "gemm_pair") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "gemm_pair must be 0, 1 or 2");
     m->gemm_pair = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "attention_tc") == 0) {
+    m->attention_tc = value != 0;
     m->plans.clear();
     return MT_OK;
   }
@@ -1058,8 +1070,9 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
 }
 
 int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx, int32_t batch, int32_t seq,
-                        int32_t heads, void* stream) {
-  if (d_qkv == nullptr || d_lengths == nullptr || d_ctx == nullptr || batch < 1 || seq < 1 || heads < 1)
+                        int32_t heads, int32_t tensor_memory, uint32_t* d_status, void* stream) {
+  if (d_qkv == nullptr || d_lengths == nullptr || d_ctx == nullptr || batch < 1 || seq < 1 || heads < 1 ||
+      (tensor_memory != 0 && seq > kAttnTensorMemoryMaxSeq))
     return MT_ERR_INVALID_ARG;
   AttnParams p;
   memset(&p, 0, sizeof(p));
@@ -1067,6 +1080,13 @@ int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx
   p.ctx[0] = static_cast<bf16*>(d_ctx);
   p.lengths = d_lengths;
   p.n_groups = 1; p.batch = batch; p.seq = seq; p.heads = heads;
+  p.status = d_status;
+  if (tensor_memory != 0) {
+    p.tensor_memory = 1;
+    if (make_tmap(&p.tmap_qkv[0], d_qkv, static_cast<int64_t>(batch) * seq, 3 * static_cast<int64_t>(heads) * kHeadDim,
+                  kAttnTensorMemoryMaxSeq, kHeadDim, false) != cudaSuccess)
+      return MT_ERR_CUDA;
+  }
   return launch_attention(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 

@@ -96,15 +96,21 @@ cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStr
 // Token layout.  The rows of sequence b start at row_start[b] (device array of batch + 1 ints written
 // by launch_row_starts: b * seq for the padded layout, the running sum of the lengths for the packed
 // layout, in which only valid tokens exist).  A null row_start means the padded layout.
-struct AttnParams {
+struct alignas(64) AttnParams {
+  CUtensorMap tmap_qkv[kMaxGroups];  // qkv_g: dims {3H, rows}, box {64, 128}, 128-byte swizzle (tensor-memory kernel only)
   const bf16* qkv[kMaxGroups];  // [rows, 3*H] = [Q | K | V]
   bf16* ctx[kMaxGroups];        // [rows, H]
   const int32_t* lengths;       // [B]
   const int32_t* row_start;     // [B + 1] or null
   int32_t packed;               // 1: no padded rows exist, nothing is written beyond a sequence's length
   int32_t n_groups, batch, seq, heads;
+  int32_t tensor_memory;        // 1: the tcgen05 kernel (seq <= 128, tmap_qkv filled); 0: the mma.sync kernel
+  uint32_t* status;             // sticky device status word (may be null)
 };
+// Longest sequence the tensor-memory attention kernel handles (one CTA holds all keys of a sequence).
+constexpr int kAttnTensorMemoryMaxSeq = 128;
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_attention_tc(const AttnParams& p, cudaStream_t stream);
 
 // Attention of the first token of every sequence only (the last layer of a task branch: its head
 // reads nothing but that row).  Writes the context compactly, ctx[b, :], and gathers the fp32

@@ -23,6 +23,7 @@ from . import binding as mt
 L2_FLUSH_BYTES = 256 << 20
 USE_GRAPH = False
 CTA_PAIR = False
+TENSOR_MEMORY = True
 
 
 def _time(fn, iters, warmup, flush):
@@ -84,7 +85,7 @@ def bench_attention(batch, seq, heads, len_lo, iters, warmup, flush):
     qkv = torch.randn(batch * seq, 3 * hidden, device="cuda").to(torch.bfloat16)
     lengths = torch.randint(len_lo, seq + 1, (batch,), device="cuda", dtype=torch.int32)
     ctx = torch.empty(batch * seq, hidden, device="cuda", dtype=torch.bfloat16)
-    ms = _time(lambda: mt.mt_kernel_attention(qkv, lengths, ctx, batch, seq, heads), iters, warmup, flush)
+    ms = _time(lambda: mt.mt_kernel_attention(qkv, lengths, ctx, batch, seq, heads, tensor_memory=TENSOR_MEMORY and seq <= 128), iters, warmup, flush)
     bytes_ = 2.0 * 4 * batch * seq * hidden
     n = lengths.double()
     flops = float((4.0 * hidden * n * n).sum())
@@ -121,10 +122,12 @@ def main():
     ap.add_argument("--flush", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
     ap.add_argument("--pair", action="store_true", help="linear: pairs of CTAs on 256-row tiles (cta_group::2)")
+    ap.add_argument("--mma-sync", action="store_true", help="attention: the mma.sync kernel also where seq <= 128")
     a = ap.parse_args()
-    global USE_GRAPH, CTA_PAIR
+    global USE_GRAPH, CTA_PAIR, TENSOR_MEMORY
     USE_GRAPH = a.graph
     CTA_PAIR = a.pair
+    TENSOR_MEMORY = not a.mma_sync
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))

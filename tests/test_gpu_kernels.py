@@ -66,6 +66,8 @@ def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
     ctx = np.zeros((B * S, H))
     for b in range(B):
         n = int(lengths[b])
+        if n == 0:
+            continue
         blk = qkv[b * S:b * S + n]
         for a in range(heads):
             q, k, v = (blk[:, i * H + a * 64:i * H + (a + 1) * 64] for i in range(3))
@@ -73,14 +75,19 @@ def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
     return ctx
 
 
-@pytest.mark.parametrize("B,S,heads,lengths", [
-    (2, 32, 12, [32, 32]),
-    (4, 128, 12, [128, 37, 1, 64]),
-    (3, 100, 2, [100, 65, 9]),       # seq not a multiple of the tile
-    (2, 512, 16, [512, 300]),
-    (1, 1, 1, [1]),
+@pytest.mark.parametrize("B,S,heads,lengths,tensor_memory", [
+    (2, 32, 12, [32, 32], False),
+    (4, 128, 12, [128, 37, 1, 64], False),
+    (3, 100, 2, [100, 65, 9], False),       # seq not a multiple of the tile
+    (2, 512, 16, [512, 300], False),
+    (1, 1, 1, [1], False),
+    (2, 32, 12, [32, 32], True),
+    (6, 128, 12, [128, 37, 1, 64, 65, 127], True),
+    (3, 100, 2, [100, 65, 9], True),        # the 128-row tile reaches into the next sequence and past the buffer
+    (1, 1, 1, [1], True),
+    (5, 128, 16, [0, 128, 0, 16, 113], True),   # empty sequences
 ])
-def test_attention_matches_oracle(B, S, heads, lengths):
+def test_attention_matches_oracle(B, S, heads, lengths, tensor_memory):
     H = heads * 64
     qb, qkv = rand_bf16(21, f"qkv{B}.{S}.{heads}", (B * S, 3 * H), 1.5)
     # poison the padded rows of the input: they must not leak into valid rows
@@ -89,8 +96,10 @@ def test_attention_matches_oracle(B, S, heads, lengths):
     for b, n in enumerate(lengths):
         qkv_dev[b * S + n:(b + 1) * S] = float("nan")
     ctx = torch.full((B * S, H), float("nan"), dtype=torch.bfloat16, device="cuda")
-    mt.mt_kernel_attention(qkv_dev, lens, ctx, B, S, heads)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mt.mt_kernel_attention(qkv_dev, lens, ctx, B, S, heads, tensor_memory=tensor_memory, status=status)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0
     got = dev_bf16_to_f64(ctx)
     want = oracle_attention_from_qkv(qkv, lengths, B, S, heads)
     assert np.all(np.isfinite(got))
