@@ -233,6 +233,8 @@ def main():
     host_in = [(torch.from_numpy(b.token_ids).pin_memory(), torch.from_numpy(b.segment_ids).pin_memory(),
                 torch.from_numpy(b.lengths).pin_memory()) for b in batches]
     logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32, device=device)
+    # what a server knows about its traffic: the mean number of valid tokens per batch (tile shapes only)
+    model.set_option("expected_tokens", int(round(float(np.mean([int(b.lengths.sum()) for b in batches])))))
     host_logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32).pin_memory()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
     stream = torch.cuda.current_stream()

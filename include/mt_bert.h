@@ -182,7 +182,11 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * of batch*seq padded rows; logits agree to rounding either way.  key "gemm_pair" (0 never, 1 always, 2 = by launch size, the default; any
  * time): run GEMM launches as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2, each CTA stages half
  * of a weight tile) instead of single CTAs on 128-row tiles; faster on large launches (+11 % at 8192^3),
- * slower on small ones; the results are bit-identical.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * slower on small ones; the results are bit-identical.  key "attention_tc" (0/1, default 1, any time): attention
+ * for seq <= 128 runs on tcgen05 with its accumulators in tensor memory (1) or on mma.sync (0, also
+ * used for every longer seq).  key "expected_tokens" (>= 0, default 0 = every row, any time): the caller's
+ * estimate of the valid tokens per batch; with the packed layout the GEMM tile widths are chosen for
+ * that many rows instead of batch*seq; it never changes a result.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);

@@ -447,24 +447,44 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
 
 template <bool PAIR>
 cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
-  switch (gemm_block_n(p.N, epilogue)) {
+  switch (p.block_n) {
     case 256: return launch_bn<256, PAIR>(p, epilogue, sm_count, stream);
     case 192: return launch_bn<192, PAIR>(p, epilogue, sm_count, stream);
-    default: return launch_bn<128, PAIR>(p, epilogue, sm_count, stream);
+    case 128: return launch_bn<128, PAIR>(p, epilogue, sm_count, stream);
+    default: return cudaErrorInvalidValue;
   }
 }
 
 }  // namespace
 
-int gemm_block_n(int N, int epilogue) {
-  if (epilogue != kEpiBiasResidual && N % 256 == 0 && N >= 2048) return 256;
-  return N % 192 == 0 ? 192 : 128;  // 768 = 4 x 192: 128 tiles per 4096 rows, one wave of 148 SMs
+int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int sm_count) {
+  const int candidates[3] = {256, 192, 128};
+  const int64_t tile_m = pair ? 2 * kGemmBlockM : kGemmBlockM;
+  const int64_t workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
+  const int64_t m_tiles = (rows + tile_m - 1) / tile_m;
+  int best = 128;
+  int64_t best_cost = -1;
+  for (int bn : candidates) {
+    if (N % bn != 0) continue;
+    if (bn == 256 && epilogue == kEpiBiasResidual) continue;   // not instantiated: two fp32 staging buffers do not fit
+    const int64_t tiles = m_tiles * (N / bn) * groups;
+    const int64_t rounds = (tiles + workers - 1) / workers;
+    // per 64 of K a CTA stages 128 rows of X and bn (a pair's CTA: bn / 2) rows of W, and its tensor
+    // core needs about bn of the same units
+    const int64_t staged = 128 + (pair ? bn / 2 : bn);
+    const int64_t cost = rounds * (staged > bn ? staged : bn);
+    if (best_cost < 0 || cost < best_cost) {   // candidates run from wide to narrow: ties keep the wider tile
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
 }
 int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
-int gemm_w_box_rows(int N, int epilogue, bool pair) { return gemm_block_n(N, epilogue) / (pair ? 2 : 1); }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
-  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.N % 128 != 0 || p.M < 1)
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.block_n < 1 || p.N % p.block_n != 0 ||
+      p.M < 1)
     return cudaErrorInvalidValue;
   return p.pair ? launch_any<true>(p, epilogue, sm_count, stream) : launch_any<false>(p, epilogue, sm_count, stream);
 }

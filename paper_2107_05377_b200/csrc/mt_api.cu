@@ -157,7 +157,7 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
   const bool res = epilogue == kEpiBiasResidual;
   cudaError_t e;
   if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
-  if ((e = make_tmap(&g->tmap_w[i], w, N, K, gemm_w_box_rows(N, epilogue, g->pair != 0), kGemmBlockK, false)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_w[i], w, N, K, g->block_n / (g->pair != 0 ? 2 : 1), kGemmBlockK, false)) != cudaSuccess) return e;
   if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), res)) != cudaSuccess) return e;
   if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
   g->group[i].bias = bias;
@@ -182,6 +182,7 @@ struct mt_model {
   bool debug_capture;
   bool pack_tokens;  // packed token layout: only valid tokens are stored and computed
   bool cls_only;     // the last layer of a task branch is evaluated for the first token of a sequence only
+  int64_t expected_tokens;  // caller's estimate of the valid tokens per batch (0 = every row); tunes tile shapes only
   bool attention_tc;  // attention on tcgen05 with tensor-memory accumulators when seq <= 128 (else mma.sync)
   int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
@@ -350,21 +351,30 @@ int32_t use_pair(const mt_model* m, int64_t rows, int64_t groups) {
   if (m->gemm_pair != 2) return m->gemm_pair;
   return rows * groups >= 12288 ? 1 : 0;
 }
+// Tile width of a grouped GEMM launch (see gemm_block_n).  `rows` are the rows the launch is sized for;
+// with the packed token layout only the valid tokens are in use, and the caller's estimate of their
+// number (option "expected_tokens"), when given, replaces it.
+void choose_block_n(const mt_model* m, GemmParams* g, int epilogue, bool all_rows_valid, int32_t groups) {
+  int64_t rows = g->M;
+  if (!all_rows_valid && m->pack_tokens && m->expected_tokens > 0 && m->expected_tokens < rows) rows = m->expected_tokens;
+  g->block_n = gemm_block_n(g->N, epilogue, rows, groups < 1 ? 1 : groups, g->pair != 0, m->sm_count);
+}
 
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
   const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
   const int32_t* rows_valid =
       all_rows_valid ? nullptr : reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
-  auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K) {
+  auto init_gemm = [&](GemmParams* g, int32_t N, int32_t K, int epilogue) {
     memset(g, 0, sizeof(*g));
     g->M = rows; g->N = N; g->K = K;
     g->pair = use_pair(m, rows, groups);
+    choose_block_n(m, g, epilogue, all_rows_valid, groups);
     g->m_valid = rows_valid;
     g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   };
-  init_gemm(&t->attn_out, H, H);
-  init_gemm(&t->ffn_up, F, H);
-  init_gemm(&t->ffn_down, H, F);
+  init_gemm(&t->attn_out, H, H, kEpiBiasResidual);
+  init_gemm(&t->ffn_up, F, H, kEpiBiasGelu);
+  init_gemm(&t->ffn_down, H, F, kEpiBiasResidual);
   memset(&t->ln1, 0, sizeof(t->ln1));
   memset(&t->ln2, 0, sizeof(t->ln2));
   t->ln1.rows_valid = t->ln2.rows_valid = rows_valid;
@@ -408,6 +418,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   ck->qkv.n_groups = static_cast<int32_t>(count);
   ck->qkv.M = M; ck->qkv.N = 3 * H; ck->qkv.K = H;
   ck->qkv.pair = use_pair(m, M, static_cast<int64_t>(count));
+  choose_block_n(m, &ck->qkv, kEpiBias, false, static_cast<int32_t>(count));
   ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   int32_t n_full = 0;
@@ -618,6 +629,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->early_heads = false;
   m->gemm_pair = 2;
   m->attention_tc = true;
+  m->expected_tokens = 0;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -683,6 +695,12 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "gemm_pair must be 0, 1 or 2");
     m->gemm_pair = static_cast<int32_t>(value);
     m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "expected_tokens") == 0) {
+    if (value < 0) return fail(m, MT_ERR_INVALID_ARG, "expected_tokens must be >= 0");
+    if (value != m->expected_tokens) m->plans.clear();
+    m->expected_tokens = value;
     return MT_OK;
   }
   if (strcmp(key, "attention_tc") == 0) {
@@ -1063,6 +1081,7 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   memset(&p, 0, sizeof(p));
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
   p.pair = cta_pair != 0 ? 1 : 0;
+  p.block_n = gemm_block_n(N, epilogue, M, 1, p.pair != 0, sms);
   if (set_gemm_group(&p, 0, epilogue, d_x, d_w, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
                      d_y) != cudaSuccess)
     return MT_ERR_CUDA;

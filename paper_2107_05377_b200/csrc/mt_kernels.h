@@ -81,16 +81,18 @@ struct alignas(64) GemmParams {
   int32_t M, N, K;
   const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
   int32_t pair;            // 1: run as pairs of CTAs on 256-row tiles (the W maps then fetch half a tile's rows)
+  int32_t block_n;         // tile width along N: 128, 192 or 256 (gemm_block_n); N % block_n == 0
   uint32_t* status;        // sticky device status word (may be null)
 };
 
-// Tile width along N chosen for a given N and epilogue (fixed, so results never depend on grouping),
-// and the width in elements of the 128-byte output box (64 bf16 or 32 fp32 columns; 32 rows).
-int gemm_block_n(int N, int epilogue);
+// Tile width along N for a launch of `groups` problems with about `rows` rows in use each, from a cost
+// model of the kernel: the tiles are dealt out in rounds over the SMs (or SM pairs), and a round costs
+// about (128 + width) per 64 of K because a CTA is bound by the bytes it stages.  Fewer, wider tiles
+// re-read X less; narrower ones waste less of the last round.  Every output element is accumulated
+// over K in the same order whatever the width, so the choice never changes a result.
+int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int sm_count);
+// Width in elements of the 128-byte output box (64 bf16 or 32 fp32 columns; 32 rows).
 int gemm_out_box_cols(int epilogue);
-// Rows of W one TMA box fetches: the tile width, or half of it when the GEMM runs as CTA pairs
-// (each CTA of a pair stages half of the W tile).
-int gemm_w_box_rows(int N, int epilogue, bool pair);
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream);
 
 // Token layout.  The rows of sequence b start at row_start[b] (device array of batch + 1 ints written

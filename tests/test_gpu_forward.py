@@ -17,9 +17,13 @@ LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
 def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None,
-              gemm_pair=None):
+              gemm_pair=None, attention_tc=None, expected_tokens=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
+    if attention_tc is not None:
+        model.set_option("attention_tc", attention_tc)
+    if expected_tokens is not None:
+        model.set_option("expected_tokens", expected_tokens)
     if gemm_pair is not None:
         model.set_option("gemm_pair", gemm_pair)
     if pack_tokens is not None:
@@ -123,6 +127,34 @@ def test_cta_pair_gemms_match_oracle_and_single_cta_bits():
     assert torch.equal(p8, s8)
     _, auto8 = run_model(big, blob8, b8)          # default: pairs for the large grouped launches only
     assert torch.equal(auto8, s8)
+
+
+def test_tile_width_follows_expected_tokens_without_changing_bits():
+    """The GEMM tile width is chosen per launch from the rows expected to be in use (option
+    "expected_tokens"): every output element is still one fixed-order sum over K, so logits are
+    bit-identical whatever the estimate, and equal to the oracle's within tolerance."""
+    big = synth.config_glue8()
+    w8, blob8, wf8 = cached_weights(big, 0)
+    b8 = synth.batch_glue8(big)
+    _, base = run_model(big, blob8, b8)
+    tokens = int(b8.lengths.sum())
+    for hint in (tokens, 128, 1000, 4096):
+        for pair in (0, 2):
+            model, got = run_model(big, blob8, b8, expected_tokens=hint, gemm_pair=pair)
+            assert torch.equal(got, base), (hint, pair)
+    check_against_oracle(big, wf8, b8, model, got, rows=[0, 17], check_hidden=False)
+
+
+def test_attention_kernels_agree_in_the_forward():
+    """The tensor-memory attention (default for seq <= 128) and the mma.sync attention both meet the
+    oracle's tolerance in a whole forward; their logits differ only by rounding."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 5, 100, 1, 100, seed=9)
+    for tc in (1, 0):
+        model, logits = run_model(cfg, blob, batch, debug=True, attention_tc=tc)
+        check_against_oracle(cfg, wf, batch, model, logits, rows=range(5))
 
 
 def test_padded_layout_matches_oracle_and_packed_layout():
