@@ -188,6 +188,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the oracle (N=1 only)")
+    ap.add_argument("--set", action="append", default=[], metavar="KEY=VALUE",
+                    help="library option (mt_set_option) to set before the run, e.g. --set fused_tail=0; repeatable")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -224,8 +226,6 @@ def main():
     blob = torch.from_numpy(synth.pack_weights(cfg, weights)).pin_memory()
     model.load_weights(blob)
     mask = model.full_mask()
-    plan = model.plan_summary(mask)
-    launches_per_step = model.plan_launches(mask)
 
     batches = [synth.batch_glue8(cfg, BATCH, SEQ, LEN_LO, LEN_HI, seed=1 + i) for i in range(N_INPUT_BATCHES)]
     dev_in = [(torch.from_numpy(b.token_ids).to(device), torch.from_numpy(b.segment_ids).to(device),
@@ -235,6 +235,11 @@ def main():
     logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32, device=device)
     # what a server knows about its traffic: the mean number of valid tokens per batch (tile shapes only)
     model.set_option("expected_tokens", int(round(float(np.mean([int(b.lengths.sum()) for b in batches])))))
+    for kv in args.set:
+        key, _, value = kv.partition("=")
+        model.set_option(key, int(value))
+    plan = model.plan_summary(mask)
+    launches_per_step = model.plan_launches(mask)
     host_logits = torch.zeros(BATCH, cfg.total_classes, dtype=torch.float32).pin_memory()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
     stream = torch.cuda.current_stream()

@@ -186,7 +186,17 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * for seq <= 128 runs on tcgen05 with its accumulators in tensor memory (1) or on mma.sync (0, also
  * used for every longer seq).  key "expected_tokens" (>= 0, default 0 = every row, any time): the caller's
  * estimate of the valid tokens per batch; with the packed layout the GEMM tile widths are chosen for
- * that many rows instead of batch*seq; it never changes a result.  key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
+ * that many rows instead of batch*seq; it never changes a result.  key "fused_tail" (0 never, the default; 1 always; 2 = where a wave
+ * has at least "fused_min_groups" (default 3) layers; any time): the part of
+ * a layer after attention (output projection + residual, LayerNorm, FFN up + GELU, FFN down + residual,
+ * LayerNorm) runs, for all layers of a wave, as ONE persistent launch whose tiles wait on per-row-block
+ * counters in the workspace, instead of five launches; bit-identical results.  Measured slower than the
+ * five launches at batch 32 x seq 128 (each hand-over between tiles through global memory costs 2-3 us).  Its CTAs wait for one
+ * another, so all of them must be resident: forwards of several models or streams that overlap on one
+ * device can make those waits run out (status flag MT_FLAG_WAIT_TIMEOUT) - serialise them, or set 0.
+ * keys "tail_bn0", "tail_bn1", "tail_bn2" (0 = automatic, 128, 192; any time): tile widths of the three
+ * GEMMs of that launch; they never change a result.
+ * key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */
 int mt_set_option(mt_model* m, const char* key, int64_t value);
@@ -205,7 +215,8 @@ int mt_set_option(mt_model* m, const char* key, int64_t value);
 #define MT_CLASS_FFN_DOWN  6  /* GEMM: FFN down projection + residual               */
 #define MT_CLASS_LN2       7  /* LayerNorm after the FFN                            */
 #define MT_CLASS_HEAD      8  /* pooler + head                                      */
-#define MT_NUM_CLASSES     9
+#define MT_CLASS_TAIL      9  /* fused layer tail: classes 3-7 as one launch            */
+#define MT_NUM_CLASSES     10
 int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class);
 
 /* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out (padded

@@ -18,7 +18,7 @@ MT_OK = 0
 ERRORS = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "NOT_BOUND", -4: "NOT_LOADED", -5: "BLOB_MISMATCH",
           -6: "CUDA", -7: "UNSUPPORTED", -8: "DEVICE_FLAG"}
 FLAG_BAD_TOKEN, FLAG_BAD_SEGMENT, FLAG_BAD_LENGTH, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head")
+KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head", "tail")
 
 
 class TrunkConfig(C.Structure):

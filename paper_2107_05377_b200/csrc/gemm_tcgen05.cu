@@ -46,21 +46,6 @@ __host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair) {
          kNumEpilogueWarps * gemm_staging_bufs(bn, pair) * kStagingBytes + 512 + 1024;
 }
 
-// Exact-form GELU x * Phi(x), Phi(x) = 1/2 erfc(-x / sqrt 2), with erfc evaluated branch-free by the
-// rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7, far below the bf16
-// rounding of the result): erfc(z) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-z^2), t = 1 / (1 + p z),
-// z >= 0.  The negative side uses Phi(x) = 1 - Phi(-x) without cancellation.
-__device__ __forceinline__ float gelu_erf(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float half_erfc = 0.5f * poly * t * __expf(-z * z);   // Phi(-|x|)
-  return x * (x >= 0.0f ? 1.0f - half_erfc : half_erfc);
-}
-
 // ---- the kernel -------------------------------------------------------------------------------
 
 // PAIR: the kernel runs as clusters of two CTAs that share 256 x BN tiles (tcgen05 cta_group::2).

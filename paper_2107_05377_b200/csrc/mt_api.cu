@@ -77,6 +77,9 @@ struct LayerTail {
   GemmParams attn_out, ffn_up, ffn_down;
   LayerNormParams ln1, ln2;
   int32_t count = 0;
+  // the same five steps as one persistent launch (option "fused_tail"), with its own tile widths
+  bool fused = false;
+  ChainParams chain;
 };
 struct DumpCopy {
   const bf16* src;
@@ -107,6 +110,7 @@ struct PlanStep {
 struct Plan {
   std::vector<PlanStep> steps;
   int32_t launches = 0;
+  size_t sync_bytes = 0;  // counters of the fused layer-tail launches, zeroed at the start of a forward
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -186,6 +190,10 @@ struct mt_model {
   bool attention_tc;  // attention on tcgen05 with tensor-memory accumulators when seq <= 128 (else mma.sync)
   int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
+  int32_t fused_tail;  // steps 3-7 of a layer (output projection .. second LayerNorm) as one persistent launch per
+                       // wave: 0 never, 1 always, 2 where the wave has at least fused_min_groups layers
+  int32_t fused_min_groups;
+  int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
   // device memory (caller-owned)
   uint8_t* d_weights;
@@ -195,7 +203,8 @@ struct mt_model {
 
   // workspace layout (byte offsets)
   size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
-      ws_slot0, ws_cls0, ws_dump0;
+      ws_slot0, ws_cls0, ws_dump0, ws_sync;
+  size_t sync_bytes;   // room for the counters of all fused layer-tail launches of one forward
   size_t cls_bytes, cls_h_bytes, cls_h32_bytes;  // per-task first-token scratch and its [B,H] bf16 / fp32 pieces
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
@@ -256,6 +265,19 @@ void layout_workspace(mt_model* m) {
   m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
   // tanh pooler outputs of the tasks of one head launch: fp32 [kMaxGroups][max_batch][H]
   m->ws_pooled = take(static_cast<size_t>(kMaxGroups) * m->max_batch * H * sizeof(float));
+  {
+    // counters of the fused layer-tail launches: every launch of a forward has its own, so one memset at
+    // the start of the forward clears them all.  Launches per forward: per wave the chunks of at most
+    // n_slots layers, plus the first-token tails (at most one more step per wave and chunk of tasks).
+    int32_t max_branch = 0;
+    for (const TaskEntry& t : m->tasks) max_branch = std::max(max_branch, t.cfg.branch_layers);
+    const size_t T = m->tasks.size();
+    const size_t per_wave = (T + 1 + std::max<int32_t>(m->max_groups, 1) - 1) / std::max<int32_t>(m->max_groups, 1) +
+                            (T + kMaxGroups - 1) / kMaxGroups;
+    const size_t launches = static_cast<size_t>(m->trunk.trunk_layers + max_branch + 1) * per_wave;
+    m->sync_bytes = launches * pad256(chain_sync_bytes(kMaxGroups, static_cast<int64_t>(M)));
+    m->ws_sync = take(m->sync_bytes);
+  }
   m->ws_trunk[0] = take(m->state_bytes);
   m->ws_trunk[1] = take(m->state_bytes);
   m->ws_task0 = off;
@@ -360,6 +382,16 @@ void choose_block_n(const mt_model* m, GemmParams* g, int epilogue, bool all_row
   g->block_n = gemm_block_n(g->N, epilogue, rows, groups < 1 ? 1 : groups, g->pair != 0, m->sm_count);
 }
 
+// Whether the part of `groups` layers after attention runs as one persistent launch (see ChainParams).  Its
+// tiles hand over to one another through global memory, two to three microseconds per hand-over and four
+// hand-overs per layer; measured on the 32 x 128 batch that costs more than the four kernel boundaries it
+// removes (which programmatic dependent launch already hides in part), so it is off unless asked for.
+bool use_fused_tail(const mt_model* m, int32_t groups) {
+  if (groups < 1 || !chain_supported(m->trunk.hidden, m->trunk.ffn)) return false;
+  if (m->fused_tail != 2) return m->fused_tail != 0;
+  return groups >= m->fused_min_groups;
+}
+
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
   const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
   const int32_t* rows_valid =
@@ -382,6 +414,24 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.hidden = t->ln2.hidden = H;
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
+  t->fused = use_fused_tail(m, groups);
+  if (t->fused) {
+    memset(&t->chain, 0, sizeof(t->chain));
+    const GemmParams* like[3] = {&t->attn_out, &t->ffn_up, &t->ffn_down};
+    int64_t rows_used = rows;
+    if (!all_rows_valid && m->pack_tokens && m->expected_tokens > 0 && m->expected_tokens < rows) rows_used = m->expected_tokens;
+    for (int ph = 0; ph < 3; ++ph) {
+      GemmParams* g = &t->chain.gemm[ph];
+      g->M = like[ph]->M; g->N = like[ph]->N; g->K = like[ph]->K;
+      g->pair = 0;
+      g->block_n = chain_block_n(ph, g->N, rows_used, groups, m->sm_count);
+      if (m->tail_bn[ph] != 0 && g->N % m->tail_bn[ph] == 0) g->block_n = m->tail_bn[ph];
+      g->m_valid = rows_valid;
+      g->status = like[ph]->status;
+    }
+    t->chain.sync = nullptr;   // assigned by build_plan
+    t->chain.sync_blocks = (rows + kGemmBlockM - 1) / kGemmBlockM;
+  }
 }
 
 // Steps 3-7 of a layer for one group of a tail: u = ctx Wo^T + bo + residual; h1 = LN(u);
@@ -405,6 +455,18 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
   t->ln2.y[i] = out; t->ln2.y32[i] = out32;
   t->count = i + 1;
   t->attn_out.n_groups = t->ffn_up.n_groups = t->ffn_down.n_groups = t->ln1.n_groups = t->ln2.n_groups = t->count;
+  if (t->fused) {
+    ChainParams* c = &t->chain;
+    if ((e = set_gemm_group(&c->gemm[0], i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) != cudaSuccess)
+      return e;
+    if ((e = set_gemm_group(&c->gemm[1], i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) != cudaSuccess)
+      return e;
+    if ((e = set_gemm_group(&c->gemm[2], i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) != cudaSuccess)
+      return e;
+    c->gemm[0].n_groups = c->gemm[1].n_groups = c->gemm[2].n_groups = t->count;
+    c->ln[0] = t->ln1;
+    c->ln[1] = t->ln2;
+  }
   return cudaSuccess;
 }
 
@@ -517,7 +579,8 @@ cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks,
 int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count) {
   size_t n_cls = 0;
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
-  return 1 + (n_cls < count ? 6 : 0) + (n_cls > 0 ? 1 : 0);
+  const bool fused = use_fused_tail(m, static_cast<int32_t>(count - n_cls));
+  return 1 + (n_cls < count ? (fused ? 2 : 6) : 0) + (n_cls > 0 ? 1 : 0);
 }
 // Active tasks whose last branch layer is finished on first tokens right after wave w (1-based):
 // those whose last layer is in wave w with option early_heads, otherwise all of them after the last wave.
@@ -535,6 +598,16 @@ std::vector<int32_t> cls_tasks_after_wave(const mt_model* m, const Schedule& s, 
 cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
   plan->steps.clear();
   plan->launches = 2;  // row starts, embedding
+  plan->sync_bytes = 0;
+  // gives a fused layer tail its own counters
+  auto assign_sync = [&](LayerTail* t) -> cudaError_t {
+    if (!t->fused || t->count == 0) return cudaSuccess;
+    const size_t bytes = pad256(chain_sync_bytes(t->count, t->chain.gemm[0].M));
+    if (plan->sync_bytes + bytes > m->sync_bytes) return cudaErrorMemoryAllocation;
+    t->chain.sync = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_sync + plan->sync_bytes);
+    plan->sync_bytes += bytes;
+    return cudaSuccess;
+  };
   auto add_heads = [&](const std::vector<int32_t>& tasks) {
     for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
       const size_t count = std::min<size_t>(kMaxGroups, tasks.size() - first);
@@ -570,6 +643,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       st.kind = 0;
       cudaError_t e = build_chunk(m, ops, first, count, batch, seq, &st.chunk);
       if (e != cudaSuccess) return e;
+      if ((e = assign_sync(&st.chunk.full)) != cudaSuccess) return e;
       plan->steps.push_back(std::move(st));
       plan->launches += chunk_launches(m, ops, first, count);
     }
@@ -581,8 +655,9 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         st.kind = 2;
         cudaError_t e = build_cls_tail(m, tasks, first, std::min<size_t>(kMaxGroups, tasks.size() - first), batch, &st);
         if (e != cudaSuccess) return e;
+        if ((e = assign_sync(&st.tail)) != cudaSuccess) return e;
+        plan->launches += st.tail.fused ? 1 : 5;
         plan->steps.push_back(std::move(st));
-        plan->launches += 5;
       }
     }
     add_heads(s.heads[w]);
@@ -630,6 +705,9 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->gemm_pair = 2;
   m->attention_tc = true;
   m->expected_tokens = 0;
+  m->fused_tail = 0;
+  m->fused_min_groups = 3;
+  m->tail_bn[0] = m->tail_bn[1] = m->tail_bn[2] = 0;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -701,6 +779,24 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     if (value < 0) return fail(m, MT_ERR_INVALID_ARG, "expected_tokens must be >= 0");
     if (value != m->expected_tokens) m->plans.clear();
     m->expected_tokens = value;
+    return MT_OK;
+  }
+  if (strcmp(key, "fused_tail") == 0) {
+    if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_tail must be 0, 1 or 2");
+    m->fused_tail = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "fused_min_groups") == 0) {
+    if (value < 1) return fail(m, MT_ERR_INVALID_ARG, "fused_min_groups must be >= 1");
+    m->fused_min_groups = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strncmp(key, "tail_bn", 7) == 0 && key[7] >= '0' && key[7] <= '2' && key[8] == 0) {
+    if (value != 0 && value != 128 && value != 192) return fail(m, MT_ERR_INVALID_ARG, "tail_bn must be 0, 128 or 192");
+    m->tail_bn[key[7] - '0'] = static_cast<int32_t>(value);
+    m->plans.clear();
     return MT_OK;
   }
   if (strcmp(key, "attention_tc") == 0) {
@@ -847,7 +943,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
       const std::vector<OpDesc>& ops = s.waves[w - 1];
       for (size_t first = 0; first < ops.size(); first += m->n_slots)
         n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
-      n += 5 * static_cast<int32_t>((cls_tasks_after_wave(m, s, w).size() + kMaxGroups - 1) / kMaxGroups);
+      const size_t n_cls_tasks = cls_tasks_after_wave(m, s, w).size();
+      for (size_t first = 0; first < n_cls_tasks; first += kMaxGroups)
+        n += use_fused_tail(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first))) ? 1 : 5;
     }
     n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
   }
@@ -915,6 +1013,23 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     }                                                                                        \
   } while (0)
 
+  // Steps 3-7 of the layers of a wave: one persistent launch, or the five separate ones.
+#define MT_TAIL(tail)                                                                                                  \
+  do {                                                                                                                 \
+    LayerTail* t_ = (tail);                                                                                            \
+    if (t_->fused) {                                                                                                   \
+      MT_TIMED(MT_CLASS_TAIL, launch_chain(t_->chain, m->sm_count, stream), "fused layer-tail kernel");                \
+    } else {                                                                                                           \
+      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t_->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM"); \
+      MT_TIMED(MT_CLASS_LN1, launch_layernorm(t_->ln1, stream), "LayerNorm 1");                                        \
+      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");            \
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t_->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");  \
+      MT_TIMED(MT_CLASS_LN2, launch_layernorm(t_->ln2, stream), "LayerNorm 2");                                        \
+    }                                                                                                                  \
+  } while (0)
+
+  if (plan.sync_bytes > 0)
+    MT_LAUNCH(cudaMemsetAsync(m->d_workspace + m->ws_sync, 0, plan.sync_bytes, stream), "clearing the tile counters");
   int32_t* row_start = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_row_start);
   MT_LAUNCH(launch_row_starts(d_lengths, batch, seq, m->pack_tokens ? 1 : 0, row_start,
                               reinterpret_cast<int32_t*>(m->d_workspace + m->ws_rows_valid), stream),
@@ -943,26 +1058,14 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
       if (ck.full.count > 0) MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
       if (ck.n_cls > 0)
         MT_TIMED(MT_CLASS_ATTENTION, launch_cls_attention(ck.attn_cls, stream), "first-token attention kernel");
-      if (ck.full.count > 0) {
-        LayerTail* t = &ck.full;
-        MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
-        MT_TIMED(MT_CLASS_LN1, launch_layernorm(t->ln1, stream), "LayerNorm 1");
-        MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
-        MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
-        MT_TIMED(MT_CLASS_LN2, launch_layernorm(t->ln2, stream), "LayerNorm 2");
-      }
+      if (ck.full.count > 0) MT_TAIL(&ck.full);
       for (const DumpCopy& d : ck.dumps)
         MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.slot, d.src,
                                   d.compact ? static_cast<size_t>(batch) * m->trunk.hidden * sizeof(bf16) : act_used,
                                   cudaMemcpyDeviceToDevice, stream),
                   "debug capture");
     } else if (st.kind == 2) {
-      LayerTail* t = &st.tail;
-      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM");
-      MT_TIMED(MT_CLASS_LN1, launch_layernorm(t->ln1, stream), "LayerNorm 1");
-      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");
-      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");
-      MT_TIMED(MT_CLASS_LN2, launch_layernorm(t->ln2, stream), "LayerNorm 2");
+      MT_TAIL(&st.tail);
       for (const DumpCopy& d : st.dumps)
         MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0 + m->act_bytes * d.slot, d.src,
                                   static_cast<size_t>(batch) * m->trunk.hidden * sizeof(bf16), cudaMemcpyDeviceToDevice,
@@ -977,6 +1080,7 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
             MT_LAUNCH(cudaEventRecord(reinterpret_cast<cudaEvent_t>(task_events[t]), stream), "recording a task event");
     }
   }
+#undef MT_TAIL
 #undef MT_TIMED
 #undef MT_LAUNCH
   m->last_batch = batch;
