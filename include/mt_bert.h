@@ -196,6 +196,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * device can make those waits run out (status flag MT_FLAG_WAIT_TIMEOUT) - serialise them, or set 0.
  * keys "tail_bn0", "tail_bn1", "tail_bn2" (0 = automatic, 128, 192; any time): tile widths of the three
  * GEMMs of that launch; they never change a result.
+ * key "pool_gemm" (0/1, default 1, any time): the pooler of tasks whose last branch layer was evaluated on
+ * first tokens only runs as one grouped GEMM with a tanh epilogue on the tensor cores (1) or in the
+ * row-wise pooler kernel (0, also used for every other task); logits agree to rounding.
  * key "pdl" (0/1, default 1, applies to the whole process): launch every kernel
  * with programmatic stream serialization, so that a kernel's set-up overlaps the previous kernel's
  * tail; results are identical either way. */

@@ -278,10 +278,10 @@ __global__ void __launch_bounds__(kAttnThreads, 4) attention_kernel(const __grid
   }
 }
 
-// First-token attention: one warp = one (sequence, head).  Lanes split the keys for the scores
-// (each lane a whole 128-byte K row per key), then split the 64 output dimensions for the weighted
-// sum of V rows, the probability of each key being broadcast from the lane that owns it.  fp32
-// throughout; only the output is rounded to bf16.
+// First-token attention: one warp = one (sequence, head).  Lanes split the keys, for the scores
+// (each lane a whole 128-byte K row per key) and for the weighted sum of V rows alike (each lane the
+// whole V rows of its keys, then a butterfly sum over the lanes).  fp32 throughout; only the output
+// is rounded to bf16.
 constexpr int kClsWarps = 4;
 constexpr int kClsMaxKeysPerLane = 16;  // sequences of up to 512 keys
 
@@ -353,19 +353,42 @@ __global__ void __launch_bounds__(kClsWarps * 32) cls_attention_kernel(const Cls
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
 
-  float o0 = 0.f, o1 = 0.f;
-  const bf16* vbase = base + 2 * H + 2 * lane;
+  // P . V with the keys spread over the lanes exactly as for the scores: every lane accumulates
+  // its own keys' rows of V (all of its loads are independent, so they are in flight together), then
+  // the 32 partial rows of 64 columns are summed by a butterfly that halves the columns a lane keeps
+  // at every step; lane l ends with columns 2l and 2l + 1.  The order of the additions is fixed.
+  float o[kHeadDim];
+#pragma unroll
+  for (int c = 0; c < kHeadDim; ++c) o[c] = 0.f;
 #pragma unroll
   for (int i = 0; i < kClsMaxKeysPerLane; ++i) {
-    if (i * 32 >= len) break;   // warp-uniform
-    const int n = min(32, len - i * 32);
-    for (int jj = 0; jj < n; ++jj) {
-      const float pj = __shfl_sync(0xffffffffu, sc[i], jj);
-      const uint32_t v = *reinterpret_cast<const uint32_t*>(vbase + static_cast<size_t>(i * 32 + jj) * ld);
-      o0 = fmaf(pj, __uint_as_float(v << 16), o0);
-      o1 = fmaf(pj, __uint_as_float(v & 0xFFFF0000u), o1);
+    const int j = i * 32 + lane;
+    if (j < len) {
+      const uint4* vrow = reinterpret_cast<const uint4*>(base + static_cast<size_t>(j) * ld + 2 * H);
+      const float pj = sc[i];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 u = vrow[c];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          o[c * 8 + 2 * t] = fmaf(pj, __uint_as_float(w[t] << 16), o[c * 8 + 2 * t]);
+          o[c * 8 + 2 * t + 1] = fmaf(pj, __uint_as_float(w[t] & 0xFFFF0000u), o[c * 8 + 2 * t + 1]);
+        }
+      }
     }
   }
+#pragma unroll
+  for (int width = 32; width >= 2; width >>= 1) {   // columns kept after this step
+    const bool upper = (lane & (width >> 1)) != 0;  // lane bit 4, 3, .. 0 for width 32, 16, .. 2
+#pragma unroll
+    for (int c = 0; c < width; ++c) {
+      const float send = upper ? o[c] : o[c + width];
+      const float keep = upper ? o[c + width] : o[c];
+      o[c] = keep + __shfl_xor_sync(0xffffffffu, send, width >> 1);
+    }
+  }
+  const float o0 = o[0], o1 = o[1];
   const float inv = 1.f / sum;
   *reinterpret_cast<uint32_t*>(p.ctx[g] + static_cast<size_t>(b) * H + head * kHeadDim + 2 * lane) =
       pack_bf16(o0 * inv, o1 * inv);

@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     const int quarter = warp & 3;                       // TMEM lanes this warp may read
     const int col_group = e >> 2;                       // which share of the column chunks
     constexpr int COL_GROUPS = kNumEpilogueWarps / 4;
-    constexpr int CHUNK_COLS = (EPI == kEpiBiasResidual) ? 32 : 64;
+    constexpr int CHUNK_COLS = (EPI == kEpiBiasResidual || EPI == kEpiBiasTanhF32) ? 32 : 64;
     constexpr int CHUNKS = BN / CHUNK_COLS;
     const uint32_t my_stage = sStage + static_cast<uint32_t>(e * NBUF * kStagingBytes);
     const uint32_t my_res_bar = bar_res + 16 * e;       // two barriers, one per staging buffer
@@ -327,6 +327,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
             r1.w += __uint_as_float(v[q * 8 + 7]) + bf16_hi(bw[3]);
             *s0 = r0;
             *s1 = r1;
+          }
+        } else if (EPI == kEpiBiasTanhF32) {
+          // the store that last read this staging buffer must be done with it
+          if (lane == 0) {
+            if (NBUF == 2) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
+          }
+          __syncwarp();
+          uint32_t v[32];
+          tmem_ld_32x32(taddr, v);
+          tmem_ld_wait();
+          const uint4* bias4 = reinterpret_cast<const uint4*>(bias + col);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 b = __ldg(bias4 + q);
+            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+            float4 r0, r1;
+            r0.x = tanhf(__uint_as_float(v[q * 8 + 0]) + bf16_lo(bw[0]));
+            r0.y = tanhf(__uint_as_float(v[q * 8 + 1]) + bf16_hi(bw[0]));
+            r0.z = tanhf(__uint_as_float(v[q * 8 + 2]) + bf16_lo(bw[1]));
+            r0.w = tanhf(__uint_as_float(v[q * 8 + 3]) + bf16_hi(bw[1]));
+            r1.x = tanhf(__uint_as_float(v[q * 8 + 4]) + bf16_lo(bw[2]));
+            r1.y = tanhf(__uint_as_float(v[q * 8 + 5]) + bf16_hi(bw[2]));
+            r1.z = tanhf(__uint_as_float(v[q * 8 + 6]) + bf16_lo(bw[3]));
+            r1.w = tanhf(__uint_as_float(v[q * 8 + 7]) + bf16_hi(bw[3]));
+            *reinterpret_cast<float4*>(sbuf + staging_off(lane, 2 * q)) = r0;
+            *reinterpret_cast<float4*>(sbuf + staging_off(lane, 2 * q + 1)) = r1;
           }
         } else {
           // the store that last read this staging buffer must be done with it
@@ -426,6 +452,9 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
     case kEpiBiasResidual:
       if constexpr (BN != 256) return launch_one<BN, kEpiBiasResidual, PAIR>(p, sm_count, stream);
       return cudaErrorInvalidValue;  // 256-wide tiles are not used with the residual epilogue
+    case kEpiBiasTanhF32:   // the pooler: a few rows, single CTAs on 128-wide tiles only
+      if constexpr (BN == 128 && !PAIR) return launch_one<BN, kEpiBiasTanhF32, PAIR>(p, sm_count, stream);
+      return cudaErrorInvalidValue;
     default: return cudaErrorInvalidValue;
   }
 }
@@ -443,6 +472,7 @@ cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStre
 }  // namespace
 
 int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int sm_count) {
+  if (epilogue == kEpiBiasTanhF32) return 128;
   const int candidates[3] = {256, 192, 128};
   const int64_t tile_m = pair ? 2 * kGemmBlockM : kGemmBlockM;
   const int64_t workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
@@ -465,7 +495,7 @@ int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int s
   }
   return best;
 }
-int gemm_out_box_cols(int epilogue) { return epilogue == kEpiBiasResidual ? 32 : 64; }
+int gemm_out_box_cols(int epilogue) { return (epilogue == kEpiBiasResidual || epilogue == kEpiBiasTanhF32) ? 32 : 64; }
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.block_n < 1 || p.N % p.block_n != 0 ||

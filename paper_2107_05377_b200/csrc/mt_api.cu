@@ -103,6 +103,8 @@ struct PlanStep {
   int kind;  // 0 = chunk, 1 = heads, 2 = cls tail
   Chunk chunk;
   HeadParams heads;
+  bool pool_gemm = false;           // heads step: the pooler runs as a grouped GEMM (`pool`), then the head kernel
+  GemmParams pool;
   std::vector<int32_t> head_tasks;  // tasks of a heads step, in group order
   LayerTail tail;
   std::vector<DumpCopy> dumps;
@@ -159,10 +161,11 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
                            const float* residual, void* y) {
   const int M = g->M, N = g->N, K = g->K;
   const bool res = epilogue == kEpiBiasResidual;
+  const bool f32_out = res || epilogue == kEpiBiasTanhF32;
   cudaError_t e;
   if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
   if ((e = make_tmap(&g->tmap_w[i], w, N, K, g->block_n / (g->pair != 0 ? 2 : 1), kGemmBlockK, false)) != cudaSuccess) return e;
-  if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), res)) != cudaSuccess) return e;
+  if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), f32_out)) != cudaSuccess) return e;
   if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
   g->group[i].bias = bias;
   return cudaSuccess;
@@ -193,6 +196,7 @@ struct mt_model {
   int32_t fused_tail;  // steps 3-7 of a layer (output projection .. second LayerNorm) as one persistent launch per
                        // wave: 0 never, 1 always, 2 where the wave has at least fused_min_groups layers
   int32_t fused_min_groups;
+  bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
   int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
   // device memory (caller-owned)
@@ -361,6 +365,10 @@ float* f32_of(const mt_model* m, bf16* state) {
   return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(state) + m->act_bytes);
 }
 
+// True when the final state of a task is [B, H], one row per sequence.
+bool is_compact_task(const mt_model* m, int32_t task) {
+  return m->cls_only && m->tasks[task].cfg.branch_layers > 0;
+}
 // True for the last layer of a task branch when only the first token's state is needed downstream.
 bool is_cls_op(const mt_model* m, const OpDesc& op) {
   return m->cls_only && op.task >= 0 && op.layer == m->tasks[op.task].cfg.branch_layers;
@@ -608,7 +616,13 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
     plan->sync_bytes += bytes;
     return cudaSuccess;
   };
-  auto add_heads = [&](const std::vector<int32_t>& tasks) {
+  // Pooler + head of a set of tasks.  Tasks whose final state is compact ([B, H], one row per sequence:
+  // the last branch layer was evaluated on first tokens only) get their pooler as one grouped GEMM on
+  // the tensor cores, Y_t = tanh(X_t . Wp_t^T + bp_t) in fp32, followed by the head kernel; the others
+  // pool rows gathered by row_start with the two row-wise kernels.  The split is per task, so a task's
+  // logits never depend on which other tasks are active.
+  cudaError_t heads_error = cudaSuccess;
+  auto add_heads_of = [&](const std::vector<int32_t>& tasks, bool compact) {
     for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
       const size_t count = std::min<size_t>(kMaxGroups, tasks.size() - first);
       PlanStep st;
@@ -619,6 +633,16 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       st.heads.logits_stride = m->c_total;
       st.heads.pooled = reinterpret_cast<float*>(m->d_workspace + m->ws_pooled);
       st.heads.row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
+      st.pool_gemm = compact && m->pool_gemm;
+      if (st.pool_gemm) {
+        memset(&st.pool, 0, sizeof(st.pool));
+        st.pool.n_groups = static_cast<int32_t>(count);
+        st.pool.M = batch; st.pool.N = m->trunk.hidden; st.pool.K = m->trunk.hidden;
+        st.pool.pair = 0;
+        st.pool.block_n = gemm_block_n(st.pool.N, kEpiBiasTanhF32, batch, static_cast<int>(count), false, m->sm_count);
+        st.pool.m_valid = nullptr;
+        st.pool.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
+      }
       for (size_t i = 0; i < count; ++i) {
         const int32_t t = tasks[first + i];
         const TaskEntry& te = m->tasks[t];
@@ -627,12 +651,23 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         ht.pool_w = w_ptr(m, te.pool_w); ht.pool_b = w_ptr(m, te.pool_b);
         ht.cls_w = w_ptr(m, te.cls_w); ht.cls_b = w_ptr(m, te.cls_b);
         ht.num_classes = te.cfg.num_classes; ht.col0 = te.col0;
-        ht.compact = (m->cls_only && te.cfg.branch_layers > 0) ? 1 : 0;
+        ht.compact = compact ? 1 : 0;
         st.head_tasks.push_back(t);
+        if (st.pool_gemm) {
+          cudaError_t e = set_gemm_group(&st.pool, static_cast<int>(i), kEpiBiasTanhF32, ht.hidden, ht.pool_w, ht.pool_b,
+                                         nullptr, st.heads.pooled + i * static_cast<size_t>(batch) * m->trunk.hidden);
+          if (e != cudaSuccess) heads_error = e;
+        }
       }
       plan->steps.push_back(std::move(st));
       plan->launches += 2;
     }
+  };
+  auto add_heads = [&](const std::vector<int32_t>& tasks) {
+    std::vector<int32_t> compact, gathered;
+    for (int32_t t : tasks) (is_compact_task(m, t) ? compact : gathered).push_back(t);
+    add_heads_of(gathered, false);
+    add_heads_of(compact, true);
   };
   add_heads(s.heads[0]);
   for (size_t w = 1; w <= s.waves.size(); ++w) {
@@ -662,7 +697,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
     }
     add_heads(s.heads[w]);
   }
-  return cudaSuccess;
+  return heads_error;
 }
 
 cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -706,6 +741,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->attention_tc = true;
   m->expected_tokens = 0;
   m->fused_tail = 0;
+  m->pool_gemm = true;
   m->fused_min_groups = 3;
   m->tail_bn[0] = m->tail_bn[1] = m->tail_bn[2] = 0;
   m->last_lengths = nullptr;
@@ -784,6 +820,11 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "fused_tail") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_tail must be 0, 1 or 2");
     m->fused_tail = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "pool_gemm") == 0) {
+    m->pool_gemm = value != 0;
     m->plans.clear();
     return MT_OK;
   }
@@ -947,7 +988,10 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
       for (size_t first = 0; first < n_cls_tasks; first += kMaxGroups)
         n += use_fused_tail(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first))) ? 1 : 5;
     }
-    n += 2 * static_cast<int32_t>((s.heads[w].size() + kMaxGroups - 1) / kMaxGroups);
+    size_t n_compact = 0;
+    for (int32_t t : s.heads[w]) n_compact += is_compact_task(m, t) ? 1 : 0;
+    n += 2 * static_cast<int32_t>((n_compact + kMaxGroups - 1) / kMaxGroups +
+                                  (s.heads[w].size() - n_compact + kMaxGroups - 1) / kMaxGroups);
   }
   *n_launches = n;
   return MT_OK;
@@ -1073,7 +1117,12 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
                   "debug capture");
     } else {
       st.heads.logits = d_logits;
-      MT_TIMED(MT_CLASS_HEAD, launch_pooler_head(st.heads, stream), "pooler/head kernel");
+      if (st.pool_gemm) {
+        MT_TIMED(MT_CLASS_HEAD, launch_gemm(st.pool, kEpiBiasTanhF32, m->sm_count, stream), "pooler GEMM");
+        MT_TIMED(MT_CLASS_HEAD, launch_head(st.heads, stream), "head kernel");
+      } else {
+        MT_TIMED(MT_CLASS_HEAD, launch_pooler_head(st.heads, stream), "pooler/head kernel");
+      }
       if (task_events != nullptr)
         for (int32_t t : st.head_tasks)
           if (task_events[t] != nullptr)

@@ -61,11 +61,12 @@ cudaError_t launch_kernel(void (*kernel)(Param), dim3 grid, dim3 block, size_t s
 }
 #endif
 
-enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2 };
+enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2, kEpiBiasTanhF32 = 3 };
 
 // One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).
 // All groups of a launch share M, N, K and the epilogue.  kEpiBias and kEpiBiasGelu write bf16;
-// kEpiBiasResidual adds an fp32 residual and writes fp32 (the pre-LayerNorm sum is never rounded).
+// kEpiBiasResidual adds an fp32 residual and writes fp32 (the pre-LayerNorm sum is never rounded);
+// kEpiBiasTanhF32 writes tanh(.) in fp32 (the pooler; single CTAs on 128-wide tiles only).
 // The output and the residual are reached through the tensor maps of GemmParams.
 struct GemmGroup {
   const bf16* bias;
@@ -206,5 +207,7 @@ cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const
                                int32_t batch, int32_t seq, int32_t hidden, int32_t compact, cudaStream_t stream);
 // Two launches: pooler (tanh features into `pooled`), then head (logits).
 cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream);
+// The head alone, for a caller that has filled `pooled` itself (the pooler as a grouped GEMM).
+cudaError_t launch_head(const HeadParams& p, cudaStream_t stream);
 
 }  // namespace mt

@@ -269,4 +269,12 @@ cudaError_t launch_pooler_head(const HeadParams& p, cudaStream_t stream) {
   return launch_kernel(head_kernel, dim3(chunks, p.n_tasks), dim3(kHeadThreads), 0, stream, p);
 }
 
+cudaError_t launch_head(const HeadParams& p, cudaStream_t stream) {
+  if (p.n_tasks < 1 || p.n_tasks > kMaxGroups || p.batch < 1 || p.hidden % 256 != 0 || p.hidden > 1024 ||
+      p.pooled == nullptr)
+    return cudaErrorInvalidValue;
+  const int chunks = (p.batch + kSeqPerCta - 1) / kSeqPerCta;
+  return launch_kernel(head_kernel, dim3(chunks, p.n_tasks), dim3(kHeadThreads), 0, stream, p);
+}
+
 }  // namespace mt
