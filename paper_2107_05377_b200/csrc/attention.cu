@@ -394,11 +394,114 @@ __global__ void __launch_bounds__(kClsWarps * 32) cls_attention_kernel(const Cls
       pack_bf16(o0 * inv, o1 * inv);
 }
 
+// The same for sequences of at most 128 tokens: one CTA of four warps = one (sequence, head), one key
+// per lane.  A lane's K row and V row (128 bytes each) are requested together, before anything is
+// computed, so the whole kernel is two trips to memory deep: (length, first row) and then (q, K, V).
+// Maximum, sum and the 64 output columns are combined across the four warps through shared memory
+// in warp order, so the result does not depend on timing.
+constexpr int kClsShortMaxSeq = 128;
+
+__global__ void __launch_bounds__(128) cls_attention_short_kernel(const ClsAttnParams p) {
+  __shared__ float s_max[4], s_sum[4];
+  __shared__ float s_out[4][kHeadDim];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int head = blockIdx.x, b = blockIdx.y, g = blockIdx.z;
+  const int H = p.heads * kHeadDim, ld = 3 * H;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  int len = p.lengths[b];
+  len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
+  const size_t row0 = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b]) : static_cast<size_t>(b) * p.seq;
+  const bf16* base = p.qkv[g] + row0 * ld + head * kHeadDim;
+  const int j = warp * 32 + lane;   // this lane's key
+  const bool valid = j < len;
+
+  uint4 qv[8], kv[8], vv[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) qv[c] = __ldg(reinterpret_cast<const uint4*>(base) + c);
+  if (valid) {
+    const uint4* krow = reinterpret_cast<const uint4*>(base + static_cast<size_t>(j) * ld + H);
+    const uint4* vrow = reinterpret_cast<const uint4*>(base + static_cast<size_t>(j) * ld + 2 * H);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) kv[c] = krow[c];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) vv[c] = vrow[c];
+  }
+  // this head's 64 columns of the first token's fp32 residual
+  if (threadIdx.x < kHeadDim / 4) {
+    const int col = head * kHeadDim + threadIdx.x * 4;
+    *reinterpret_cast<float4*>(p.res[g] + static_cast<size_t>(b) * H + col) =
+        *reinterpret_cast<const float4*>(p.in32[g] + row0 * H + col);
+  }
+
+  float score = -INFINITY;
+  if (valid) {
+    float acc = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint32_t qw[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+      const uint32_t kw[4] = {kv[c].x, kv[c].y, kv[c].z, kv[c].w};
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        acc = fmaf(__uint_as_float(qw[t] << 16), __uint_as_float(kw[t] << 16), acc);
+        acc = fmaf(__uint_as_float(qw[t] & 0xFFFF0000u), __uint_as_float(kw[t] & 0xFFFF0000u), acc);
+      }
+    }
+    score = acc;
+  }
+  float mx = score;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) s_max[warp] = mx;
+  __syncthreads();
+  mx = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));   // key 0 is always valid: finite
+  const float scale_log2 = 0.125f * 1.4426950408889634f;
+  const float pj = valid ? exp2f((score - mx) * scale_log2) : 0.f;
+  float sum = pj;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) s_sum[warp] = sum;
+
+  float o[kHeadDim];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint32_t w[4] = {vv[c].x, vv[c].y, vv[c].z, vv[c].w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      o[c * 8 + 2 * t] = valid ? pj * __uint_as_float(w[t] << 16) : 0.f;
+      o[c * 8 + 2 * t + 1] = valid ? pj * __uint_as_float(w[t] & 0xFFFF0000u) : 0.f;
+    }
+  }
+#pragma unroll
+  for (int width = 32; width >= 2; width >>= 1) {   // columns kept after this step; lane l ends with 2l, 2l + 1
+    const bool upper = (lane & (width >> 1)) != 0;
+#pragma unroll
+    for (int c = 0; c < width; ++c) {
+      const float send = upper ? o[c] : o[c + width];
+      const float keep = upper ? o[c + width] : o[c];
+      o[c] = keep + __shfl_xor_sync(0xffffffffu, send, width >> 1);
+    }
+  }
+  s_out[warp][2 * lane] = o[0];
+  s_out[warp][2 * lane + 1] = o[1];
+  __syncthreads();
+  if (warp == 0) {
+    const float total = ((s_sum[0] + s_sum[1]) + s_sum[2]) + s_sum[3];
+    const float inv = 1.f / total;
+    const float o0 = ((s_out[0][2 * lane] + s_out[1][2 * lane]) + s_out[2][2 * lane]) + s_out[3][2 * lane];
+    const float o1 = ((s_out[0][2 * lane + 1] + s_out[1][2 * lane + 1]) + s_out[2][2 * lane + 1]) + s_out[3][2 * lane + 1];
+    *reinterpret_cast<uint32_t*>(p.ctx[g] + static_cast<size_t>(b) * H + head * kHeadDim + 2 * lane) =
+        pack_bf16(o0 * inv, o1 * inv);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_cls_attention(const ClsAttnParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1 || p.seq > 32 * kClsMaxKeysPerLane)
     return cudaErrorInvalidValue;
+  if (p.seq <= kClsShortMaxSeq)
+    return launch_kernel(cls_attention_short_kernel, dim3(p.heads, p.batch, p.n_groups), dim3(128), 0, stream, p);
   dim3 grid((p.heads + kClsWarps - 1) / kClsWarps, p.batch, p.n_groups);
   return launch_kernel(cls_attention_kernel, grid, dim3(kClsWarps * 32), 0, stream, p);
 }
