@@ -54,6 +54,7 @@ SIGNATURES = {
     "mt_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "mt_last_error_string": (C.c_char_p, [_P]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_kernel_linear_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
@@ -115,6 +116,14 @@ def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream
     N = w.shape[0]
     _check(lib().mt_kernel_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), M, N, K, epilogue,
                                   1 if cta_pair else 0, _ptr(status), _stream(stream)), "mt_kernel_linear")
+
+
+def mt_kernel_linear_layernorm(x, w, bias, residual, gamma, beta, y, y_f32, eps: float, status=None, stream=None) -> None:
+    M, K = x.shape
+    N = w.shape[0]
+    _check(lib().mt_kernel_linear_layernorm(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(y),
+                                            _ptr(y_f32), M, N, K, eps, _ptr(status), _stream(stream)),
+           "mt_kernel_linear_layernorm")
 
 
 def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None,

@@ -80,6 +80,9 @@ struct LayerTail {
   // the same five steps as one persistent launch (option "fused_tail"), with its own tile widths
   bool fused = false;
   ChainParams chain;
+  // each residual GEMM together with the LayerNorm after it, as one cluster launch (option "fused_ln")
+  bool ln_fused = false;
+  GemmLnParams attn_out_ln, ffn_down_ln;
 };
 struct DumpCopy {
   const bf16* src;
@@ -196,6 +199,9 @@ struct mt_model {
   int32_t fused_tail;  // steps 3-7 of a layer (output projection .. second LayerNorm) as one persistent launch per
                        // wave: 0 never, 1 always, 2 where the wave has at least fused_min_groups layers
   int32_t fused_min_groups;
+  int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always,
+                     // 2 for launches of at most fused_ln_max_groups layers
+  int32_t fused_ln_max_groups;
   bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
   int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
@@ -400,6 +406,17 @@ bool use_fused_tail(const mt_model* m, int32_t groups) {
   return groups >= m->fused_min_groups;
 }
 
+// Whether the residual GEMMs of `groups` layers carry their LayerNorm (see GemmLnParams).
+bool use_fused_ln(const mt_model* m, int32_t groups) {
+  if (groups < 1 || !gemm_ln_supported(m->trunk.hidden) || m->fused_ln == 0) return false;
+  return m->fused_ln == 1 || groups <= m->fused_ln_max_groups;
+}
+// Launches of steps 3-7 for `groups` layers.
+int32_t tail_launches(const mt_model* m, int32_t groups) {
+  if (use_fused_tail(m, groups)) return 1;
+  return use_fused_ln(m, groups) ? 3 : 5;
+}
+
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
   const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
   const int32_t* rows_valid =
@@ -423,6 +440,18 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
   t->fused = use_fused_tail(m, groups);
+  t->ln_fused = !t->fused && use_fused_ln(m, groups);
+  if (t->ln_fused) {
+    auto init_ln = [&](GemmLnParams* g, int32_t K) {
+      memset(g, 0, sizeof(*g));
+      g->M = rows; g->N = H; g->K = K;
+      g->m_valid = rows_valid;
+      g->eps = m->trunk.ln_eps;
+      g->status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
+    };
+    init_ln(&t->attn_out_ln, H);
+    init_ln(&t->ffn_down_ln, F);
+  }
   if (t->fused) {
     memset(&t->chain, 0, sizeof(t->chain));
     const GemmParams* like[3] = {&t->attn_out, &t->ffn_up, &t->ffn_down};
@@ -463,6 +492,24 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
   t->ln2.y[i] = out; t->ln2.y32[i] = out32;
   t->count = i + 1;
   t->attn_out.n_groups = t->ffn_up.n_groups = t->ffn_down.n_groups = t->ln1.n_groups = t->ln2.n_groups = t->count;
+  if (t->ln_fused) {
+    auto set_ln = [&](GemmLnParams* g, const void* x, size_t w, size_t b, size_t gamma, size_t beta, const float* res,
+                      bf16* y, float* y32) -> cudaError_t {
+      cudaError_t err;
+      if ((err = make_tmap(&g->tmap_x[i], x, g->M, g->K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return err;
+      if ((err = make_tmap(&g->tmap_w[i], w_ptr(m, w), g->N, g->K, 128, kGemmBlockK, false)) != cudaSuccess) return err;
+      if ((err = make_tmap(&g->tmap_res[i], res, g->M, g->N, 32, 32, true)) != cudaSuccess) return err;
+      if ((err = make_tmap(&g->tmap_y[i], y, g->M, g->N, 32, 64, false)) != cudaSuccess) return err;
+      if ((err = make_tmap(&g->tmap_y32[i], y32, g->M, g->N, 32, 32, true)) != cudaSuccess) return err;
+      g->bias[i] = w_ptr(m, b); g->gamma[i] = w_ptr(m, gamma); g->beta[i] = w_ptr(m, beta);
+      g->n_groups = i + 1;
+      return cudaSuccess;
+    };
+    // (a state is its bf16 copy followed by room for its fp32 copy: the fp32 result always has a home)
+    float* out32_home = out32 != nullptr ? out32 : f32_of(m, out);
+    if ((e = set_ln(&t->attn_out_ln, ctx, lo->wo, lo->bo, lo->ln1_g, lo->ln1_b, residual, h1, h1_32)) != cudaSuccess) return e;
+    if ((e = set_ln(&t->ffn_down_ln, f, lo->w2, lo->b2, lo->ln2_g, lo->ln2_b, h1_32, out, out32_home)) != cudaSuccess) return e;
+  }
   if (t->fused) {
     ChainParams* c = &t->chain;
     if ((e = set_gemm_group(&c->gemm[0], i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) != cudaSuccess)
@@ -587,8 +634,7 @@ cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks,
 int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count) {
   size_t n_cls = 0;
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
-  const bool fused = use_fused_tail(m, static_cast<int32_t>(count - n_cls));
-  return 1 + (n_cls < count ? (fused ? 2 : 6) : 0) + (n_cls > 0 ? 1 : 0);
+  return 1 + (n_cls < count ? 1 + tail_launches(m, static_cast<int32_t>(count - n_cls)) : 0) + (n_cls > 0 ? 1 : 0);
 }
 // Active tasks whose last branch layer is finished on first tokens right after wave w (1-based):
 // those whose last layer is in wave w with option early_heads, otherwise all of them after the last wave.
@@ -691,7 +737,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         cudaError_t e = build_cls_tail(m, tasks, first, std::min<size_t>(kMaxGroups, tasks.size() - first), batch, &st);
         if (e != cudaSuccess) return e;
         if ((e = assign_sync(&st.tail)) != cudaSuccess) return e;
-        plan->launches += st.tail.fused ? 1 : 5;
+        plan->launches += tail_launches(m, st.tail.count);
         plan->steps.push_back(std::move(st));
       }
     }
@@ -742,6 +788,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->expected_tokens = 0;
   m->fused_tail = 0;
   m->pool_gemm = true;
+  m->fused_ln = 2;
+  m->fused_ln_max_groups = 1;
   m->fused_min_groups = 3;
   m->tail_bn[0] = m->tail_bn[1] = m->tail_bn[2] = 0;
   m->last_lengths = nullptr;
@@ -820,6 +868,18 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "fused_tail") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_tail must be 0, 1 or 2");
     m->fused_tail = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "fused_ln") == 0) {
+    if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1 or 2");
+    m->fused_ln = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "fused_ln_max_groups") == 0) {
+    if (value < 1) return fail(m, MT_ERR_INVALID_ARG, "fused_ln_max_groups must be >= 1");
+    m->fused_ln_max_groups = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
   }
@@ -986,7 +1046,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
         n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
       const size_t n_cls_tasks = cls_tasks_after_wave(m, s, w).size();
       for (size_t first = 0; first < n_cls_tasks; first += kMaxGroups)
-        n += use_fused_tail(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first))) ? 1 : 5;
+        n += tail_launches(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first)));
     }
     size_t n_compact = 0;
     for (int32_t t : s.heads[w]) n_compact += is_compact_task(m, t) ? 1 : 0;
@@ -1063,6 +1123,10 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     LayerTail* t_ = (tail);                                                                                            \
     if (t_->fused) {                                                                                                   \
       MT_TIMED(MT_CLASS_TAIL, launch_chain(t_->chain, m->sm_count, stream), "fused layer-tail kernel");                \
+    } else if (t_->ln_fused) {                                                                                         \
+      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm_ln(t_->attn_out_ln, stream), "attention output GEMM + LayerNorm");       \
+      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");            \
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm_ln(t_->ffn_down_ln, stream), "FFN down GEMM + LayerNorm");               \
     } else {                                                                                                           \
       MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t_->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM"); \
       MT_TIMED(MT_CLASS_LN1, launch_layernorm(t_->ln1, stream), "LayerNorm 1");                                        \
@@ -1239,6 +1303,28 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
                      d_y) != cudaSuccess)
     return MT_ERR_CUDA;
   return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_linear_layernorm(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
+                               const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32, int32_t M, int32_t N,
+                               int32_t K, float eps, uint32_t* d_status, void* stream) {
+  if (d_x == nullptr || d_w == nullptr || d_bias == nullptr || d_residual == nullptr || d_gamma == nullptr ||
+      d_beta == nullptr || d_y == nullptr || d_y_f32 == nullptr || M < 1 || !gemm_ln_supported(N) || K < 64 || K % 64 != 0 ||
+      !(eps >= 0.f))
+    return MT_ERR_INVALID_ARG;
+  GemmLnParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.eps = eps; p.status = d_status;
+  if (make_tmap(&p.tmap_x[0], d_x, M, K, kGemmBlockM, kGemmBlockK, false) != cudaSuccess ||
+      make_tmap(&p.tmap_w[0], d_w, N, K, 128, kGemmBlockK, false) != cudaSuccess ||
+      make_tmap(&p.tmap_res[0], d_residual, M, N, 32, 32, true) != cudaSuccess ||
+      make_tmap(&p.tmap_y[0], d_y, M, N, 32, 64, false) != cudaSuccess ||
+      make_tmap(&p.tmap_y32[0], d_y_f32, M, N, 32, 32, true) != cudaSuccess)
+    return MT_ERR_CUDA;
+  p.bias[0] = static_cast<const bf16*>(d_bias);
+  p.gamma[0] = static_cast<const bf16*>(d_gamma);
+  p.beta[0] = static_cast<const bf16*>(d_beta);
+  return launch_gemm_ln(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
 int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx, int32_t batch, int32_t seq,

@@ -168,6 +168,30 @@ bool chain_supported(int hidden, int ffn);
 int chain_block_n(int phase, int N, int64_t rows, int groups, int sm_count);
 cudaError_t launch_chain(const ChainParams& p, int sm_count, cudaStream_t stream);
 
+// Residual GEMM with the LayerNorm that follows it, in one launch:
+//   Y_g = LN( X_g[M,K] . W_g[N,K]^T + bias_g + residual_g ) * gamma_g + beta_g      N = hidden
+// written twice, bf16 (the next GEMM's operand) and fp32 (the next residual).  The N / 128 CTAs that hold
+// the column blocks of one block of 128 rows form a thread-block cluster and exchange per-row partial
+// statistics through distributed shared memory, so the pre-normalisation sum never goes to global memory.
+struct alignas(64) GemmLnParams {
+  CUtensorMap tmap_x[kMaxGroups];     // X_g: dims {K, M}, box {64, 128}
+  CUtensorMap tmap_w[kMaxGroups];     // W_g: dims {K, N}, box {64, 128}
+  CUtensorMap tmap_res[kMaxGroups];   // residual_g fp32: dims {N, M}, box {32, 32}
+  CUtensorMap tmap_y[kMaxGroups];     // Y_g bf16: dims {N, M}, box {64, 32}
+  CUtensorMap tmap_y32[kMaxGroups];   // Y_g fp32: dims {N, M}, box {32, 32}
+  const bf16* bias[kMaxGroups];
+  const bf16* gamma[kMaxGroups];
+  const bf16* beta[kMaxGroups];
+  int32_t n_groups;
+  int32_t M, N, K;
+  const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
+  float eps;
+  uint32_t* status;        // sticky device status word (may be null)
+};
+// N must be 768 or 1024 (clusters of 6 or 8 CTAs), K a multiple of 64.
+bool gemm_ln_supported(int N);
+cudaError_t launch_gemm_ln(const GemmLnParams& p, cudaStream_t stream);
+
 struct EmbedParams {
   const int32_t* token_ids;
   const int32_t* segment_ids;

@@ -17,9 +17,11 @@ LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
 def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None,
-              gemm_pair=None, attention_tc=None, expected_tokens=None, fused_tail=None, tail_bn=None):
+              gemm_pair=None, attention_tc=None, expected_tokens=None, fused_tail=None, tail_bn=None, fused_ln=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
+    if fused_ln is not None:
+        model.set_option("fused_ln", fused_ln)
     if fused_tail is not None:
         model.set_option("fused_tail", fused_tail)
     if tail_bn is not None:
@@ -112,6 +114,46 @@ def test_every_token_in_last_branch_layers_matches_oracle_and_first_token_only()
     assert float((first - full).abs().max()) <= 2e-3
 
 
+def test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches():
+    """Residual GEMM + LayerNorm as one cluster launch (option "fused_ln", the default; per-row statistics
+    exchanged through distributed shared memory) against the separate GEMM and LayerNorm launches: both
+    match the oracle at every hidden state, and, because every LayerNorm of the library sums its row
+    statistics over the same 64-column segments in the same order, they agree bit for bit - which is what
+    lets the default choose between them by the size of a launch."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
+    m_sep, separate = run_model(cfg, blob, batch, debug=True, fused_ln=0)
+    check_against_oracle(cfg, wf, batch, m_sep, separate, rows=range(6))
+    m_fus, fused = run_model(cfg, blob, batch, debug=True, fused_ln=1)
+    check_against_oracle(cfg, wf, batch, m_fus, fused, rows=range(6))
+    assert torch.equal(fused, separate)
+    B, S = batch.token_ids.shape
+    for t, layer in ((-1, 1), (-1, 3), (1, 1), (1, 2), (3, 1)):
+        assert torch.equal(m_fus.debug_hidden(t, layer, B, S), m_sep.debug_hidden(t, layer, B, S)), (t, layer)
+    _, auto = run_model(cfg, blob, batch, fused_ln=2)
+    assert torch.equal(auto, separate)
+    # all rows in the last layers, padded layout: more and fuller row blocks
+    m_full, full = run_model(cfg, blob, batch, debug=True, cls_only=0, pack_tokens=0, fused_ln=1)
+    check_against_oracle(cfg, wf, batch, m_full, full, rows=range(6), cls_only=False)
+    # the 8-task tree, repeated forwards: deterministic bits, oracle parity on sampled sequences
+    big = synth.config_glue8()
+    w8, blob8, wf8 = cached_weights(big, 0)
+    b8 = synth.batch_glue8(big)
+    _, sep8 = run_model(big, blob8, b8, fused_ln=0)
+    m8, first = run_model(big, blob8, b8, fused_ln=1)
+    assert torch.equal(first, sep8)
+    tok, seg, lens = dev_batch(b8)
+    again = torch.zeros_like(first)
+    for _ in range(3):
+        m8.forward(tok, seg, lens, again)
+    torch.cuda.synchronize()
+    assert m8.poll_status() == 0
+    assert torch.equal(again, first)
+    check_against_oracle(big, wf8, b8, m8, again, rows=[0, 13, 31], check_hidden=False)
+
+
 def test_fused_layer_tail_matches_oracle_and_separate_launches_bits():
     """The part of a layer after attention as one persistent launch per wave (option "fused_tail", the
     default) against the five separate launches: every element is the same arithmetic, so hidden
@@ -120,7 +162,7 @@ def test_fused_layer_tail_matches_oracle_and_separate_launches_bits():
                                                   synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
     w, blob, wf = cached_weights(cfg, 5, random_affine=True)
     batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
-    m_sep, separate = run_model(cfg, blob, batch, debug=True, fused_tail=0)
+    m_sep, separate = run_model(cfg, blob, batch, debug=True, fused_tail=0, fused_ln=0)
     m_fus, fused = run_model(cfg, blob, batch, debug=True, fused_tail=1)
     check_against_oracle(cfg, wf, batch, m_fus, fused, rows=range(6))
     assert torch.equal(fused, separate)
@@ -131,13 +173,13 @@ def test_fused_layer_tail_matches_oracle_and_separate_launches_bits():
         _, got = run_model(cfg, blob, batch, fused_tail=1, tail_bn=bn)
         assert torch.equal(got, separate), bn
     # every token in the last branch layers too (more rows in the fused launches), and the padded layout
-    _, full_sep = run_model(cfg, blob, batch, cls_only=0, pack_tokens=0, fused_tail=0)
+    _, full_sep = run_model(cfg, blob, batch, cls_only=0, pack_tokens=0, fused_tail=0, fused_ln=0)
     _, full_fus = run_model(cfg, blob, batch, cls_only=0, pack_tokens=0, fused_tail=1)
     assert torch.equal(full_fus, full_sep)
     big = synth.config_glue8()
     w8, blob8, wf8 = cached_weights(big, 0)
     b8 = synth.batch_glue8(big)
-    _, s8 = run_model(big, blob8, b8, fused_tail=0)
+    _, s8 = run_model(big, blob8, b8, fused_tail=0, fused_ln=0)
     for _ in range(3):   # repeated forwards reuse the counters after the memset
         m8, f8 = run_model(big, blob8, b8, fused_tail=1)
         assert torch.equal(f8, s8)

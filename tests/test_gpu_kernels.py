@@ -61,6 +61,49 @@ def test_linear_matches_oracle(M, N, K, epi, pair):
         assert np.max(np.abs(got - want)) <= bf16_round_tol(want)
 
 
+@pytest.mark.parametrize("M,N,K", [
+    (40, 768, 768),           # fewer rows than one tile: a single cluster of six CTAs
+    (333, 768, 768),          # ragged last row block
+    (2409, 768, 3072),        # FFN down + LayerNorm at the valid-token count of the 32 x 128 batch
+    (4096, 768, 768),         # more row blocks than clusters fit the GPU at once: several tiles per cluster
+    (700, 1024, 4096),        # BERT-large width: clusters of eight
+])
+def test_linear_layernorm_cluster_matches_oracle_and_separate_kernels(M, N, K):
+    """Residual GEMM + LayerNorm in one cluster launch (row statistics through distributed shared memory):
+    against the oracle's linear + residual + layer_norm, and bit for bit against the plain residual GEMM
+    followed by the LayerNorm kernel, which sums the row statistics in the same order."""
+    xb, x = rand_bf16(21, f"x{M}.{N}.{K}", (M, K), 1.0)
+    wb, w = rand_bf16(22, f"w{M}.{N}.{K}", (N, K), 0.05)
+    bb, b = rand_bf16(23, f"b{M}.{N}.{K}", (N,), 0.5)
+    gb, g = rand_bf16(24, f"g{N}", (N,), 0.3, mean=1.0)
+    beb, be = rand_bf16(25, f"be{N}", (N,), 0.2)
+    r32 = (synth.standard_normal(26, f"r{M}.{N}.{K}", M * N).astype(np.float32)).reshape(M, N)
+    g_dev = to_dev_bf16(gb)
+    res = torch.from_numpy(r32).cuda()
+    y = torch.full((M + 8, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y32 = torch.full((M + 8, N), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    xd, wd, bd, bed = to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(bb), to_dev_bf16(beb)
+    mt.mt_kernel_linear_layernorm(xd, wd, bd, res, g_dev, bed, y[:M], y32[:M], 1e-12, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.isnan(y[M:].float()).all() and torch.isnan(y32[M:]).all(), "rows beyond M were written"
+    want = orc.layer_norm(orc.linear(x, w, b) + r32.astype(np.float64), g, be, 1e-12)
+    got32 = y32[:M].cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got32))
+    assert rel_l2(got32, want) <= 1e-5
+    got = y[:M].float().cpu().numpy().astype(np.float64)
+    assert rel_l2(got, want) <= OUT_REL_L2
+    assert np.max(np.abs(got - want)) <= bf16_round_tol(want)
+    u = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    z = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    z32 = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    mt.mt_kernel_linear(xd, wd, bd, res, u, 2)
+    mt.mt_kernel_layernorm(u, g_dev, bed, z, 1e-12, y_f32=z32)
+    torch.cuda.synchronize()
+    assert torch.equal(z32, y32[:M]) and torch.equal(z, y[:M])
+
+
 def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
     H = heads * 64
     ctx = np.zeros((B * S, H))

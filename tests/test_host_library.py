@@ -71,6 +71,14 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
         assert m.plan_summary(mask)["layers"] == want
     with pytest.raises(binding.MTError):
         m.plan_summary(0)
+    # fused_ln = 1: each residual GEMM carries the LayerNorm after it, so a layer on all tokens is 5 launches
+    # (projection, attention, output + LN, FFN up, FFN down + LN), a first-token tail 3
+    m.set_option("fused_ln", 1)
+    assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 3 + 2
+    # default (2): only where a single layer is on all tokens: waves 1-4 and wave 9
+    m.set_option("fused_ln", 2)
+    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 7 + 7 + 8 + 8 + 6 + 2 + 5 + 2
+    m.set_option("fused_ln", 0)
     # fused_tail = 1: the part of a layer after attention is one launch, so a wave is projection + attention
     # + fused tail (+ first-token attention where a branch ends); one fused first-token tail; pooler + head
     m.set_option("fused_tail", 1)
@@ -94,6 +102,7 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     m.close()
     m2 = binding.MTModel(cfg, 32, 128, max_groups=2, bind=False)
     m2.set_option("cls_only_last_layer", 0)
+    m2.set_option("fused_ln", 0)
     assert m2.plan_summary(0xFF)["layers"] == 24
     assert m2.plan_launches(0xFF) == 2 + 7 * (1 + 1 + 1 + 1 + 1 + 2 + 3 + 3 + 2 + 1) + 2
     m2.close()
