@@ -1,6 +1,7 @@
 """Micro-benchmark of the single steps of the path, each called through the C ABI.
 
     python -m paper_2107_05377_b200.kernel_bench linear --m 4096 --n 2304 --k 768 --epilogue 0
+    python -m paper_2107_05377_b200.kernel_bench linear_ln --m 4096 --n 768 --k 3072   # residual GEMM + LayerNorm, one launch
     python -m paper_2107_05377_b200.kernel_bench attention --batch 32 --seq 128 --heads 12
     python -m paper_2107_05377_b200.kernel_bench layernorm --rows 4096 --hidden 768
     python -m paper_2107_05377_b200.kernel_bench suite          # the shapes of the 32 x 128 workload
@@ -80,6 +81,22 @@ def bench_linear(m, n, k, epilogue, iters, warmup, flush):
             "tflops": flops / ms / 1e9, "min_gbytes_per_s": bytes_ / ms / 1e6}
 
 
+def bench_linear_ln(m, n, k, iters, warmup, flush):
+    x = torch.randn(m, k, device="cuda").to(torch.bfloat16)
+    w = (0.02 * torch.randn(n, k, device="cuda")).to(torch.bfloat16)
+    b = (0.02 * torch.randn(n, device="cuda")).to(torch.bfloat16)
+    g = torch.ones(n, device="cuda", dtype=torch.bfloat16)
+    be = torch.zeros(n, device="cuda", dtype=torch.bfloat16)
+    r = torch.randn(m, n, device="cuda")
+    y = torch.empty(m, n, device="cuda", dtype=torch.bfloat16)
+    y32 = torch.empty(m, n, device="cuda")
+    ms = _time(lambda: mt.mt_kernel_linear_layernorm(x, w, b, r, g, be, y, y32, 1e-12), iters, warmup, flush)
+    flops = 2.0 * m * n * k
+    bytes_ = 2.0 * (m * k + n * k) + (4.0 + 2.0 + 4.0) * m * n
+    return {"kernel": "linear_ln", "M": m, "N": n, "K": k, "us": 1e3 * ms, "tflops": flops / ms / 1e9,
+            "min_gbytes_per_s": bytes_ / ms / 1e6}
+
+
 def bench_attention(batch, seq, heads, len_lo, iters, warmup, flush):
     hidden = heads * 64
     qkv = torch.randn(batch * seq, 3 * hidden, device="cuda").to(torch.bfloat16)
@@ -106,7 +123,7 @@ def bench_layernorm(rows, hidden, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["linear", "attention", "layernorm", "suite"])
+    ap.add_argument("kernel", choices=["linear", "linear_ln", "attention", "layernorm", "suite"])
     ap.add_argument("--m", type=int, default=4096)
     ap.add_argument("--n", type=int, default=2304)
     ap.add_argument("--k", type=int, default=768)
@@ -131,6 +148,8 @@ def main():
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
+    elif a.kernel == "linear_ln":
+        print(json.dumps(bench_linear_ln(a.m, a.n, a.k, a.iters, a.warmup, a.flush)))
     elif a.kernel == "attention":
         print(json.dumps(bench_attention(a.batch, a.seq, a.heads, a.len_lo, a.iters, a.warmup, a.flush)))
     elif a.kernel == "layernorm":
@@ -139,6 +158,8 @@ def main():
         for m in (4096, 24576):   # one layer, and six layers' worth of rows
             for (n, k, e) in ((2304, 768, 0), (768, 768, 2), (3072, 768, 1), (768, 3072, 2)):
                 print(json.dumps(bench_linear(m, n, k, e, a.iters, a.warmup, a.flush)))
+            for (n, k) in ((768, 768), (768, 3072)):
+                print(json.dumps(bench_linear_ln(m, n, k, a.iters, a.warmup, a.flush)))
         print(json.dumps(bench_linear(8192, 8192, 8192, 0, 10, 2, a.flush)))
         print(json.dumps(bench_attention(32, 128, 12, 16, a.iters, a.warmup, a.flush)))
         print(json.dumps(bench_attention(16, 512, 12, 128, a.iters, a.warmup, a.flush)))
