@@ -40,9 +40,18 @@ REFERENCE_SAMPLE = 8          # sequences per step of the oracle arm
 L2_FLUSH_BYTES = 256 << 20    # larger than the 126 MB L2
 
 # DRAM traffic of the dominant kernel from one ncu capture (bytes per launch, averaged over the GEMM
-# launches of one forward), valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"gemm_source_sha256": "471f7cbefcedde05ccd6681669ad8ca1bce1af445f6f7fc575ac90168a68f0aa",
-               "bytes_per_launch": 25007170}  # profiles/bench_glue8_b32_s128_launch_list.md
+# launches of the forwards of `bench.py --steps 2`), valid only for the kernel sources it was taken on.
+GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_ln_tcgen05.cu", "tc_ptx.cuh", "rowwise.cuh")
+NCU_TRAFFIC = {"gemm_sources_sha256": "9f4580f4763ed2eabf2f0c982de0a6f57ac61e727a964d190084a7ced0cd254d",
+               "bytes_per_launch": 25205938}  # profiles/bench_glue8_b32_s128_launch_list.md
+
+
+def gemm_sources_digest():
+    h = hashlib.sha256()
+    for name in GEMM_SOURCES:
+        with open(os.path.join(ROOT, "paper_2107_05377_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def measured_peaks():
@@ -302,9 +311,7 @@ def main():
         n_first = sum(1 for t in cfg.tasks if t.branch_layers > 0)   # last branch layers: first token only
         gemm_flops = sum(gemm_flops_per_forward(cfg, plan["layers"], t, n_first, BATCH) for t in step_tokens)
         achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
-        src = open(os.path.join(ROOT, "paper_2107_05377_b200", "csrc", "gemm_tcgen05.cu"), "rb").read()
-        traffic = NCU_TRAFFIC["bytes_per_launch"] \
-            if NCU_TRAFFIC["gemm_source_sha256"] == hashlib.sha256(src).hexdigest() else None
+        traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["gemm_sources_sha256"] == gemm_sources_digest() else None
         valid_tokens = float(np.mean(step_tokens))
         padded_flops = gemm_flops_per_forward(cfg, plan["layers"], m_rows) + \
             plan["layers"] * BATCH * 4.0 * cfg.hidden * SEQ * SEQ
@@ -328,7 +335,8 @@ def main():
             "e2e": {"value": aggregate_throughput(world, BATCH, args.steps, e2e_s), "unit": UNIT,
                     "h2d_bytes_per_step": 2 * BATCH * SEQ * 4 + BATCH * 4,
                     "d2h_bytes_per_step": BATCH * cfg.total_classes * 4},
-            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches)",
+            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 and gemm_ln_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches; where a "
+                                   "single layer is in the launch the two residual GEMMs include the LayerNorm after them)",
                          "flops": "valid tokens only; the last layer of each branch counts its Q/K/V projection on all "
                                   "tokens and the rest on one token per sequence",
                          "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
