@@ -79,6 +79,12 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void st_cluster_f2(uint32_t cluster_addr, float a, float b) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(cluster_addr), "f"(a), "f"(b) : "memory");
 }
+// Release at cluster scope once, then arrivals that carry no ordering of their own: one fence instead of
+// one per peer.
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ uint32_t cluster_id_x() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
@@ -308,9 +314,11 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
       const uint32_t slot = sStats + static_cast<uint32_t>((((parity * kLnMaxCluster + rank) * 2 + half) * kGemmBlockM + row_in_tile) * 8);
       for (int peer = 0; peer < cluster_size; ++peer) st_cluster_f2(map_to_cta(slot, static_cast<uint32_t>(peer)), mean_l, m2_l);
       __syncwarp();
-      if (lane == 0)
+      if (lane == 0) {
+        fence_acq_rel_cluster();
         for (int peer = 0; peer < cluster_size; ++peer)
-          mbar_arrive_cluster(map_to_cta(bar_stats + 8 * parity, static_cast<uint32_t>(peer)));
+          mbar_arrive_cluster_relaxed(map_to_cta(bar_stats + 8 * parity, static_cast<uint32_t>(peer)));
+      }
       if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_stats + 8 * parity, stats_phase[parity], abort_flag))) break;
       stats_phase[parity] ^= 1u;
       // merge the 2 * cluster_size segment statistics of this row, in column order
