@@ -115,11 +115,24 @@ def pooler_head(g: np.ndarray, task_w: Dict[str, np.ndarray]) -> np.ndarray:
     return linear(pooled, task_w["cls_w"], task_w["cls_b"])
 
 
+def token_head(g: np.ndarray, task_w: Dict[str, np.ndarray]) -> np.ndarray:
+    """Token-level task (the production system of Appendix E serves token-level tasks beside the
+    sequence-level ones and gives no formula for their output layer): the plain reading, one linear
+    map on every token's final state, logits_i = W_c g_i + b_c, no pooler.  Returns [n, C]."""
+    return linear(g, task_w["cls_w"], task_w["cls_b"])
+
+
 # ---------------------------------------------------------------------------
 # the merged tree (Fig. 1(c)) and the stand-alone students (Fig. 1(b))
 # ---------------------------------------------------------------------------
 
-TaskTriple = Tuple[int, int, int]  # (fork_depth x, branch_layers y, num_classes)
+# (fork_depth x, branch_layers y, num_classes) or, with a head kind, (x, y, num_classes, kind):
+# kind 0 = sequence-level head (pooler on the first token + linear), kind 1 = token-level head.
+TaskTriple = Tuple[int, ...]
+
+
+def head_kind(task: TaskTriple) -> int:
+    return int(task[3]) if len(task) > 3 else 0
 
 
 def active_tasks(n_tasks: int, task_mask: Optional[int]) -> List[int]:
@@ -180,7 +193,7 @@ def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weight
 
     out = {}
     for t in act:
-        x, y, _ = tasks[t]
+        x, y = tasks[t][0], tasks[t][1]
         g = forks[x]
         for j in range(1, y + 1):
             g = encoder_layer(g, weights["tasks"][t]["layers"][j - 1], heads, eps)
@@ -188,7 +201,7 @@ def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weight
                 counter.count += 1
             if hidden_out is not None:
                 hidden_out[("task", t, j)] = g
-        out[t] = pooler_head(g, weights["tasks"][t])
+        out[t] = token_head(g, weights["tasks"][t]) if head_kind(tasks[t]) == 1 else pooler_head(g, weights["tasks"][t])
     return out
 
 
@@ -198,7 +211,7 @@ def forward_sequence_st(tokens: np.ndarray, segments: np.ndarray, n: int, weight
     """The stand-alone student of ``task`` run by itself: its x frozen layers,
     then its y task layers, then its head.  Deliberately written as its own
     straight-line loop, sharing no state with the merged evaluation."""
-    x, y, _ = tasks[task]
+    x, y = tasks[task][0], tasks[task][1]
     g = embed(np.asarray(tokens[:n], dtype=np.int64), np.asarray(segments[:n], dtype=np.int64),
               weights["emb"], eps)
     chain = [weights["trunk"][l] for l in range(x)] + [weights["tasks"][task]["layers"][j] for j in range(y)]
@@ -206,26 +219,42 @@ def forward_sequence_st(tokens: np.ndarray, segments: np.ndarray, n: int, weight
         g = encoder_layer(g, layer, heads, eps)
         if counter is not None:
             counter.count += 1
+    if head_kind(tasks[task]) == 1:
+        return token_head(g, weights["tasks"][task])
     return pooler_head(g, weights["tasks"][task])
 
 
 def forward_batch_mt(token_ids: np.ndarray, segment_ids: np.ndarray, lengths: np.ndarray, weights: Dict,
                      tasks: Sequence[TaskTriple], heads: int, eps: float,
                      task_mask: Optional[int] = None, rows: Optional[Iterable[int]] = None,
-                     hidden_out: Optional[List[Dict]] = None) -> np.ndarray:
+                     hidden_out: Optional[List[Dict]] = None,
+                     token_logits_out: Optional[List[np.ndarray]] = None) -> np.ndarray:
     """Merged forward of a padded batch.  Returns float64 logits
-    [B, sum C_t]; task t occupies columns [off_t, off_t + C_t); columns of
-    inactive tasks and rows not in ``rows`` are NaN.  Sequences are
-    independent, so ``rows`` selects an exact subset."""
-    B = token_ids.shape[0]
-    offs = np.concatenate([[0], np.cumsum([c for _, _, c in tasks])]).astype(int)
+    [B, sum C_t over the sequence-level tasks]; task t occupies columns
+    [off_t, off_t + C_t); columns of inactive tasks and rows not in ``rows``
+    are NaN.  Token-level tasks have columns of their own, counted over the
+    token-level tasks only, in a [B, S, sum C_t] array appended to
+    ``token_logits_out`` (NaN at positions >= length, for inactive tasks and
+    for rows not selected).  Sequences are independent, so ``rows`` selects an
+    exact subset."""
+    B, S = token_ids.shape
+    seq_c = [0 if head_kind(t) == 1 else t[2] for t in tasks]
+    tok_c = [t[2] if head_kind(t) == 1 else 0 for t in tasks]
+    offs = np.concatenate([[0], np.cumsum(seq_c)]).astype(int)
+    tok_offs = np.concatenate([[0], np.cumsum(tok_c)]).astype(int)
     logits = np.full((B, offs[-1]), np.nan, dtype=np.float64)
+    token_logits = np.full((B, S, tok_offs[-1]), np.nan, dtype=np.float64)
     for b in (range(B) if rows is None else rows):
         hid = {} if hidden_out is not None else None
         res = forward_sequence_mt(token_ids[b], segment_ids[b], int(lengths[b]), weights, tasks, heads, eps,
                                   task_mask=task_mask, hidden_out=hid)
         for t, lg in res.items():
-            logits[b, offs[t]:offs[t + 1]] = lg
+            if head_kind(tasks[t]) == 1:
+                token_logits[b, :lg.shape[0], tok_offs[t]:tok_offs[t + 1]] = lg
+            else:
+                logits[b, offs[t]:offs[t + 1]] = lg
         if hidden_out is not None:
             hidden_out.append(hid)
+    if token_logits_out is not None:
+        token_logits_out.append(token_logits)
     return logits

@@ -288,6 +288,72 @@ def test_pooler_head_row0_tanh_scalar():
     assert orc.pooler_head(g, w["tasks"][2]).shape == (1,)  # 1-wide regression head, raw output
 
 
+def test_token_head_is_one_linear_map_per_token_scalar():
+    """Token-level head: logits[i, c] = b_c + sum_k g[i, k] W_c[c, k] for every token i, by scalar loops;
+    a token's logits depend on that token's state alone; no pooler weights are involved."""
+    rng = np.random.default_rng(18)
+    w, tasks = tiny_model(rng)
+    tw = w["tasks"][1]
+    g = rng.normal(size=(5, 8))
+    got = orc.token_head(g, tw)
+    assert got.shape == (5, 3)
+    for i in range(5):
+        for c in range(3):
+            want = tw["cls_b"][c] + sum(g[i, k] * tw["cls_w"][c, k] for k in range(8))
+            assert abs(got[i, c] - want) <= 1e-14
+    g2 = g.copy()
+    g2[3] += 1.0
+    again = orc.token_head(g2, tw)
+    assert np.array_equal(np.delete(again, 3, axis=0), np.delete(got, 3, axis=0)) and not np.array_equal(again[3], got[3])
+    tw2 = dict(tw)
+    tw2["pool_w"] = tw["pool_w"] + 1.0
+    tw2["pool_b"] = tw["pool_b"] - 1.0
+    assert np.array_equal(orc.token_head(g, tw2), got)
+    # zero weight matrix: every token gets the bias
+    tw3 = dict(tw)
+    tw3["cls_w"] = np.zeros_like(tw["cls_w"])
+    assert np.array_equal(orc.token_head(g, tw3), np.tile(tw["cls_b"], (5, 1)))
+
+
+def test_token_level_tasks_in_the_merged_tree():
+    """A tree that mixes sequence-level and token-level tasks: merged == stand-alone for both kinds, the
+    token-level task's logits are its final state through the linear head, padding and task masking
+    leave them untouched, and the two kinds of output have separate column spaces."""
+    rng = np.random.default_rng(19)
+    tasks = ((2, 1, 2, 0), (4, 2, 3, 1), (0, 1, 1), (3, 0, 2, 1))
+    w, _ = tiny_model(rng, tasks=tuple(t[:3] for t in tasks))
+    tok, seg, lens = _inputs(rng, 3, 10, 20, [10, 4, 1])
+    for b in range(3):
+        hid = {}
+        mt = orc.forward_sequence_mt(tok[b], seg[b], lens[b], w, tasks, 2, 1e-12, hidden_out=hid)
+        for t in range(4):
+            st = orc.forward_sequence_st(tok[b], seg[b], lens[b], w, t, tasks, 2, 1e-12)
+            want_shape = (lens[b], tasks[t][2]) if orc.head_kind(tasks[t]) == 1 else (tasks[t][2],)
+            assert mt[t].shape == want_shape
+            assert np.max(np.abs(mt[t] - st)) <= 1e-12
+        final1 = hid[("task", 1, 2)]
+        assert np.array_equal(mt[1], final1 @ w["tasks"][1]["cls_w"].T + w["tasks"][1]["cls_b"])
+        assert np.array_equal(mt[3], hid[("trunk", 3)] @ w["tasks"][3]["cls_w"].T + w["tasks"][3]["cls_b"])
+    tl = []
+    logits = orc.forward_batch_mt(tok, seg, lens, w, tasks, 2, 1e-12, token_logits_out=tl)
+    assert logits.shape == (3, 3) and tl[0].shape == (3, 10, 5)     # sequence-level: 2 + 1; token-level: 3 + 2
+    assert np.all(np.isnan(tl[0][1, 4:])) and np.all(np.isfinite(tl[0][1, :4])) and np.all(np.isfinite(logits))
+    # padding invariance: more padded positions with arbitrary ids behind them change nothing
+    tok2 = np.concatenate([tok, rng.integers(1, 20, (3, 2))], axis=1)
+    seg2 = np.concatenate([seg, np.ones((3, 2), dtype=np.int64)], axis=1)
+    tl2 = []
+    logits2 = orc.forward_batch_mt(tok2, seg2, lens, w, tasks, 2, 1e-12, token_logits_out=tl2)
+    assert np.array_equal(logits2, logits) and np.array_equal(tl2[0][:, :10], tl[0], equal_nan=True)
+    # masking: an active task's outputs do not depend on the others
+    tl3 = []
+    part = orc.forward_batch_mt(tok, seg, lens, w, tasks, 2, 1e-12, task_mask=0b1010, token_logits_out=tl3)
+    assert np.all(np.isnan(part)) and np.array_equal(tl3[0], tl[0], equal_nan=True)
+    tl4 = []
+    part = orc.forward_batch_mt(tok, seg, lens, w, tasks, 2, 1e-12, task_mask=0b0011, token_logits_out=tl4)
+    assert np.array_equal(part[:, :2], logits[:, :2]) and np.all(np.isnan(part[:, 2:]))
+    assert np.array_equal(tl4[0][..., :3], tl[0][..., :3], equal_nan=True) and np.all(np.isnan(tl4[0][..., 3:]))
+
+
 # ---------------------------------------------------------------------------
 # the merged tree: the paper's claims
 # ---------------------------------------------------------------------------
