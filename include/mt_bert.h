@@ -70,7 +70,14 @@ typedef struct {
   int32_t fork_depth;     /* 0..trunk_layers; 0 forks off the embedding output */
   int32_t branch_layers;  /* >= 0; 0 pools the trunk state directly            */
   int32_t num_classes;    /* >= 1; 1 = regression head (raw output)            */
+  int32_t head_kind;      /* MT_HEAD_SEQUENCE or MT_HEAD_TOKEN                 */
 } mt_task_config;
+/* Output layer of a task.  The paper's GLUE tasks are sequence-level: tanh pooler on the first token,
+ * then a linear head.  Its production system (Appendix E) also serves token-level tasks and gives no
+ * formula for them; the reading here is one linear map on every token's final state, no pooler (the
+ * task's pooler tensors stay in the blob, unused). */
+#define MT_HEAD_SEQUENCE 0
+#define MT_HEAD_TOKEN    1
 
 typedef struct mt_model mt_model;
 
@@ -146,6 +153,19 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
 int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
                       const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
                       float* d_logits, void* const* task_events, void* stream);
+
+/* mt_forward_events for trees with token-level tasks (mt_task_config.head_kind = MT_HEAD_TOKEN).
+ *   d_logits       : fp32 [batch, C_total], C_total counted over the sequence-level tasks only, task t in
+ *                    columns [off_t, off_t + C_t) among them (may be NULL if none is active)
+ *   d_token_logits : fp32 [batch, seq, Ct_total], Ct_total counted over the token-level tasks only;
+ *                    element (b, pos, off_t + c) for pos < length(b); positions >= length and columns of
+ *                    tasks not in the mask are left untouched (may be NULL if no token-level task is active)
+ * A token-level task's last branch layer is evaluated on all tokens (nothing to skip), and its head
+ * runs right after the wave that completes its branch.  mt_forward and mt_forward_events are this call
+ * with d_token_logits = NULL: they fail with INVALID_ARG if the mask selects a token-level task. */
+int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
+                      const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
+                      float* d_logits, float* d_token_logits, void* const* task_events, void* stream);
 
 /* Same computation from HOST buffers: copies the three inputs to the workspace, runs mt_forward,
  * copies the logits back to h_logits ([batch, C_total] fp32) and synchronises the stream.

@@ -28,7 +28,8 @@ class TrunkConfig(C.Structure):
 
 
 class TaskConfig(C.Structure):
-    _fields_ = [("fork_depth", C.c_int32), ("branch_layers", C.c_int32), ("num_classes", C.c_int32)]
+    _fields_ = [("fork_depth", C.c_int32), ("branch_layers", C.c_int32), ("num_classes", C.c_int32),
+                ("head_kind", C.c_int32)]
 
 
 # name -> (restype, argtypes); the list is also what the symbol-export test checks.
@@ -45,6 +46,7 @@ SIGNATURES = {
     "mt_load_task_weights": (C.c_int, [_P, _I32, _P, _SZ, _P]),
     "mt_forward": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
     "mt_forward_events": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, C.POINTER(_P), _P]),
+    "mt_forward_tokens": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P, C.POINTER(_P), _P]),
     "mt_forward_host": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
     "mt_poll_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "mt_plan_summary": (C.c_int, [_P, _U64, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32)]),
@@ -181,7 +183,7 @@ class MTModel:
         self.handle = _P()
         trunk = TrunkConfig(cfg.vocab_size, cfg.max_position, cfg.type_vocab, cfg.hidden, cfg.heads, cfg.ffn,
                             cfg.trunk_layers, cfg.ln_eps, 0)
-        tasks = (TaskConfig * cfg.n_tasks)(*[TaskConfig(t.fork_depth, t.branch_layers, t.num_classes)
+        tasks = (TaskConfig * cfg.n_tasks)(*[TaskConfig(t.fork_depth, t.branch_layers, t.num_classes, 1 if t.token_level else 0)
                                              for t in cfg.tasks])
         _check(lib().mt_create(C.byref(trunk), tasks, cfg.n_tasks, max_batch, max_seq, C.byref(self.handle)),
                "mt_create")
@@ -258,6 +260,16 @@ class MTModel:
         mask = self.full_mask() if task_mask is None else task_mask
         _check(lib().mt_forward(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
                                 _ptr(logits), _stream(stream)), "mt_forward", self.handle)
+
+    def forward_tokens(self, token_ids, segment_ids, lengths, logits, token_logits, task_mask: Optional[int] = None,
+                       stream=None) -> None:
+        """forward() for trees with token-level tasks: ``logits`` [B, total_classes] (or None) and
+        ``token_logits`` [B, S, total_token_classes] (or None), both fp32, written in place."""
+        batch, seq = token_ids.shape
+        mask = self.full_mask() if task_mask is None else task_mask
+        _check(lib().mt_forward_tokens(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
+                                       _ptr(logits), _ptr(token_logits), None, _stream(stream)),
+               "mt_forward_tokens", self.handle)
 
     def forward_events(self, token_ids, segment_ids, lengths, logits, task_events, task_mask: Optional[int] = None,
                        stream=None) -> None:

@@ -103,7 +103,8 @@ struct Chunk {
   std::vector<DumpCopy> dumps;
 };
 struct PlanStep {
-  int kind;  // 0 = chunk, 1 = heads, 2 = cls tail
+  int kind;  // 0 = chunk, 1 = heads, 2 = cls tail, 3 = token-level heads
+  TokenHeadParams token_heads;
   Chunk chunk;
   HeadParams heads;
   bool pool_gemm = false;           // heads step: the pooler runs as a grouped GEMM (`pool`), then the head kernel
@@ -179,7 +180,7 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
 struct mt_model {
   mt_trunk_config trunk;
   std::vector<TaskEntry> tasks;
-  int32_t max_batch, max_seq, c_total;
+  int32_t max_batch, max_seq, c_total, ct_total;  // columns of the sequence-level / of the token-level tasks
 
   // arena
   size_t emb_word, emb_pos, emb_type, emb_ln_g, emb_ln_b;
@@ -354,7 +355,8 @@ bool build_schedule(const mt_model* m, uint64_t mask, Schedule* s) {
   for (int32_t t = 0; t < T; ++t) {
     if (!((mask >> t) & 1)) continue;
     const mt_task_config& c = m->tasks[t].cfg;
-    const bool now = c.branch_layers == 0 || m->early_heads;
+    // (a token-level head reads every row of the final state and has no tail to share: it runs at once too)
+    const bool now = c.branch_layers == 0 || m->early_heads || c.head_kind == MT_HEAD_TOKEN;
     s->heads[now ? c.fork_depth + c.branch_layers : last_wave].push_back(t);
   }
   return true;
@@ -372,12 +374,13 @@ float* f32_of(const mt_model* m, bf16* state) {
 }
 
 // True when the final state of a task is [B, H], one row per sequence.
+bool is_token_task(const mt_model* m, int32_t task) { return m->tasks[task].cfg.head_kind == MT_HEAD_TOKEN; }
 bool is_compact_task(const mt_model* m, int32_t task) {
-  return m->cls_only && m->tasks[task].cfg.branch_layers > 0;
+  return m->cls_only && m->tasks[task].cfg.branch_layers > 0 && !is_token_task(m, task);
 }
 // True for the last layer of a task branch when only the first token's state is needed downstream.
 bool is_cls_op(const mt_model* m, const OpDesc& op) {
-  return m->cls_only && op.task >= 0 && op.layer == m->tasks[op.task].cfg.branch_layers;
+  return m->cls_only && op.task >= 0 && op.layer == m->tasks[op.task].cfg.branch_layers && !is_token_task(m, op.task);
 }
 
 // Whether a grouped GEMM launch of `groups` problems of `rows` (padded) rows runs as CTA pairs.  Pairs
@@ -709,9 +712,35 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       plan->launches += 2;
     }
   };
+  // Token-level tasks: one linear map on every valid token of the final state, written by position.
+  auto add_token_heads = [&](const std::vector<int32_t>& tasks) {
+    for (size_t first = 0; first < tasks.size(); first += kMaxGroups) {
+      const size_t count = std::min<size_t>(kMaxGroups, tasks.size() - first);
+      PlanStep st;
+      st.kind = 3;
+      memset(&st.heads, 0, sizeof(st.heads));
+      memset(&st.token_heads, 0, sizeof(st.token_heads));
+      TokenHeadParams& th = st.token_heads;
+      th.n_tasks = static_cast<int32_t>(count);
+      th.batch = batch; th.seq = seq; th.hidden = m->trunk.hidden;
+      th.logits_stride = m->ct_total;
+      th.row_start = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start);
+      for (size_t i = 0; i < count; ++i) {
+        const int32_t t = tasks[first + i];
+        const TaskEntry& te = m->tasks[t];
+        th.hidden_state[i] = te.cfg.branch_layers == 0 ? trunk_buf(m, te.cfg.fork_depth) : task_buf(m, t);
+        th.cls_w[i] = w_ptr(m, te.cls_w); th.cls_b[i] = w_ptr(m, te.cls_b);
+        th.num_classes[i] = te.cfg.num_classes; th.col0[i] = te.col0;
+        st.head_tasks.push_back(t);
+      }
+      plan->steps.push_back(std::move(st));
+      plan->launches += 1;
+    }
+  };
   auto add_heads = [&](const std::vector<int32_t>& tasks) {
-    std::vector<int32_t> compact, gathered;
-    for (int32_t t : tasks) (is_compact_task(m, t) ? compact : gathered).push_back(t);
+    std::vector<int32_t> compact, gathered, token;
+    for (int32_t t : tasks) (is_token_task(m, t) ? token : (is_compact_task(m, t) ? compact : gathered)).push_back(t);
+    add_token_heads(token);
     add_heads_of(gathered, false);
     add_heads_of(compact, true);
   };
@@ -771,7 +800,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   if (static_cast<int64_t>(max_batch) * max_seq > (int64_t(1) << 24)) return MT_ERR_SHAPE;
   for (int32_t t = 0; t < n_tasks; ++t) {
     if (tasks[t].fork_depth < 0 || tasks[t].fork_depth > trunk->trunk_layers || tasks[t].branch_layers < 0 ||
-        tasks[t].num_classes < 1)
+        tasks[t].num_classes < 1 || (tasks[t].head_kind != MT_HEAD_SEQUENCE && tasks[t].head_kind != MT_HEAD_TOKEN))
       return MT_ERR_INVALID_ARG;
   }
   mt_model* m = new mt_model();
@@ -811,7 +840,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->emb_ln_b = take(H);
   m->trunk_layers.resize(trunk->trunk_layers);
   for (int32_t l = 0; l < trunk->trunk_layers; ++l) off = place_layer(*trunk, off, &m->trunk_layers[l]);
-  int32_t col = 0;
+  int32_t col = 0, col_tok = 0;
   m->tasks.resize(n_tasks);
   for (int32_t t = 0; t < n_tasks; ++t) {
     TaskEntry& te = m->tasks[t];
@@ -824,12 +853,19 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
     te.cls_w = take(static_cast<size_t>(tasks[t].num_classes) * H);
     te.cls_b = take(tasks[t].num_classes);
     te.section_bytes = off - te.section_begin;
-    te.col0 = col;
-    col += tasks[t].num_classes;
+    // sequence-level and token-level tasks have output arrays, and column counts, of their own
+    if (tasks[t].head_kind == MT_HEAD_TOKEN) {
+      te.col0 = col_tok;
+      col_tok += tasks[t].num_classes;
+    } else {
+      te.col0 = col;
+      col += tasks[t].num_classes;
+    }
     te.loaded = false;
   }
   m->weights_bytes = off;
   m->c_total = col;
+  m->ct_total = col_tok;
   layout_workspace(m);
   *out = m;
   return MT_OK;
@@ -1048,10 +1084,14 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
       for (size_t first = 0; first < n_cls_tasks; first += kMaxGroups)
         n += tail_launches(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first)));
     }
-    size_t n_compact = 0;
-    for (int32_t t : s.heads[w]) n_compact += is_compact_task(m, t) ? 1 : 0;
+    size_t n_compact = 0, n_token = 0;
+    for (int32_t t : s.heads[w]) {
+      n_compact += is_compact_task(m, t) ? 1 : 0;
+      n_token += is_token_task(m, t) ? 1 : 0;
+    }
+    n += static_cast<int32_t>((n_token + kMaxGroups - 1) / kMaxGroups);
     n += 2 * static_cast<int32_t>((n_compact + kMaxGroups - 1) / kMaxGroups +
-                                  (s.heads[w].size() - n_compact + kMaxGroups - 1) / kMaxGroups);
+                                  (s.heads[w].size() - n_compact - n_token + kMaxGroups - 1) / kMaxGroups);
   }
   *n_launches = n;
   return MT_OK;
@@ -1065,9 +1105,23 @@ int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment
 int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
                       uint64_t task_mask, int32_t batch, int32_t seq, float* d_logits, void* const* task_events,
                       void* stream_) {
+  return mt_forward_tokens(m, d_token_ids, d_segment_ids, d_lengths, task_mask, batch, seq, d_logits, nullptr, task_events,
+                           stream_);
+}
+
+int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
+                      uint64_t task_mask, int32_t batch, int32_t seq, float* d_logits, float* d_token_logits,
+                      void* const* task_events, void* stream_) {
   if (m == nullptr) return MT_ERR_INVALID_ARG;
-  if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr || d_logits == nullptr)
-    return fail(m, MT_ERR_INVALID_ARG, "null input or output pointer");
+  if (d_token_ids == nullptr || d_segment_ids == nullptr || d_lengths == nullptr)
+    return fail(m, MT_ERR_INVALID_ARG, "null input pointer");
+  for (size_t t = 0; t < m->tasks.size(); ++t) {
+    if (!((task_mask >> t) & 1)) continue;
+    const bool token = m->tasks[t].cfg.head_kind == MT_HEAD_TOKEN;
+    if (token && d_token_logits == nullptr)
+      return fail(m, MT_ERR_INVALID_ARG, "a token-level task is active: its logits need d_token_logits (mt_forward_tokens)");
+    if (!token && d_logits == nullptr) return fail(m, MT_ERR_INVALID_ARG, "null output pointer");
+  }
   if (batch < 1 || seq < 1) return fail(m, MT_ERR_INVALID_ARG, "batch and seq must be positive");
   if (batch > m->max_batch || seq > m->max_seq) return fail(m, MT_ERR_SHAPE, "batch/seq beyond the limits of mt_create");
   if (m->d_workspace == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
@@ -1180,11 +1234,16 @@ int mt_forward_events(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
                                   stream),
                   "debug capture");
     } else {
-      st.heads.logits = d_logits;
-      if (st.pool_gemm) {
+      if (st.kind == 3) {
+        st.token_heads.logits = d_token_logits;
+        st.token_heads.lengths = d_lengths;
+        MT_TIMED(MT_CLASS_HEAD, launch_token_heads(st.token_heads, stream), "token-level head kernel");
+      } else if (st.pool_gemm) {
+        st.heads.logits = d_logits;
         MT_TIMED(MT_CLASS_HEAD, launch_gemm(st.pool, kEpiBiasTanhF32, m->sm_count, stream), "pooler GEMM");
         MT_TIMED(MT_CLASS_HEAD, launch_head(st.heads, stream), "head kernel");
       } else {
+        st.heads.logits = d_logits;
         MT_TIMED(MT_CLASS_HEAD, launch_pooler_head(st.heads, stream), "pooler/head kernel");
       }
       if (task_events != nullptr)

@@ -221,6 +221,20 @@ struct HeadParams {
   int32_t n_tasks, batch, seq, hidden, logits_stride;
 };
 
+// Token-level heads: logits[(b * seq + pos) * logits_stride + col0_t + c] = cls_w_t[c, :] . h_t[row(b, pos), :] + cls_b_t[c]
+// for every valid position of every sequence; positions >= length are not written.
+struct TokenHeadParams {
+  const bf16* hidden_state[kMaxGroups];  // final state of the task, [rows, H]
+  const bf16* cls_w[kMaxGroups];
+  const bf16* cls_b[kMaxGroups];
+  int32_t num_classes[kMaxGroups], col0[kMaxGroups];
+  float* logits;             // fp32 [batch, seq, logits_stride]
+  const int32_t* lengths;
+  const int32_t* row_start;  // [B + 1] or null (padded layout)
+  int32_t n_tasks, batch, seq, hidden, logits_stride;
+};
+cudaError_t launch_token_heads(const TokenHeadParams& p, cudaStream_t stream);
+
 // row_start[b] for b = 0..batch and *rows_valid = row_start[batch]: b * seq (padded) or the running sum
 // of the lengths clamped to [1, seq] (packed).
 cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,

@@ -240,6 +240,50 @@ cudaError_t launch_unpack_rows(const bf16* packed, const int32_t* lengths, const
   return cudaGetLastError();
 }
 
+// Token-level heads: one warp per (task, sequence, position); the token's state is read once (16-byte
+// loads, held in registers as fp32) and dotted with every class row of the head matrix, which stays in
+// L1/L2; fp32 throughout.  HBM-bound on the states: 2 H bytes per token and task.
+template <int V>
+__global__ void __launch_bounds__(kRowThreads) token_head_kernel(const TokenHeadParams p) {
+  constexpr int H = V * 256;
+  const int lane = threadIdx.x & 31;
+  const int pos = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+  const int b = blockIdx.y, t = blockIdx.z;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  int len = p.lengths[b];
+  len = len < 1 ? 1 : (len > p.seq ? p.seq : len);
+  if (pos >= len) return;
+  const size_t row = p.row_start != nullptr ? static_cast<size_t>(p.row_start[b]) + pos : static_cast<size_t>(b) * p.seq + pos;
+  const bf16* h = p.hidden_state[t] + row * H;
+  float x[V][8];
+#pragma unroll
+  for (int v = 0; v < V; ++v) unpack8(*reinterpret_cast<const uint4*>(h + (v * 32 + lane) * 8), x[v]);
+  float* out = p.logits + (static_cast<size_t>(b) * p.seq + pos) * p.logits_stride + p.col0[t];
+  for (int c = 0; c < p.num_classes[t]; ++c) {
+    const bf16* wrow = p.cls_w[t] + static_cast<size_t>(c) * H;
+    float acc = 0.f;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      float w[8];
+      unpack8(__ldg(reinterpret_cast<const uint4*>(wrow + (v * 32 + lane) * 8)), w);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc = fmaf(x[v][i], w[i], acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) out[c] = acc + __bfloat162float(p.cls_b[t][c]);
+  }
+}
+
+cudaError_t launch_token_heads(const TokenHeadParams& p, cudaStream_t stream) {
+  if (p.n_tasks < 1 || p.n_tasks > kMaxGroups || p.batch < 1 || p.seq < 1 || p.logits == nullptr || p.lengths == nullptr)
+    return cudaErrorInvalidValue;
+  dim3 grid((p.seq + kRowThreads / 32 - 1) / (kRowThreads / 32), p.batch, p.n_tasks);
+  if (p.hidden == 768) return launch_kernel(token_head_kernel<3>, grid, dim3(kRowThreads), 0, stream, p);
+  if (p.hidden == 1024) return launch_kernel(token_head_kernel<4>, grid, dim3(kRowThreads), 0, stream, p);
+  return cudaErrorInvalidValue;
+}
+
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1) return cudaErrorInvalidValue;
   dim3 grid((p.rows + kRowThreads / 32 - 1) / (kRowThreads / 32), p.n_groups);

@@ -32,11 +32,13 @@ import numpy as np
 class TaskSpec:
     """One task of the tree: forks after trunk layer ``fork_depth`` (0 = the
     embedding output), runs ``branch_layers`` task-specific layers, and ends in
-    a pooler plus a linear head with ``num_classes`` outputs."""
+    a pooler plus a linear head with ``num_classes`` outputs - or, with
+    ``token_level``, in a linear head applied to every token's final state."""
 
     fork_depth: int
     branch_layers: int
     num_classes: int
+    token_level: bool = False
 
 
 @dataclass(frozen=True)
@@ -57,15 +59,25 @@ class TreeConfig:
 
     @property
     def logit_offsets(self) -> List[int]:
-        offs, acc = [], 0
+        """First column of every task in its output array: sequence-level tasks are counted among
+        themselves ([B, total_classes]), token-level tasks among themselves ([B, S, total_token_classes])."""
+        offs, acc, acc_tok = [], 0, 0
         for t in self.tasks:
-            offs.append(acc)
-            acc += t.num_classes
+            if t.token_level:
+                offs.append(acc_tok)
+                acc_tok += t.num_classes
+            else:
+                offs.append(acc)
+                acc += t.num_classes
         return offs
 
     @property
     def total_classes(self) -> int:
-        return sum(t.num_classes for t in self.tasks)
+        return sum(t.num_classes for t in self.tasks if not t.token_level)
+
+    @property
+    def total_token_classes(self) -> int:
+        return sum(t.num_classes for t in self.tasks if t.token_level)
 
 
 def _tasks(depths: Sequence[int], branches: Sequence[int], classes: Sequence[int]) -> Tuple[TaskSpec, ...]:

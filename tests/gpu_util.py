@@ -39,7 +39,8 @@ def cached_weights(cfg, seed=0, random_affine=False):
 
 
 def task_triples(cfg):
-    return [(t.fork_depth, t.branch_layers, t.num_classes) for t in cfg.tasks]
+    """Task tuples for the oracle; token-level tasks carry their head kind as a fourth entry."""
+    return [(t.fork_depth, t.branch_layers, t.num_classes) + ((1,) if t.token_level else ()) for t in cfg.tasks]
 
 
 def dev_batch(batch):

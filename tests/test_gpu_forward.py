@@ -486,3 +486,54 @@ def test_large_width_tree_sampled_rows():
     batch = synth.make_batch(cfg, 8, 128, 32, 128, seed=1)
     model, logits = run_model(cfg, blob, batch, debug=True)
     check_against_oracle(cfg, wf, batch, model, logits, rows=[0, 5])
+
+
+def test_token_level_heads_match_oracle_and_standalone_bits():
+    """A tree that mixes sequence-level and token-level tasks (mt_forward_tokens): both kinds of logits
+    against the oracle, nothing written at positions >= length or in columns of inactive tasks, the
+    token-level task alone (its stand-alone student) gives the same bits, and mt_forward refuses a mask
+    that needs the token output."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 5, token_level=True),
+                                                  synth.TaskSpec(3, 0, 3, token_level=True), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 7, random_affine=True)
+    for S, lo in ((72, 1), (150, 30)):
+        batch = synth.make_batch(cfg, 5, S, lo, S, seed=11)
+        B = 5
+        model = mt.MTModel(cfg, B, S)
+        model.load_weights(blob)
+        tok, seg, lens = dev_batch(batch)
+        logits = torch.full((B, cfg.total_classes), float("nan"), device="cuda")
+        tlog = torch.full((B, S, cfg.total_token_classes), float("nan"), device="cuda")
+        model.forward_tokens(tok, seg, lens, logits, tlog)
+        torch.cuda.synchronize()
+        assert model.poll_status() == 0
+        tl = []
+        want = orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, wf, task_triples(cfg), cfg.heads,
+                                    cfg.ln_eps, token_logits_out=tl)
+        got = logits.cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(got - want)) <= LOGIT_MAX_ABS
+        got_t = tlog.cpu().numpy().astype(np.float64)
+        valid = np.arange(S)[None, :] < batch.lengths[:, None]
+        assert np.all(np.isnan(got_t[~valid])) and np.all(np.isfinite(got_t[valid]))
+        assert np.array_equal(np.isnan(tl[0]), np.isnan(got_t))
+        assert np.max(np.abs(got_t[valid] - tl[0][valid])) <= LOGIT_MAX_ABS
+        assert rel_l2(got_t[valid], tl[0][valid]) <= HIDDEN_REL_L2
+        # one token-level task alone: same bits in its columns, the others untouched
+        alone = torch.full_like(tlog, float("nan"))
+        model.forward_tokens(tok, seg, lens, None, alone, task_mask=0b0010)
+        torch.cuda.synchronize()
+        assert torch.equal(alone[..., :5][torch.from_numpy(valid).cuda()], tlog[..., :5][torch.from_numpy(valid).cuda()])
+        assert torch.isnan(alone[..., 5:]).all()
+        st_cfg = synth.TreeConfig(trunk_layers=3, tasks=(cfg.tasks[1],))
+        st = mt.MTModel(st_cfg, B, S)
+        st_w = {"emb": w["emb"], "trunk": w["trunk"], "tasks": [w["tasks"][1]]}
+        st.load_weights(synth.pack_weights(st_cfg, st_w))
+        st_out = torch.full((B, S, 5), float("nan"), device="cuda")
+        st.forward_tokens(tok, seg, lens, None, st_out)
+        torch.cuda.synchronize()
+        assert torch.equal(st_out[torch.from_numpy(valid).cuda()], tlog[..., :5][torch.from_numpy(valid).cuda()])
+        with pytest.raises(mt.MTError):
+            model.forward(tok, seg, lens, logits)          # the mask holds token-level tasks: no place for their output
+        model.forward(tok, seg, lens, logits, task_mask=0b1001)   # sequence-level tasks only: fine
+        torch.cuda.synchronize()
+        assert np.max(np.abs(logits.cpu().numpy().astype(np.float64) - want)) <= LOGIT_MAX_ABS

@@ -108,6 +108,27 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     m2.close()
 
 
+def test_token_level_tasks_in_the_plan(lib):
+    """A token-level task needs every row of its last layer (no first-token shortcut) and gets its head,
+    one launch, right after the wave that completes it; sequence-level tasks are planned as before."""
+    seq_only = small_cfg([(2, 2, 2), (1, 1, 3)], trunk_layers=2)
+    mixed = synth.TreeConfig(trunk_layers=2, tasks=(synth.TaskSpec(2, 2, 2), synth.TaskSpec(1, 1, 3, token_level=True)))
+    assert mixed.total_classes == 2 and mixed.total_token_classes == 3 and mixed.logit_offsets == [0, 0]
+    a = binding.MTModel(seq_only, 2, 32, bind=False)
+    b = binding.MTModel(mixed, 2, 32, bind=False)
+    for m in (a, b):
+        m.set_option("fused_ln", 0)
+    assert a.plan_summary(0b11) == b.plan_summary(0b11)
+    # wave 1: trunk (7); wave 2: trunk + the last layer of task 1: first tokens only (7 + first-token attention),
+    # or all tokens for the token-level task (7, two groups); wave 3, 4: task 0 (7, then projection + first-token
+    # attention); first-token tails: 5 per tail launch; heads: pooler GEMM + head = 2, token-level head = 1
+    assert a.plan_launches(0b11) == 2 + 7 + 8 + 7 + 2 + 5 + 2
+    assert b.plan_launches(0b11) == 2 + 7 + 7 + 1 + 7 + 2 + 5 + 2
+    assert b.plan_launches(0b10) == 2 + 7 + 7 + 1
+    a.close()
+    b.close()
+
+
 def test_create_rejects_bad_configurations(lib):
     def create(trunk_kw=None, tasks=((4, 1, 2),), max_batch=2, max_seq=32):
         kw = dict(vocab_size=64, max_position=64, type_vocab=2, hidden=768, heads=12, ffn=3072, trunk_layers=4,
@@ -126,6 +147,8 @@ def test_create_rejects_bad_configurations(lib):
     assert create(tasks=((4, -1, 2),)) == -1
     assert create(tasks=((4, 1, 0),)) == -1
     assert create(tasks=((0, 0, 1),)) == 0              # fork at the embeddings, no branch, regression head
+    assert create(tasks=((4, 1, 5, 1),)) == 0           # token-level head
+    assert create(tasks=((4, 1, 5, 2),)) == -1          # unknown head kind
     assert create({"hidden": 512, "heads": 8}) == -7    # width not implemented
     assert create({"heads": 8}) == -7                   # head width != 64
     assert create({"activation": 1}) == -7
