@@ -8,8 +8,9 @@ One JSON line per case:
     fork), eagerly launched and replayed from a CUDA graph;
   * eight independent full-depth (12-layer) single-task models over the same inputs, through the same
     library, to reproduce the paper's sharing saving (Table 2: 96 layers against the merged tree's 24);
-  * the long-sequence variant (16 x 512, lengths in [128, 512]) and the BERT-large-width tree
-    (64 x 128, lengths in [32, 128]).
+  * the long-sequence variant (16 x 512, lengths in [128, 512]), the BERT-large-width tree
+    (64 x 128, lengths in [32, 128]) and a 21-task tree shaped like the production model of Appendix E
+    (8 shared + 32 task layers, a third of the tasks token-level; 32 x 128, lengths in [16, 128]).
 Weights are seeded random (timing does not depend on their values; the eight single-task models are
 loaded from one blob into eight separate arenas).  Inputs are resident on the device.
 """
@@ -63,10 +64,12 @@ def run_tree(name, cfg, blob, batch, masks, iters, out):
     model = binding.MTModel(cfg, B, S)
     model.load_weights(blob)
     tok, seg, lens = _dev(batch)
-    logits = torch.zeros(B, cfg.total_classes, dtype=torch.float32, device="cuda")
+    logits = torch.zeros(B, max(cfg.total_classes, 1), dtype=torch.float32, device="cuda")
+    token_logits = torch.zeros(B, S, cfg.total_token_classes, dtype=torch.float32, device="cuda") \
+        if cfg.total_token_classes > 0 else None
     for label, mask in masks:
         plan = model.plan_summary(mask)
-        fn = lambda: model.forward(tok, seg, lens, logits, task_mask=mask)  # noqa: E731
+        fn = lambda: model.forward_tokens(tok, seg, lens, logits, token_logits, task_mask=mask)  # noqa: E731
         eager = _time_ms(fn, iters, False)
         graph = _time_ms(fn, iters, True)
         assert model.poll_status() == 0
@@ -157,6 +160,13 @@ def main():
         big_blob = synth.pack_weights(big, synth.make_weights(big, seed=0))
         run_tree("large-width tree", big, big_blob, synth.make_batch(big, 64, 128, 32, 128, seed=1),
                  [("all 8", 0xFF)], 20, out)
+        del big_blob
+        prod = synth.config_production21()
+        prod_blob = synth.pack_weights(prod, synth.make_weights(prod, seed=0))
+        seq_only = sum(1 << t for t, spec in enumerate(prod.tasks) if not spec.token_level)
+        run_tree("production-shaped tree (21 tasks, 7 token-level)", prod, prod_blob,
+                 synth.make_batch(prod, 32, 128, 16, 128, seed=1),
+                 [("all 21", (1 << 21) - 1), ("the 14 sequence-level tasks", seq_only)], 20, out)
 
 
 if __name__ == "__main__":

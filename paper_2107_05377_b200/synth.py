@@ -102,6 +102,16 @@ def config_large8() -> TreeConfig:
                       tasks=_tasks([18, 17, 16, 15, 14, 13, 12, 16], [2] * 8, [2, 2, 2, 3, 2, 2, 2, 3]))
 
 
+def config_production21() -> TreeConfig:
+    """Shaped like the production model of Appendix E: 21 tasks on a BERT-base trunk, 8 shared layers and
+    32 task layers in all (eleven branches of 2 layers, ten of 1).  Every third task is token-level (9
+    tags, as a slot-filling or entity task would have), the others are sequence-level with 2-4 classes."""
+    branches = [2 if t % 2 == 0 else 1 for t in range(21)]
+    classes = [9 if t % 3 == 2 else 2 + t % 3 for t in range(21)]
+    tasks = tuple(TaskSpec(8, branches[t], classes[t], token_level=(t % 3 == 2)) for t in range(21))
+    return TreeConfig(tasks=tasks)
+
+
 def config_single_task(base: TreeConfig, task: int) -> TreeConfig:
     """The stand-alone single-task model of ``task``: same trunk prefix, its
     branch alone (Fig. 1(b): one student before merging)."""
