@@ -187,7 +187,7 @@ int mt_poll_status(mt_model* m, void* stream, uint32_t* flags);
  * otherwise room for trunk_layers + max branch_layers + 1 ints). */
 int mt_plan_summary(const mt_model* m, uint64_t task_mask, int32_t* n_layers, int32_t* n_waves,
                     int32_t* trunk_depth, int32_t* groups_per_wave);
-/* Kernel launches one mt_forward enqueues for this mask (after its plan exists). */
+/* Kernel launches one mt_forward at batch = max_batch, seq = max_seq enqueues for this mask. */
 int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches);
 
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
@@ -216,8 +216,8 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * device can make those waits run out (status flag MT_FLAG_WAIT_TIMEOUT) - serialise them, or set 0.
  * keys "tail_bn0", "tail_bn1", "tail_bn2" (0 = automatic, 128, 192; any time): tile widths of the three
  * GEMMs of that launch; they never change a result.
- * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 1) layers,
- * the default; any time): the attention-output and FFN-down projections carry the LayerNorm that follows
+ * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 2) layers
+ * and for launches of at most "fused_ln_max_rows" (default 0) rows per layer, the default; any time): the attention-output and FFN-down projections carry the LayerNorm that follows
  * them: the CTAs holding the column blocks of the same 128 rows form a thread-block cluster and exchange
  * per-row statistics through distributed shared memory, so the pre-normalisation sum never goes to global
  * memory and no LayerNorm launch follows.  Results agree with the separate launches to fp32 rounding of

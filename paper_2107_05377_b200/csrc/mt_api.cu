@@ -203,6 +203,7 @@ struct mt_model {
   int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always,
                      // 2 for launches of at most fused_ln_max_groups layers
   int32_t fused_ln_max_groups;
+  int32_t fused_ln_max_rows;
   bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
   int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
@@ -410,14 +411,16 @@ bool use_fused_tail(const mt_model* m, int32_t groups) {
 }
 
 // Whether the residual GEMMs of `groups` layers carry their LayerNorm (see GemmLnParams).
-bool use_fused_ln(const mt_model* m, int32_t groups) {
+// (mode 2: few layers in the launch; optionally also launches of few rows per layer, the first-token tails,
+// which measured 0.3 % slower that way on the 32 x 128 batch; all ways give the same bits)
+bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) {
   if (groups < 1 || !gemm_ln_supported(m->trunk.hidden) || m->fused_ln == 0) return false;
-  return m->fused_ln == 1 || groups <= m->fused_ln_max_groups;
+  return m->fused_ln == 1 || groups <= m->fused_ln_max_groups || rows <= m->fused_ln_max_rows;
 }
 // Launches of steps 3-7 for `groups` layers.
-int32_t tail_launches(const mt_model* m, int32_t groups) {
+int32_t tail_launches(const mt_model* m, int32_t groups, int64_t rows) {
   if (use_fused_tail(m, groups)) return 1;
-  return use_fused_ln(m, groups) ? 3 : 5;
+  return use_fused_ln(m, groups, rows) ? 3 : 5;
 }
 
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
@@ -443,7 +446,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
   t->fused = use_fused_tail(m, groups);
-  t->ln_fused = !t->fused && use_fused_ln(m, groups);
+  t->ln_fused = !t->fused && use_fused_ln(m, groups, rows);
   if (t->ln_fused) {
     auto init_ln = [&](GemmLnParams* g, int32_t K) {
       memset(g, 0, sizeof(*g));
@@ -634,10 +637,10 @@ cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks,
   return cudaSuccess;
 }
 
-int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count) {
+int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int64_t rows) {
   size_t n_cls = 0;
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
-  return 1 + (n_cls < count ? 1 + tail_launches(m, static_cast<int32_t>(count - n_cls)) : 0) + (n_cls > 0 ? 1 : 0);
+  return 1 + (n_cls < count ? 1 + tail_launches(m, static_cast<int32_t>(count - n_cls), rows) : 0) + (n_cls > 0 ? 1 : 0);
 }
 // Active tasks whose last branch layer is finished on first tokens right after wave w (1-based):
 // those whose last layer is in wave w with option early_heads, otherwise all of them after the last wave.
@@ -755,7 +758,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       if (e != cudaSuccess) return e;
       if ((e = assign_sync(&st.chunk.full)) != cudaSuccess) return e;
       plan->steps.push_back(std::move(st));
-      plan->launches += chunk_launches(m, ops, first, count);
+      plan->launches += chunk_launches(m, ops, first, count, static_cast<int64_t>(batch) * seq);
     }
     {
       // first-token tails: of the tasks finishing in this wave (early_heads), or of all tasks after the last wave
@@ -766,7 +769,7 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         cudaError_t e = build_cls_tail(m, tasks, first, std::min<size_t>(kMaxGroups, tasks.size() - first), batch, &st);
         if (e != cudaSuccess) return e;
         if ((e = assign_sync(&st.tail)) != cudaSuccess) return e;
-        plan->launches += tail_launches(m, st.tail.count);
+        plan->launches += tail_launches(m, st.tail.count, batch);
         plan->steps.push_back(std::move(st));
       }
     }
@@ -818,7 +821,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->fused_tail = 0;
   m->pool_gemm = true;
   m->fused_ln = 2;
-  m->fused_ln_max_groups = 1;
+  m->fused_ln_max_groups = 2;
+  m->fused_ln_max_rows = 0;
   m->fused_min_groups = 3;
   m->tail_bn[0] = m->tail_bn[1] = m->tail_bn[2] = 0;
   m->last_lengths = nullptr;
@@ -910,6 +914,12 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "fused_ln") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1 or 2");
     m->fused_ln = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "fused_ln_max_rows") == 0) {
+    if (value < 0) return fail(m, MT_ERR_INVALID_ARG, "fused_ln_max_rows must be >= 0");
+    m->fused_ln_max_rows = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
   }
@@ -1079,10 +1089,11 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
     if (w >= 1) {
       const std::vector<OpDesc>& ops = s.waves[w - 1];
       for (size_t first = 0; first < ops.size(); first += m->n_slots)
-        n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first));
+        n += chunk_launches(m, ops, first, std::min<size_t>(m->n_slots, ops.size() - first),
+                            static_cast<int64_t>(m->max_batch) * m->max_seq);
       const size_t n_cls_tasks = cls_tasks_after_wave(m, s, w).size();
       for (size_t first = 0; first < n_cls_tasks; first += kMaxGroups)
-        n += tail_launches(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first)));
+        n += tail_launches(m, static_cast<int32_t>(std::min<size_t>(kMaxGroups, n_cls_tasks - first)), m->max_batch);
     }
     size_t n_compact = 0, n_token = 0;
     for (int32_t t : s.heads[w]) {

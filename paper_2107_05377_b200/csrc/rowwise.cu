@@ -164,9 +164,19 @@ __global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) 
   grid_launch_dependents();
   for (int o = warp; o < tk.num_classes * nb; o += kHeadThreads / 32) {
     const int c = o / nb, s = o - c * nb;
+    // eight consecutive columns per lane and step (H is a multiple of 256): every load of the dot
+    // product is independent of the others, so they are all in flight together
+    const bf16* wrow = tk.cls_w + static_cast<size_t>(c) * H;
+    const float* prow = pooled + static_cast<size_t>(b0 + s) * H;
     float acc = 0.f;
-    for (int k = lane; k < H; k += 32)
-      acc += __bfloat162float(tk.cls_w[static_cast<size_t>(c) * H + k]) * pooled[static_cast<size_t>(b0 + s) * H + k];
+    for (int k = lane * 8; k < H; k += 256) {
+      float w[8];
+      unpack8(__ldg(reinterpret_cast<const uint4*>(wrow + k)), w);
+      const float4 p0 = *reinterpret_cast<const float4*>(prow + k);
+      const float4 p1 = *reinterpret_cast<const float4*>(prow + k + 4);
+      acc = fmaf(w[0], p0.x, acc); acc = fmaf(w[1], p0.y, acc); acc = fmaf(w[2], p0.z, acc); acc = fmaf(w[3], p0.w, acc);
+      acc = fmaf(w[4], p1.x, acc); acc = fmaf(w[5], p1.y, acc); acc = fmaf(w[6], p1.z, acc); acc = fmaf(w[7], p1.w, acc);
+    }
     acc = warp_sum(acc);
     if (lane == 0)
       p.logits[static_cast<size_t>(b0 + s) * p.logits_stride + tk.col0 + c] = acc + __bfloat162float(tk.cls_b[c]);

@@ -75,9 +75,11 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     # (projection, attention, output + LN, FFN up, FFN down + LN), a first-token tail 3
     m.set_option("fused_ln", 1)
     assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 3 + 2
-    # default (2): only where a single layer is on all tokens: waves 1-4 and wave 9
+    # default (2): where at most two layers are on all tokens: waves 1-5 and wave 9
     m.set_option("fused_ln", 2)
-    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 7 + 7 + 8 + 8 + 6 + 2 + 5 + 2
+    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 5 + 2
+    m.set_option("fused_ln_max_rows", 128)   # also the first-token tail (32 rows per layer)
+    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 3 + 2
     m.set_option("fused_ln", 0)
     # fused_tail = 1: the part of a layer after attention is one launch, so a wave is projection + attention
     # + fused tail (+ first-token attention where a branch ends); one fused first-token tail; pooler + head
