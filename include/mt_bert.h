@@ -122,6 +122,16 @@ int mt_load_weights(mt_model* m, const void* host_blob, size_t bytes, void* stre
  * replaces the branch layers, pooler and head of one task; nothing else in the arena is touched. */
 int mt_load_task_weights(mt_model* m, int32_t task, const void* host_blob, size_t bytes, void* stream);
 
+/* Several models over ONE weights arena: a server that keeps more than one batch in flight (one model and
+ * one stream per batch in flight; the kernels of independent forwards fill one another's ramps and tails,
+ * +11 % sequences/s with two at batch 32 x seq 128) needs a workspace per model but the weights only
+ * once.  Create the second model from the same configuration, bind it with the FIRST model's d_weights
+ * and a workspace of its own, then call this instead of mt_load_weights: it marks as loaded whatever
+ * `src` has loaded.  Later mt_load_weights / mt_load_task_weights on either model write the shared
+ * arena; repeat the call on the other one.  Errors: NOT_BOUND, INVALID_ARG (different arenas),
+ * BLOB_MISMATCH (different configurations). */
+int mt_adopt_weights(mt_model* m, const mt_model* src);
+
 /* ---- the hot path ---------------------------------------------------------------------------- */
 
 /* Merged multi-task forward of one padded batch.
@@ -216,6 +226,8 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * device can make those waits run out (status flag MT_FLAG_WAIT_TIMEOUT) - serialise them, or set 0.
  * keys "tail_bn0", "tail_bn1", "tail_bn2" (0 = automatic, 128, 192; any time): tile widths of the three
  * GEMMs of that launch; they never change a result.
+ * key "sm_limit" (>= 0, default 0 = all; any time): size the persistent GEMM grids for at most this many SMs
+ * (for callers that share the GPU between several streams and want to leave room; measured no gain).
  * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 2) layers
  * and for launches of at most "fused_ln_max_rows" (default 0) rows per layer, the default; any time): the attention-output and FFN-down projections carry the LayerNorm that follows
  * them: the CTAs holding the column blocks of the same 128 rows form a thread-block cluster and exchange

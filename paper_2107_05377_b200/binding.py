@@ -43,6 +43,7 @@ SIGNATURES = {
     "mt_blob_bytes": (_SZ, [_P]),
     "mt_task_blob_bytes": (_SZ, [_P, _I32]),
     "mt_load_weights": (C.c_int, [_P, _P, _SZ, _P]),
+    "mt_adopt_weights": (C.c_int, [_P, _P]),
     "mt_load_task_weights": (C.c_int, [_P, _I32, _P, _SZ, _P]),
     "mt_forward": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
     "mt_forward_events": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, C.POINTER(_P), _P]),
@@ -177,7 +178,10 @@ class MTModel:
     """mt_create + mt_bind_memory + mt_load_weights + mt_forward around torch-owned memory."""
 
     def __init__(self, cfg, max_batch: int, max_seq: int, max_groups: Optional[int] = None,
-                 debug_capture: bool = False, device: str = "cuda:0", bind: bool = True):
+                 debug_capture: bool = False, device: str = "cuda:0", bind: bool = True, share_weights_with=None):
+        """``share_weights_with``: another MTModel of the same configuration whose weights arena this one
+        uses too (mt_adopt_weights) - a second batch in flight needs a workspace of its own, not a second
+        copy of the weights."""
         self.cfg = cfg
         self.max_batch, self.max_seq = max_batch, max_seq
         self.handle = _P()
@@ -193,8 +197,11 @@ class MTModel:
             self.set_option("debug_capture", 1)
         self.c_total = cfg.total_classes
         self.weights = self.workspace = None
+        self._shared_from = share_weights_with
         if bind:
             self.bind(device)
+            if share_weights_with is not None:
+                _check(lib().mt_adopt_weights(self.handle, share_weights_with.handle), "mt_adopt_weights", self.handle)
 
     # -- host-only ----------------------------------------------------------
     def set_option(self, key: str, value: int) -> None:
@@ -231,7 +238,8 @@ class MTModel:
         import torch
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
-        self.weights = torch.empty(self.weights_bytes(), dtype=torch.uint8, device=self.device)
+        self.weights = self._shared_from.weights if self._shared_from is not None else \
+            torch.empty(self.weights_bytes(), dtype=torch.uint8, device=self.device)
         self.workspace = torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
         _check(lib().mt_bind_memory(self.handle, self.weights.data_ptr(), self.weights.numel(),
                                     self.workspace.data_ptr(), self.workspace.numel()), "mt_bind_memory", self.handle)

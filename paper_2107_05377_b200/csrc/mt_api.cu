@@ -211,7 +211,8 @@ struct mt_model {
   uint8_t* d_weights;
   uint8_t* d_workspace;
   size_t ws_bytes_bound;
-  int sm_count;
+  int sm_count;    // SMs the persistent GEMM grids are sized for: all of the device's, or option "sm_limit"
+  int sm_device, sm_limit;
 
   // workspace layout (byte offsets)
   size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
@@ -829,6 +830,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
   m->sm_count = 0;
+  m->sm_device = 0;
+  m->sm_limit = 0;
   m->trunk_loaded = false;
   m->last_batch = m->last_seq = 0;
   m->profile = false;
@@ -914,6 +917,13 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "fused_ln") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1 or 2");
     m->fused_ln = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "sm_limit") == 0) {
+    if (value < 0) return fail(m, MT_ERR_INVALID_ARG, "sm_limit must be >= 0");
+    m->sm_limit = static_cast<int>(value);
+    if (m->sm_device > 0) m->sm_count = (m->sm_limit > 0 && m->sm_limit < m->sm_device) ? m->sm_limit : m->sm_device;
     m->plans.clear();
     return MT_OK;
   }
@@ -1005,7 +1015,8 @@ int mt_bind_memory(mt_model* m, void* d_weights, size_t weights_bytes, void* d_w
   e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
   if (e != cudaSuccess) return fail_cuda(m, e, "querying the device");
   if (major != 10) return fail(m, MT_ERR_UNSUPPORTED, "the kernels are built for sm_100a only");
-  m->sm_count = sms;
+  m->sm_device = sms;
+  m->sm_count = (m->sm_limit > 0 && m->sm_limit < sms) ? m->sm_limit : sms;
   m->d_weights = static_cast<uint8_t*>(d_weights);
   m->d_workspace = static_cast<uint8_t*>(d_workspace);
   m->ws_bytes_bound = workspace_bytes;
@@ -1050,6 +1061,20 @@ int mt_load_weights(mt_model* m, const void* host_blob, size_t bytes, void* stre
   if (e != cudaSuccess) return fail_cuda(m, e, "copying weights");
   m->trunk_loaded = true;
   for (TaskEntry& t : m->tasks) t.loaded = true;
+  return MT_OK;
+}
+
+int mt_adopt_weights(mt_model* m, const mt_model* src) {
+  if (m == nullptr || src == nullptr) return MT_ERR_INVALID_ARG;
+  if (m->d_weights == nullptr || src->d_weights == nullptr) return fail(m, MT_ERR_NOT_BOUND, "both models must be bound");
+  if (m->d_weights != src->d_weights) return fail(m, MT_ERR_INVALID_ARG, "the two models are bound to different weight arenas");
+  bool same = m->weights_bytes == src->weights_bytes && m->tasks.size() == src->tasks.size() &&
+              memcmp(&m->trunk, &src->trunk, sizeof(m->trunk)) == 0;
+  for (size_t t = 0; same && t < m->tasks.size(); ++t)
+    same = memcmp(&m->tasks[t].cfg, &src->tasks[t].cfg, sizeof(mt_task_config)) == 0;
+  if (!same) return fail(m, MT_ERR_BLOB_MISMATCH, "the two models were created from different configurations");
+  m->trunk_loaded = src->trunk_loaded;
+  for (size_t t = 0; t < m->tasks.size(); ++t) m->tasks[t].loaded = src->tasks[t].loaded;
   return MT_OK;
 }
 

@@ -537,3 +537,37 @@ def test_token_level_heads_match_oracle_and_standalone_bits():
         model.forward(tok, seg, lens, logits, task_mask=0b1001)   # sequence-level tasks only: fine
         torch.cuda.synchronize()
         assert np.max(np.abs(logits.cpu().numpy().astype(np.float64) - want)) <= LOGIT_MAX_ABS
+
+
+def test_two_batches_in_flight_over_one_weights_arena():
+    """A second model created from the same configuration adopts the first one's weights arena
+    (mt_adopt_weights) and runs on a stream of its own: forwards of different batches issued alternately
+    on the two streams give the bits of the same forwards issued one after the other on one model."""
+    cfg = synth.config_glue8()
+    w8, blob8, _ = cached_weights(cfg, 0)
+    B, S = 16, 128
+    batches = [synth.make_batch(cfg, B, S, 16, 128, seed=40 + i) for i in range(4)]
+    first = mt.MTModel(cfg, B, S)
+    first.load_weights(blob8)
+    second = mt.MTModel(cfg, B, S, share_weights_with=first)
+    assert second.weights.data_ptr() == first.weights.data_ptr()
+    dev = [dev_batch(b) for b in batches]
+    want = []
+    for d in dev:
+        out = torch.zeros(B, cfg.total_classes, device="cuda")
+        first.forward(*d, out)
+        want.append(out)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    models = [first, second]
+    got = [torch.zeros(B, cfg.total_classes, device="cuda") for _ in dev]
+    for rep in range(3):
+        for i, d in enumerate(dev):
+            models[i % 2].forward(*d, got[i], stream=streams[i % 2])
+    torch.cuda.synchronize()
+    assert first.poll_status() == 0 and second.poll_status() == 0
+    for g, x in zip(got, want):
+        assert torch.equal(g, x)
+    other = mt.MTModel(synth.config_tiny(), 2, 32)
+    with pytest.raises(mt.MTError):
+        mt._check(mt.lib().mt_adopt_weights(other.handle, first.handle), "mt_adopt_weights", other.handle)
