@@ -183,6 +183,13 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
 int mt_forward_host(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids,
                     const int32_t* h_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
                     float* h_logits, void* stream);
+/* The same without the final synchronisation: everything (three copies in, the forward, one copy out)
+ * is only enqueued on `stream`; the host buffers must stay valid, and h_logits must not be read, until
+ * the stream has reached that point.  With pinned buffers nothing here blocks the host, so the whole
+ * call can also be captured into a CUDA graph and replayed. */
+int mt_forward_host_async(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids,
+                          const int32_t* h_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
+                          float* h_logits, void* stream);
 
 /* Synchronises `stream`, reads the sticky device status word into *flags (may be NULL) and clears
  * it.  Returns MT_ERR_DEVICE_FLAG if it was non-zero. */

@@ -49,6 +49,7 @@ SIGNATURES = {
     "mt_forward_events": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, C.POINTER(_P), _P]),
     "mt_forward_tokens": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P, C.POINTER(_P), _P]),
     "mt_forward_host": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
+    "mt_forward_host_async": (C.c_int, [_P, _P, _P, _P, _U64, _I32, _I32, _P, _P]),
     "mt_poll_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "mt_plan_summary": (C.c_int, [_P, _U64, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32)]),
     "mt_plan_launches": (C.c_int, [_P, _U64, C.POINTER(_I32)]),
@@ -301,6 +302,14 @@ class MTModel:
         mask = self.full_mask() if task_mask is None else task_mask
         _check(lib().mt_forward_host(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch, seq,
                                      _ptr(logits), _stream(stream)), "mt_forward_host", self.handle)
+
+    def forward_host_async(self, token_ids, segment_ids, lengths, logits, task_mask: Optional[int] = None,
+                           stream=None) -> None:
+        """forward_host without the final synchronisation (pinned host tensors; capturable in a CUDA graph)."""
+        batch, seq = token_ids.shape
+        mask = self.full_mask() if task_mask is None else task_mask
+        _check(lib().mt_forward_host_async(self.handle, _ptr(token_ids), _ptr(segment_ids), _ptr(lengths), mask, batch,
+                                           seq, _ptr(logits), _stream(stream)), "mt_forward_host_async", self.handle)
 
     def poll_status(self, stream=None) -> int:
         flags = C.c_uint32(0)

@@ -1299,6 +1299,14 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
 
 int mt_forward_host(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids, const int32_t* h_lengths,
                     uint64_t task_mask, int32_t batch, int32_t seq, float* h_logits, void* stream_) {
+  int rc = mt_forward_host_async(m, h_token_ids, h_segment_ids, h_lengths, task_mask, batch, seq, h_logits, stream_);
+  if (rc != MT_OK) return rc;
+  cudaError_t e = cudaStreamSynchronize(as_stream(stream_));
+  return e == cudaSuccess ? MT_OK : fail_cuda(m, e, "waiting for the logits");
+}
+
+int mt_forward_host_async(mt_model* m, const int32_t* h_token_ids, const int32_t* h_segment_ids, const int32_t* h_lengths,
+                          uint64_t task_mask, int32_t batch, int32_t seq, float* h_logits, void* stream_) {
   if (m == nullptr) return MT_ERR_INVALID_ARG;
   if (h_token_ids == nullptr || h_segment_ids == nullptr || h_lengths == nullptr || h_logits == nullptr)
     return fail(m, MT_ERR_INVALID_ARG, "null input or output pointer");
@@ -1320,8 +1328,7 @@ int mt_forward_host(mt_model* m, const int32_t* h_token_ids, const int32_t* h_se
     return fail_cuda(m, e, "copying inputs to the device");
   int rc = mt_forward(m, d_tok, d_seg, d_len, task_mask, batch, seq, d_logits, stream_);
   if (rc != MT_OK) return rc;
-  if ((e = cudaMemcpyAsync(h_logits, d_logits, out_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
-      (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+  if ((e = cudaMemcpyAsync(h_logits, d_logits, out_bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
     return fail_cuda(m, e, "copying logits to the host");
   return MT_OK;
 }

@@ -342,6 +342,19 @@ def test_host_entry_point_and_error_paths():
     host_logits = torch.empty(2, cfg.total_classes, dtype=torch.float32).pin_memory()
     model.forward_host(tok, seg, lens, host_logits)
     assert torch.equal(host_logits, dev_logits.cpu())
+    # the same without the final wait, directly and replayed from a CUDA graph that holds the whole call
+    later = torch.zeros_like(host_logits).pin_memory()
+    model.forward_host_async(tok, seg, lens, later)
+    torch.cuda.synchronize()
+    assert torch.equal(later, host_logits)
+    later.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=torch.cuda.Stream()):
+        model.forward_host_async(tok, seg, lens, later)
+    later.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(later, host_logits)
     # out-of-range ids are clamped and flagged, the context stays usable
     bad = batch.token_ids.copy()
     bad[0, 3] = 40000
