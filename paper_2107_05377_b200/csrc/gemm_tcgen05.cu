@@ -35,7 +35,7 @@ constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
 
 constexpr int kStagingBytes = 4096;  // 32 rows x 128 bytes, one epilogue chunk of one warp
 // A CTA of a pair stages only its half of the W tile, which leaves room for more stages.
-__host__ __device__ constexpr int gemm_stages(int bn, bool pair) { return pair ? 5 : (bn == 128 ? 5 : 4); }
+__host__ __device__ constexpr int gemm_stages(int bn, bool pair) { return pair ? 5 : (bn == 64 ? 6 : (bn == 128 ? 5 : 4)); }
 // staging buffers per epilogue warp: two where shared memory allows (needed to prefetch residuals)
 __host__ __device__ constexpr int gemm_staging_bufs(int bn, bool pair) { return (bn == 256 && !pair) ? 1 : 2; }
 __host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
@@ -61,8 +61,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   constexpr int NBUF = gemm_staging_bufs(BN, PAIR);
   constexpr int TILE_M = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
   constexpr int ACC_ARRIVALS = PAIR ? 2 * kNumEpilogueWarps : kNumEpilogueWarps;
-  constexpr uint32_t TMEM_COLS = BN == 128 ? 256 : 512;  // two accumulators; a power of two >= 32
-  static_assert(BN == 128 || BN == 192 || BN == 256, "tile widths implemented: 128, 192, 256");
+  constexpr uint32_t TMEM_COLS = BN == 64 ? 128 : (BN == 128 ? 256 : 512);  // two accumulators; a power of two >= 32
+  static_assert(BN == 64 || BN == 128 || BN == 192 || BN == 256, "tile widths implemented: 64, 128, 192, 256");
+  static_assert(BN != 64 || !PAIR, "64-wide tiles (launches of a few rows) run as single CTAs");
   static_assert(EPI != kEpiBiasResidual || NBUF == 2, "the residual epilogue prefetches: two staging buffers");
 
   extern __shared__ uint8_t smem_raw[];
@@ -465,6 +466,9 @@ cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStre
     case 256: return launch_bn<256, PAIR>(p, epilogue, sm_count, stream);
     case 192: return launch_bn<192, PAIR>(p, epilogue, sm_count, stream);
     case 128: return launch_bn<128, PAIR>(p, epilogue, sm_count, stream);
+    case 64:
+      if constexpr (!PAIR) return launch_bn<64, PAIR>(p, epilogue, sm_count, stream);
+      return cudaErrorInvalidValue;
     default: return cudaErrorInvalidValue;
   }
 }
@@ -473,7 +477,9 @@ cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStre
 
 int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int sm_count) {
   if (epilogue == kEpiBiasTanhF32) return 128;
-  const int candidates[3] = {256, 192, 128};
+  // (64: only ever the cheapest where a launch has so few rows that even 128-wide tiles leave most SMs
+  // without work - the first-token tails - and each CTA would stream a long K by itself)
+  const int candidates[4] = {256, 192, 128, 64};
   const int64_t tile_m = pair ? 2 * kGemmBlockM : kGemmBlockM;
   const int64_t workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
   const int64_t m_tiles = (rows + tile_m - 1) / tile_m;
@@ -482,6 +488,7 @@ int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int s
   for (int bn : candidates) {
     if (N % bn != 0) continue;
     if (bn == 256 && epilogue == kEpiBiasResidual) continue;   // not instantiated: two fp32 staging buffers do not fit
+    if (bn == 64 && pair) continue;
     const int64_t tiles = m_tiles * (N / bn) * groups;
     const int64_t rounds = (tiles + workers - 1) / workers;
     // per 64 of K a CTA stages 128 rows of X and bn (a pair's CTA: bn / 2) rows of W, and its tensor
