@@ -10,12 +10,16 @@
 // launches.  Here the tiles of the three GEMMs form one ordered list (phase-major, then row block,
 // group, column block) dealt out round-robin to one persistent CTA per SM, and dependencies are
 // tracked per block of 128 rows in global memory:
-//   * a phase-1 tile waits until "h1 ready" of its row block is set,
-//   * a phase-2 tile waits until all phase-1 tiles of its row block have arrived,
-//   * the CTA whose tile is the last of a row block in phase 0 (phase 2) normalises those 128 rows
-//     right there with its eight epilogue warps, then (phase 0) sets "h1 ready".
-// A tile only ever waits for tiles that precede it in the list, every CTA takes its tiles in list
-// order and all CTAs are resident (grid <= number of SMs, one CTA per SM), so the earliest unfinished
+//   * every epilogue warp of a tile arrives on its row block's counter once the stores it issued for the
+//     tile have completed (the arrival is deferred until the warp has stored the first chunk of its next
+//     tile, so that the round trip of the last store is hidden, unless it would idle anyway),
+//   * six more warps per CTA only normalise rows: their work items are pairs of rows of a (phase, row
+//     block, group), dealt round-robin over all such warps of the grid; an item waits until all tiles of
+//     its row block have arrived, and in phase 0 adds itself to "h1 ready",
+//   * a phase-1 tile waits until "h1 ready" of its row block is complete,
+//   * a phase-2 tile waits until all phase-1 tiles of its row block have arrived.
+// A tile only ever waits for tiles (and LayerNorm items) that precede it in the list, every CTA takes
+// its tiles in list order and all CTAs are resident (grid <= number of SMs, one CTA per SM), so the earliest unfinished
 // tile can always proceed: the waits cannot deadlock.  They are bounded all the same: after
 // kDepWaitLimitNs a waiting thread raises the CTA's abort flag, the status word gets
 // kFlagWaitTimeout, every role leaves its loop, copies in flight are drained, TMEM is freed.
@@ -120,8 +124,8 @@ struct PhaseShape {
   int bn, n_tiles_n, k_blocks, tiles_per_m, first;   // first = index of the phase's first tile in the list
 };
 
-// LayerNorm of rows [row0, row_end) by the eight epilogue warps, one row per warp at a time, two rows
-// in flight per warp so that the second row's loads overlap the first row's arithmetic.
+// One row of the pre-normalisation sum into registers; L1 is bypassed because the same addresses hold
+// another phase's sum later in the same launch.
 template <int V>
 __device__ __forceinline__ void load_row(const float* xin, int lane, float (&x)[V][8]) {
 #pragma unroll

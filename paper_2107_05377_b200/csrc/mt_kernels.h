@@ -149,7 +149,7 @@ cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream);
 //   phase 2  u  = f . W2^T + b2 + h1         (fp32)      then out = LN(u)   per block of 128 rows
 // The tiles of all three GEMMs form one ordered list that the CTAs walk through; a tile waits (bounded)
 // on counters in global memory until the row block it reads has been produced by earlier tiles, and
-// the CTA that completes a row block of phase 0 or 2 normalises it.  `sync` points at 4 zeroed words
+// warps set aside for it normalise the rows of a row block of phase 0 or 2 once all its tiles have arrived.  `sync` points at 4 zeroed words
 // per (group, row block): arrivals of phase 0, "h1 ready", arrivals of phase 1, arrivals of phase 2.
 // The arithmetic of every element is that of launch_gemm / launch_layernorm, so the results are
 // bit-identical to the five separate launches.
