@@ -239,9 +239,9 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * and for launches of at most "fused_ln_max_rows" (default 0) rows per layer, the default; any time): the attention-output and FFN-down projections carry the LayerNorm that follows
  * them: the CTAs holding the column blocks of the same 128 rows form a thread-block cluster and exchange
  * per-row statistics through distributed shared memory, so the pre-normalisation sum never goes to global
- * memory and no LayerNorm launch follows.  Results agree with the separate launches to fp32 rounding of
- * the row statistics.  Measured: a few microseconds faster for a single layer, slower than the wider
- * paired tiles of the plain GEMM where several layers share a launch.
+ * memory and no LayerNorm launch follows.  Results have the same bits as the separate launches
+ * (every LayerNorm of the library sums its row statistics over the same 64-column segments in the same order).  Measured: a few microseconds faster for one or two layers, slower than the wider
+ * paired tiles of the plain GEMM where more layers share a launch.
  * key "pool_gemm" (0/1, default 1, any time): the pooler of tasks whose last branch layer was evaluated on
  * first tokens only runs as one grouped GEMM with a tanh epilogue on the tensor cores (1) or in the
  * row-wise pooler kernel (0, also used for every other task); logits agree to rounding.
