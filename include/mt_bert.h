@@ -242,6 +242,11 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * memory and no LayerNorm launch follows.  Results have the same bits as the separate launches
  * (every LayerNorm of the library sums its row statistics over the same 64-column segments in the same order).  Measured: a few microseconds faster for one or two layers, slower than the wider
  * paired tiles of the plain GEMM where more layers share a launch.
+ * key "overlap_cls" (0/1, default 1, any time): where a wave holds layers on all tokens and last branch
+ * layers, the first-token attention of the latter runs on a stream the library creates for itself (first
+ * use), forked from the caller's stream after the wave's Q/K/V projection and joined before the next
+ * step, so that it overlaps the wave's other kernels; the caller sees ordinary single-stream semantics,
+ * also under stream capture.  Same results.
  * key "pool_gemm" (0/1, default 1, any time): the pooler of tasks whose last branch layer was evaluated on
  * first tokens only runs as one grouped GEMM with a tanh epilogue on the tensor cores (1) or in the
  * row-wise pooler kernel (0, also used for every other task); logits agree to rounding.

@@ -204,6 +204,12 @@ struct mt_model {
                      // 2 for launches of at most fused_ln_max_groups layers
   int32_t fused_ln_max_groups;
   int32_t fused_ln_max_rows;
+  // The first-token attention of the branches that end in a wave depends on the wave's QKV projection only
+  // and feeds nothing before the first-token tails, so it runs on a stream of the library's own beside the
+  // wave's other kernels (fork after the projection, join before the next step); option "overlap_cls".
+  bool overlap_cls;
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
   bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
   int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
@@ -821,6 +827,9 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->expected_tokens = 0;
   m->fused_tail = 0;
   m->pool_gemm = true;
+  m->overlap_cls = true;
+  m->side_stream = nullptr;
+  m->ev_fork = m->ev_join = nullptr;
   m->fused_ln = 2;
   m->fused_ln_max_groups = 2;
   m->fused_ln_max_rows = 0;
@@ -881,6 +890,9 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
 void mt_destroy(mt_model* m) {
   if (m == nullptr) return;
   for (cudaEvent_t ev : m->events) cudaEventDestroy(ev);
+  if (m->ev_fork != nullptr) cudaEventDestroy(m->ev_fork);
+  if (m->ev_join != nullptr) cudaEventDestroy(m->ev_join);
+  if (m->side_stream != nullptr) cudaStreamDestroy(m->side_stream);
   delete m;
 }
 
@@ -937,6 +949,10 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     if (value < 1) return fail(m, MT_ERR_INVALID_ARG, "fused_ln_max_groups must be >= 1");
     m->fused_ln_max_groups = static_cast<int32_t>(value);
     m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "overlap_cls") == 0) {
+    m->overlap_cls = value != 0;
     return MT_OK;
   }
   if (strcmp(key, "pool_gemm") == 0) {
@@ -1247,14 +1263,32 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     MT_LAUNCH(cudaMemcpyAsync(m->d_workspace + m->ws_dump0, ep.out, act_used, cudaMemcpyDeviceToDevice, stream),
               "debug capture");
 
+  bool side_pending = false;   // work on the side stream that the caller's stream has not waited for yet
   for (PlanStep& st : plan.steps) {
+    if (side_pending) {
+      MT_LAUNCH(cudaStreamWaitEvent(stream, m->ev_join, 0), "joining the side stream");
+      side_pending = false;
+    }
     if (st.kind == 0) {
       Chunk& ck = st.chunk;
       ck.attn.lengths = d_lengths;
       ck.attn_cls.lengths = d_lengths;
       MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
+      const bool beside = m->overlap_cls && !m->profile && ck.n_cls > 0 && ck.full.count > 0;
+      if (beside) {
+        if (m->side_stream == nullptr) {
+          MT_LAUNCH(cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking), "creating the side stream");
+          MT_LAUNCH(cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming), "creating an event");
+          MT_LAUNCH(cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming), "creating an event");
+        }
+        MT_LAUNCH(cudaEventRecord(m->ev_fork, stream), "forking the side stream");
+        MT_LAUNCH(cudaStreamWaitEvent(m->side_stream, m->ev_fork, 0), "forking the side stream");
+        MT_LAUNCH(launch_cls_attention(ck.attn_cls, m->side_stream), "first-token attention kernel");
+        MT_LAUNCH(cudaEventRecord(m->ev_join, m->side_stream), "joining the side stream");
+        side_pending = true;
+      }
       if (ck.full.count > 0) MT_TIMED(MT_CLASS_ATTENTION, launch_attention(ck.attn, stream), "attention kernel");
-      if (ck.n_cls > 0)
+      if (ck.n_cls > 0 && !beside)
         MT_TIMED(MT_CLASS_ATTENTION, launch_cls_attention(ck.attn_cls, stream), "first-token attention kernel");
       if (ck.full.count > 0) MT_TAIL(&ck.full);
       for (const DumpCopy& d : ck.dumps)
@@ -1288,6 +1322,7 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
             MT_LAUNCH(cudaEventRecord(reinterpret_cast<cudaEvent_t>(task_events[t]), stream), "recording a task event");
     }
   }
+  if (side_pending) MT_LAUNCH(cudaStreamWaitEvent(stream, m->ev_join, 0), "joining the side stream");
 #undef MT_TAIL
 #undef MT_TIMED
 #undef MT_LAUNCH
