@@ -145,7 +145,9 @@ int mt_adopt_weights(mt_model* m, const mt_model* src);
  * branch starts from the trunk state at its fork depth; keys at positions >= length are excluded
  * from every softmax; the pooler reads position 0.  Asynchronous: only enqueues kernels on `stream`,
  * never synchronises, never allocates device memory.  The first call for a given
- * (batch, seq, task_mask) builds and caches a launch plan on the host.
+ * (batch, seq, task_mask) builds and caches a launch plan on the host; the first call that needs it also
+ * creates the model's own second stream and two events (option "overlap_cls") - make one warm-up call
+ * before capturing mt_forward into a CUDA graph.
  * Errors: INVALID_ARG, SHAPE, NOT_BOUND, NOT_LOADED, CUDA. */
 int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
                const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
