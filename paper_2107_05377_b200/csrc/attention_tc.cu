@@ -68,6 +68,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_shared();
     prefetch_tensormap(&p.tmap_qkv[g]);
+    prefetch_tensormap(&p.tmap_qkv64[g]);
   }
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTcTmemCols);
   tc_fence_before();
@@ -88,10 +89,14 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
   bool loads_in_flight = false;
   if (len > 0) {
     if (tid == 0) {
-      mbar_expect_tx(bar_load, 3 * kTcTileBytes);
-      tma_load_2d(sQ, &p.tmap_qkv[g], head * kHeadDim, row0, bar_load);
-      tma_load_2d(sK, &p.tmap_qkv[g], H + head * kHeadDim, row0, bar_load);
-      tma_load_2d(sV, &p.tmap_qkv[g], 2 * H + head * kHeadDim, row0, bar_load);
+      // a sequence of at most 64 tokens needs only the first 64 rows of each tile (the rest of the tiles
+      // keeps whatever shared memory held: query rows and keys >= length never reach a result, and the V
+      // rows >= length are overwritten with zeros below)
+      const CUtensorMap* map = len <= 64 ? &p.tmap_qkv64[g] : &p.tmap_qkv[g];
+      mbar_expect_tx(bar_load, len <= 64 ? 3 * kTcTileBytes / 2 : 3 * kTcTileBytes);
+      tma_load_2d(sQ, map, head * kHeadDim, row0, bar_load);
+      tma_load_2d(sK, map, H + head * kHeadDim, row0, bar_load);
+      tma_load_2d(sV, map, 2 * H + head * kHeadDim, row0, bar_load);
     }
     ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag)) != 0;
     loads_in_flight = !ok;

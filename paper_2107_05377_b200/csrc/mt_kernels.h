@@ -101,6 +101,7 @@ cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStr
 // layout, in which only valid tokens exist).  A null row_start means the padded layout.
 struct alignas(64) AttnParams {
   CUtensorMap tmap_qkv[kMaxGroups];  // qkv_g: dims {3H, rows}, box {64, 128}, 128-byte swizzle (tensor-memory kernel only)
+  CUtensorMap tmap_qkv64[kMaxGroups];  // the same with a box of 64 rows: sequences of at most 64 tokens fetch half
   const bf16* qkv[kMaxGroups];  // [rows, 3*H] = [Q | K | V]
   bf16* ctx[kMaxGroups];        // [rows, H]
   const int32_t* lengths;       // [B]
