@@ -8,6 +8,8 @@ One JSON line per case:
     fork), eagerly launched and replayed from a CUDA graph;
   * eight independent full-depth (12-layer) single-task models over the same inputs, through the same
     library, to reproduce the paper's sharing saving (Table 2: 96 layers against the merged tree's 24);
+  * the merged models whose layer totals the paper prints (Table 2, Table 4), at 32 x 128 with lengths in
+    [16, 128]: measured time against the paper's cost measure, the number of layers evaluated;
   * the long-sequence variant (16 x 512, lengths in [128, 512]), the BERT-large-width tree
     (64 x 128, lengths in [32, 128]) and a 21-task tree shaped like the production model of Appendix E
     (8 shared + 32 task layers, a third of the tasks token-level; 32 x 128, lengths in [16, 128]).
@@ -161,6 +163,13 @@ def main():
         run_tree("large-width tree", big, big_blob, synth.make_batch(big, 64, 128, 32, 128, seed=1),
                  [("all 8", 0xFF)], 20, out)
         del big_blob
+        # the paper's own merged models (Table 2, Table 4): measured cost against its measure, the layer count
+        for name in synth.PAPER_TREES:
+            tree = synth.config_paper_tree(name)
+            tree_blob = synth.pack_weights(tree, synth.make_weights(tree, seed=0))
+            run_tree(f"paper tree: {name}", tree, tree_blob, synth.make_batch(tree, 32, 128, 16, 128, seed=1),
+                     [("all 8", 0xFF)], 20, out)
+            del tree_blob
         prod = synth.config_production21()
         prod_blob = synth.pack_weights(prod, synth.make_weights(prod, seed=0))
         seq_only = sum(1 << t for t, spec in enumerate(prod.tasks) if not spec.token_level)

@@ -102,6 +102,30 @@ def config_large8() -> TreeConfig:
                       tasks=_tasks([18, 17, 16, 15, 14, 13, 12, 16], [2] * 8, [2, 2, 2, 3, 2, 2, 2, 3]))
 
 
+# The (x, y) = (frozen layers, task layers) lists of the merged models whose layer totals the paper prints
+# (Table 2; Table 4 for c = 2, 3), tasks in the order QNLI RTE QQP MNLI SST-2 MRPC CoLA STS-B.  The
+# "KD-n" rows print only "7 + n x 8"; the per-task x is taken from the bracketed rows, where it is fixed
+# before distillation.
+PAPER_TREES = {
+    "full fine-tuning, 8 models": [(0, 12)] * 8,
+    "ours (KD-1)": [(2, 1), (7, 1), (2, 1), (4, 1), (6, 1), (7, 1), (4, 1), (4, 1)],
+    "ours (KD-2)": [(2, 2), (7, 2), (2, 2), (4, 2), (6, 2), (7, 2), (4, 2), (4, 2)],
+    "ours (KD-3)": [(2, 3), (7, 3), (2, 3), (4, 3), (6, 3), (7, 3), (4, 3), (4, 3)],
+    "ours (w/o KD)": [(2, 10), (7, 5), (2, 10), (4, 8), (6, 6), (7, 5), (4, 8), (4, 8)],
+    "ours (mixed, c = 1)": [(2, 3), (7, 5), (2, 1), (4, 3), (6, 2), (7, 3), (4, 8), (4, 1)],
+    "ours (c = 2)": [(2, 2), (7, 1), (2, 1), (4, 2), (6, 2), (7, 1), (4, 3), (4, 1)],
+    "ours (c = 3)": [(2, 1), (7, 1), (2, 1), (4, 2), (6, 1), (7, 1), (4, 3), (4, 1)],
+}
+GLUE_CLASSES = [2, 2, 2, 3, 2, 2, 2, 1]
+
+
+def config_paper_tree(name: str) -> TreeConfig:
+    """One of the paper's merged models as a tree over a BERT-base trunk that is as deep as its deepest fork."""
+    xy = PAPER_TREES[name]
+    return TreeConfig(trunk_layers=max(x for x, _ in xy),
+                      tasks=_tasks([x for x, _ in xy], [y for _, y in xy], GLUE_CLASSES))
+
+
 def config_production21() -> TreeConfig:
     """Shaped like the production model of Appendix E: 21 tasks on a BERT-base trunk, 8 shared layers and
     32 task layers in all (eleven branches of 2 layers, ten of 1).  Every third task is token-level (9

@@ -56,6 +56,17 @@ def test_scheduler_runs_the_papers_layer_totals(lib, name, total, xy):
     m.close()
 
 
+def test_generator_paper_trees_are_the_golden_ones(lib):
+    """The (x, y) lists the serving sweep runs (synth.PAPER_TREES) are those of the golden file, in its order,
+    and the library schedules the printed layer totals for them."""
+    golden = read_paper_layer_counts()
+    assert [xy for _, _, xy in golden] == list(synth.PAPER_TREES.values())
+    for (_, total, _), name in zip(golden, synth.PAPER_TREES):
+        m = binding.MTModel(synth.config_paper_tree(name), 2, 32, bind=False)
+        assert m.plan_summary(0xFF)["layers"] == total
+        m.close()
+
+
 def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     cfg = synth.config_glue8()
     m = binding.MTModel(cfg, 32, 128, bind=False)
