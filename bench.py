@@ -200,7 +200,7 @@ def main():
     ap.add_argument("--eager", action="store_true",
                     help="launch every kernel from the host in the timed passes instead of replaying CUDA graphs")
     ap.add_argument("--set", action="append", default=[], metavar="KEY=VALUE",
-                    help="library option (mt_set_option) to set before the run, e.g. --set fused_tail=0; repeatable")
+                    help="library option (mt_set_option) to set before the run, e.g. --set fused_ln=0; repeatable")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -62,7 +62,8 @@ typedef struct {
   int32_t ffn;           /* 3072 or 4096 */
   int32_t trunk_layers;  /* number of frozen layers loaded (12 for BERT-base) */
   float   ln_eps;        /* 1e-12 */
-  int32_t activation;    /* 0 = exact (erf) GELU; nothing else is implemented */
+  int32_t activation;    /* 0 = GELU of the exact form x * Phi(x); nothing else is implemented.  The kernels evaluate
+                            it through a fitted sigmoid argument, absolute error <= 2.6e-5 before bf16 rounding */
 } mt_trunk_config;
 
 /* One student model before merging, Table 2's (x, y): x = fork_depth frozen layers, y = branch_layers. */
@@ -112,7 +113,8 @@ int mt_bind_memory(mt_model* m, void* d_weights, size_t weights_bytes, void* d_w
 size_t mt_blob_bytes(const mt_model* m);
 size_t mt_task_blob_bytes(const mt_model* m, int32_t task);
 
-/* "Load weights from multiple model checkpoints into one computation graph" (Section 3.3).
+/* Model merging (Section 3.3): the students' checkpoints, packed into one blob, are loaded into the one
+ * merged graph.
  * Validates the header against the configuration, then copies the payload to the weights arena
  * with cudaMemcpyAsync on `stream` (host_blob must stay valid until the stream reaches that point;
  * pinned memory makes the copy asynchronous).  Errors: NOT_BOUND, BLOB_MISMATCH, CUDA. */
@@ -145,9 +147,10 @@ int mt_adopt_weights(mt_model* m, const mt_model* src);
  * branch starts from the trunk state at its fork depth; keys at positions >= length are excluded
  * from every softmax; the pooler reads position 0.  Asynchronous: only enqueues kernels on `stream`,
  * never synchronises, never allocates device memory.  The first call for a given
- * (batch, seq, task_mask) builds and caches a launch plan on the host; the first call that needs it also
- * creates the model's own second stream and two events (option "overlap_cls") - make one warm-up call
- * before capturing mt_forward into a CUDA graph.
+ * (batch, seq, task_mask) builds and caches a launch plan on the host (host memory and tensor-map
+ * encoding only; the model's own second stream and its two events exist since mt_bind_memory) - make one
+ * warm-up call before capturing mt_forward into a CUDA graph.  Option "profile" creates CUDA events here.
+ * One mt_model serves one caller at a time: the cached plans carry per-call pointers.
  * Errors: INVALID_ARG, SHAPE, NOT_BOUND, NOT_LOADED, CUDA. */
 int mt_forward(mt_model* m, const int32_t* d_token_ids, const int32_t* d_segment_ids,
                const int32_t* d_lengths, uint64_t task_mask, int32_t batch, int32_t seq,
@@ -209,6 +212,13 @@ int mt_plan_summary(const mt_model* m, uint64_t task_mask, int32_t* n_layers, in
 /* Kernel launches one mt_forward at batch = max_batch, seq = max_seq enqueues for this mask. */
 int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches);
 
+/* Launch plans currently cached (host side; no device access).  mt_forward keeps one plan per distinct
+ * (task_mask, batch, seq), at most option "plan_cache" of them (default 32, >= 1, any time; setting it
+ * clears the cache); beyond that the least recently used plan is dropped and rebuilt on its next use.
+ * Serving many request shapes (Section 5.2: per-request task subsets) therefore costs bounded host memory.
+ * Returns the count, or MT_ERR_INVALID_ARG for a null model. */
+int mt_plan_cache_size(const mt_model* m);
+
 /* Options.  key "max_groups" (1..8): upper bound on layers fused into one grouped launch;
  * key "debug_capture" (0/1): keep a copy of every layer output for mt_debug_copy_hidden (changes
  * mt_workspace_bytes); both must be set before mt_bind_memory.  key "profile" (0/1): see
@@ -225,16 +235,7 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * for seq <= 128 runs on tcgen05 with its accumulators in tensor memory (1) or on mma.sync (0, also
  * used for every longer seq).  key "expected_tokens" (>= 0, default 0 = every row, any time): the caller's
  * estimate of the valid tokens per batch; with the packed layout the GEMM tile widths are chosen for
- * that many rows instead of batch*seq; it never changes a result.  key "fused_tail" (0 never, the default; 1 always; 2 = where a wave
- * has at least "fused_min_groups" (default 3) layers; any time): the part of
- * a layer after attention (output projection + residual, LayerNorm, FFN up + GELU, FFN down + residual,
- * LayerNorm) runs, for all layers of a wave, as ONE persistent launch whose tiles wait on per-row-block
- * counters in the workspace, instead of five launches; bit-identical results.  Measured slower than the
- * five launches at batch 32 x seq 128 (each hand-over between tiles through global memory costs 2-3 us).  Its CTAs wait for one
- * another, so all of them must be resident: forwards of several models or streams that overlap on one
- * device can make those waits run out (status flag MT_FLAG_WAIT_TIMEOUT) - serialise them, or set 0.
- * keys "tail_bn0", "tail_bn1", "tail_bn2" (0 = automatic, 128, 192; any time): tile widths of the three
- * GEMMs of that launch; they never change a result.
+ * that many rows instead of batch*seq; it never changes a result.
  * key "sm_limit" (>= 0, default 0 = all; any time): size the persistent GEMM grids for at most this many SMs
  * (for callers that share the GPU between several streams and want to leave room; measured no gain).
  * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 2) layers
@@ -245,8 +246,8 @@ int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches)
  * (every LayerNorm of the library sums its row statistics over the same 64-column segments in the same order).  Measured: a few microseconds faster for one or two layers, slower than the wider
  * paired tiles of the plain GEMM where more layers share a launch.
  * key "overlap_cls" (0/1, default 1, any time): where a wave holds layers on all tokens and last branch
- * layers, the first-token attention of the latter runs on a stream the library creates for itself (first
- * use), forked from the caller's stream after the wave's Q/K/V projection and joined before the next
+ * layers, the first-token attention of the latter runs on a stream the library creates for itself (in
+ * mt_bind_memory), forked from the caller's stream after the wave's Q/K/V projection and joined before the next
  * step, so that it overlaps the wave's other kernels; the caller sees ordinary single-stream semantics,
  * also under stream capture.  Same results.
  * key "pool_gemm" (0/1, default 1, any time): the pooler of tasks whose last branch layer was evaluated on
@@ -271,8 +272,7 @@ int mt_set_option(mt_model* m, const char* key, int64_t value);
 #define MT_CLASS_FFN_DOWN  6  /* GEMM: FFN down projection + residual               */
 #define MT_CLASS_LN2       7  /* LayerNorm after the FFN                            */
 #define MT_CLASS_HEAD      8  /* pooler + head                                      */
-#define MT_CLASS_TAIL      9  /* fused layer tail: classes 3-7 as one launch            */
-#define MT_NUM_CLASSES     10
+#define MT_NUM_CLASSES     9
 int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class);
 
 /* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out (padded
@@ -287,13 +287,17 @@ const char* mt_last_error_string(const mt_model* m);
 /* All pointers are device pointers; d_status may be NULL or point to one uint32 status word.      */
 
 /* Y[M,N] = epilogue(X[M,K] . W[N,K]^T + bias[N]) on tcgen05 tensor cores (X, W, bias bf16; fp32
- * accumulate).  epilogue 0: +bias, Y bf16; 1: +bias then erf-GELU, Y bf16; 2: +bias +residual with
+ * accumulate).  epilogue 0: +bias, Y bf16; 1: +bias then GELU x * Phi(x) (fitted evaluation, absolute error <= 2.6e-5, then one rounding), Y bf16; 2: +bias +residual with
  * residual fp32 [M,N] and Y fp32 [M,N] (the LayerNorm input).  K % 64 == 0, N % 128 == 0, all
  * pointers 16-byte aligned.  cta_pair != 0 runs it as pairs of CTAs (see option "gemm_pair").  This is
  * one linear map of the layer above. */
 int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
                      void* d_y, int32_t M, int32_t N, int32_t K, int32_t epilogue, int32_t cta_pair,
                      uint32_t* d_status, void* stream);
+/* Tuning aid for the kernel micro-benchmark: forces the tile width (64, 128, 192, 256; must divide N) of the
+ * following mt_kernel_linear calls of this process; 0 returns to the automatic choice.  Never changes a
+ * result: every output element is one fixed-order sum over K whatever the tile. */
+void mt_kernel_linear_force_block_n(int32_t block_n);
 
 /* Y = LN(X[M,K] . W[N,K]^T + bias[N] + residual[M,N]) * gamma[N] + beta[N] in one launch: the residual
  * sub-layer followed by LayerNorm, as the encoder layer has it twice (after attention, after the FFN).

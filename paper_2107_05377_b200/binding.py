@@ -18,7 +18,7 @@ MT_OK = 0
 ERRORS = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "NOT_BOUND", -4: "NOT_LOADED", -5: "BLOB_MISMATCH",
           -6: "CUDA", -7: "UNSUPPORTED", -8: "DEVICE_FLAG"}
 FLAG_BAD_TOKEN, FLAG_BAD_SEGMENT, FLAG_BAD_LENGTH, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head", "tail")
+KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head")
 
 
 class TrunkConfig(C.Structure):
@@ -53,10 +53,12 @@ SIGNATURES = {
     "mt_poll_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "mt_plan_summary": (C.c_int, [_P, _U64, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I32)]),
     "mt_plan_launches": (C.c_int, [_P, _U64, C.POINTER(_I32)]),
+    "mt_plan_cache_size": (C.c_int, [_P]),
     "mt_set_option": (C.c_int, [_P, C.c_char_p, C.c_int64]),
     "mt_debug_copy_hidden": (C.c_int, [_P, _I32, _I32, _P, _P]),
     "mt_profile_read": (C.c_int, [_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "mt_last_error_string": (C.c_char_p, [_P]),
+    "mt_kernel_linear_force_block_n": (None, [C.c_int32]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_linear_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
@@ -233,6 +235,9 @@ class MTModel:
         n = _I32()
         _check(lib().mt_plan_launches(self.handle, task_mask, C.byref(n)), "mt_plan_launches", self.handle)
         return n.value
+
+    def plan_cache_size(self) -> int:
+        return lib().mt_plan_cache_size(self.handle)
 
     # -- device -------------------------------------------------------------
     def bind(self, device: str = "cuda:0") -> None:

@@ -80,14 +80,14 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
   grid_launch_dependents();
 
   int len = p.lengths[b];
-  len = len < 0 ? 0 : (len > p.seq ? p.seq : len);
+  len = len < 1 ? 1 : (len > p.seq ? p.seq : len);   // as every kernel of the path: a bad length is clamped (and flagged by the embedding)
   const int row0 = p.row_start != nullptr ? p.row_start[b] : b * p.seq;
   const int rows_out = p.packed ? len : p.seq;   // the padded layout also gets its rows >= length, as zeros
   bf16* ctx = p.ctx[g];
 
   bool ok = true;
   bool loads_in_flight = false;
-  if (len > 0) {
+  {
     if (tid == 0) {
       // a sequence of at most 64 tokens needs only the first 64 rows of each tile (the rest of the tiles
       // keeps whatever shared memory held: query rows and keys >= length never reach a result, and the V
@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
     loads_in_flight = !ok;
   }
 
-  if (ok && len > 0) {
+  if (ok) {
     // keys >= length take no part: their probabilities are exactly 0, and 0 * V must stay finite
     if (tid >= len) {
 #pragma unroll
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
     ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag)) != 0;
   }
 
-  if (ok && len > 0) {
+  if (ok) {
     tc_fence_after();
     const int key_tiles = len > 64 ? 2 : 1;
     const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
@@ -220,11 +220,6 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
         *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(row0 + r) * H + head * kHeadDim + chunk * 8) = val;
       }
     }
-  } else if (ok && len == 0) {
-    // an empty sequence has rows only in the padded layout: zeros
-    const int chunk = tid & 7;
-    for (int r = tid >> 3; r < rows_out; r += kTcThreads / 8)
-      *reinterpret_cast<uint4*>(ctx + static_cast<size_t>(row0 + r) * H + head * kHeadDim + chunk * 8) = make_uint4(0, 0, 0, 0);
   }
 
   if (!ok && tid == 0) {

@@ -34,16 +34,30 @@ constexpr int kNumEpilogueWarps = 8;
 constexpr int kGemmThreads = 32 * (2 + kNumEpilogueWarps);
 
 constexpr int kStagingBytes = 4096;  // 32 rows x 128 bytes, one epilogue chunk of one warp
-// A CTA of a pair stages only its half of the W tile, which leaves room for more stages.
-__host__ __device__ constexpr int gemm_stages(int bn, bool pair) { return pair ? 5 : (bn == 64 ? 6 : (bn == 128 ? 5 : 4)); }
-// staging buffers per epilogue warp: two where shared memory allows (needed to prefetch residuals)
-__host__ __device__ constexpr int gemm_staging_bufs(int bn, bool pair) { return (bn == 256 && !pair) ? 1 : 2; }
+// Shared memory of a CTA: the ring of operand stages, the epilogue warps' staging buffers, bookkeeping.
+// The ring is what bounds a CTA's throughput (bytes in flight over the load latency), so it gets all the
+// room the staging leaves.  The residual epilogue prefetches its fp32 residual chunk while it works on
+// the previous one and needs two staging buffers per warp; the other epilogues take one or two
+// (MT_GEMM_NBUF) - with one, a warp waits for its last store to have read the buffer before refilling it.
+#ifndef MT_GEMM_NBUF
+#define MT_GEMM_NBUF 2
+#endif
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kBookBytes = 512 + 1024;   // barriers/bookkeeping + slack for manual 1024-byte alignment
 __host__ __device__ constexpr int gemm_a_bytes() { return kGemmBlockM * kGemmBlockK * 2; }
+// A CTA of a pair stages only its half of the W tile.
 __host__ __device__ constexpr int gemm_b_bytes(int bn, bool pair) { return (pair ? bn / 2 : bn) * kGemmBlockK * 2; }
-__host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair) {
-  // stages + staging + barriers/bookkeeping + slack for manual 1024-byte alignment
-  return gemm_stages(bn, pair) * (gemm_a_bytes() + gemm_b_bytes(bn, pair)) +
-         kNumEpilogueWarps * gemm_staging_bufs(bn, pair) * kStagingBytes + 512 + 1024;
+__host__ __device__ constexpr int gemm_staging_bufs(int bn, bool pair, int epi) {
+  return epi == kEpiBiasResidual ? 2 : ((bn == 256 && !pair) ? 1 : MT_GEMM_NBUF);
+}
+__host__ __device__ constexpr int gemm_stages(int bn, bool pair, int epi) {
+  const int room = kSmemLimit - kBookBytes - kNumEpilogueWarps * gemm_staging_bufs(bn, pair, epi) * kStagingBytes;
+  const int s = room / (gemm_a_bytes() + gemm_b_bytes(bn, pair));
+  return s > 8 ? 8 : s;
+}
+__host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair, int epi) {
+  return gemm_stages(bn, pair, epi) * (gemm_a_bytes() + gemm_b_bytes(bn, pair)) +
+         kNumEpilogueWarps * gemm_staging_bufs(bn, pair, epi) * kStagingBytes + kBookBytes;
 }
 
 // ---- the kernel -------------------------------------------------------------------------------
@@ -55,10 +69,10 @@ __host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair) {
 // is what bounds the single-CTA kernel (an SM takes in roughly 64 bytes per clock).
 template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __grid_constant__ GemmParams p) {
-  constexpr int STAGES = gemm_stages(BN, PAIR);
+  constexpr int STAGES = gemm_stages(BN, PAIR, EPI);
   constexpr int A_BYTES = gemm_a_bytes();
   constexpr int B_BYTES = gemm_b_bytes(BN, PAIR);   // this CTA's part of the W tile
-  constexpr int NBUF = gemm_staging_bufs(BN, PAIR);
+  constexpr int NBUF = gemm_staging_bufs(BN, PAIR, EPI);
   constexpr int TILE_M = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
   constexpr int ACC_ARRIVALS = PAIR ? 2 * kNumEpilogueWarps : kNumEpilogueWarps;
   constexpr uint32_t TMEM_COLS = BN == 64 ? 128 : (BN == 128 ? 256 : 512);  // two accumulators; a power of two >= 32
@@ -377,8 +391,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
                 float x0 = __uint_as_float(v[q * 8 + 2 * j]) + bf16_lo(bw[j]);
                 float x1 = __uint_as_float(v[q * 8 + 2 * j + 1]) + bf16_hi(bw[j]);
                 if (EPI == kEpiBiasGelu) {
-                  x0 = gelu_erf(x0);
-                  x1 = gelu_erf(x1);
+                  x0 = gelu_fitted(x0);
+                  x1 = gelu_fitted(x1);
                 }
                 ow[j] = pack_bf16(x0, x1);
               }
@@ -431,7 +445,7 @@ cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (!configured || configured_device != dev) {
-    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN, PAIR));
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN, PAIR, EPI));
     if (err != cudaSuccess) return err;
     configured = true;
     configured_device = dev;
@@ -441,7 +455,7 @@ cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
   const int workers_max = PAIR ? sm_count / 2 : sm_count;
   const int workers = tiles < workers_max ? tiles : workers_max;
   if (workers <= 0) return cudaSuccess;
-  return launch_kernel(kernel, dim3(PAIR ? 2 * workers : workers), dim3(kGemmThreads), gemm_smem_bytes(BN, PAIR), stream,
+  return launch_kernel(kernel, dim3(PAIR ? 2 * workers : workers), dim3(kGemmThreads), gemm_smem_bytes(BN, PAIR, EPI), stream,
                        p, PAIR ? 2u : 1u);
 }
 
@@ -451,8 +465,8 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
     case kEpiBias: return launch_one<BN, kEpiBias, PAIR>(p, sm_count, stream);
     case kEpiBiasGelu: return launch_one<BN, kEpiBiasGelu, PAIR>(p, sm_count, stream);
     case kEpiBiasResidual:
-      if constexpr (BN != 256) return launch_one<BN, kEpiBiasResidual, PAIR>(p, sm_count, stream);
-      return cudaErrorInvalidValue;  // 256-wide tiles are not used with the residual epilogue
+      if constexpr (BN != 256 || PAIR) return launch_one<BN, kEpiBiasResidual, PAIR>(p, sm_count, stream);
+      return cudaErrorInvalidValue;  // single CTAs: 256-wide stages and two fp32 staging buffers do not fit
     case kEpiBiasTanhF32:   // the pooler: a few rows, single CTAs on 128-wide tiles only
       if constexpr (BN == 128 && !PAIR) return launch_one<BN, kEpiBiasTanhF32, PAIR>(p, sm_count, stream);
       return cudaErrorInvalidValue;
@@ -487,7 +501,7 @@ int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int s
   int64_t best_cost = -1;
   for (int bn : candidates) {
     if (N % bn != 0) continue;
-    if (bn == 256 && epilogue == kEpiBiasResidual) continue;   // not instantiated: two fp32 staging buffers do not fit
+    if (bn == 256 && epilogue == kEpiBiasResidual && !pair) continue;   // not instantiated: two fp32 staging buffers do not fit
     if (bn == 64 && pair) continue;
     const int64_t tiles = m_tiles * (N / bn) * groups;
     const int64_t rounds = (tiles + workers - 1) / workers;

@@ -26,6 +26,7 @@ using namespace mt;
 namespace mt {
 bool g_use_pdl = true;
 }
+static int g_force_block_n = 0;   // tile width forced on mt_kernel_linear (tuning aid), 0 = chosen by gemm_block_n
 
 namespace {
 
@@ -77,9 +78,6 @@ struct LayerTail {
   GemmParams attn_out, ffn_up, ffn_down;
   LayerNormParams ln1, ln2;
   int32_t count = 0;
-  // the same five steps as one persistent launch (option "fused_tail"), with its own tile widths
-  bool fused = false;
-  ChainParams chain;
   // each residual GEMM together with the LayerNorm after it, as one cluster launch (option "fused_ln")
   bool ln_fused = false;
   GemmLnParams attn_out_ln, ffn_down_ln;
@@ -116,7 +114,7 @@ struct PlanStep {
 struct Plan {
   std::vector<PlanStep> steps;
   int32_t launches = 0;
-  size_t sync_bytes = 0;  // counters of the fused layer-tail launches, zeroed at the start of a forward
+  uint64_t last_use = 0;  // stamp of the last forward that ran this plan (least recently used goes first)
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -197,9 +195,6 @@ struct mt_model {
   bool attention_tc;  // attention on tcgen05 with tensor-memory accumulators when seq <= 128 (else mma.sync)
   int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
-  int32_t fused_tail;  // steps 3-7 of a layer (output projection .. second LayerNorm) as one persistent launch per
-                       // wave: 0 never, 1 always, 2 where the wave has at least fused_min_groups layers
-  int32_t fused_min_groups;
   int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always,
                      // 2 for launches of at most fused_ln_max_groups layers
   int32_t fused_ln_max_groups;
@@ -211,7 +206,6 @@ struct mt_model {
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
   bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
-  int32_t tail_bn[3];  // tile widths of the fused launch's three GEMMs (0 = chosen by chain_block_n)
 
   // device memory (caller-owned)
   uint8_t* d_weights;
@@ -222,8 +216,7 @@ struct mt_model {
 
   // workspace layout (byte offsets)
   size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
-      ws_slot0, ws_cls0, ws_dump0, ws_sync;
-  size_t sync_bytes;   // room for the counters of all fused layer-tail launches of one forward
+      ws_slot0, ws_cls0, ws_dump0;
   size_t cls_bytes, cls_h_bytes, cls_h32_bytes;  // per-task first-token scratch and its [B,H] bf16 / fp32 pieces
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
@@ -232,7 +225,9 @@ struct mt_model {
   int32_t n_slots, n_dump;
   size_t ws_total;
 
-  std::map<std::tuple<uint64_t, int32_t, int32_t>, Plan> plans;
+  std::map<std::tuple<uint64_t, int32_t, int32_t>, Plan> plans;  // at most plan_cache entries
+  int32_t plan_cache;
+  uint64_t use_clock;
   int32_t last_batch, last_seq;
   const int32_t* last_lengths;  // device lengths of the last forward (for mt_debug_copy_hidden)
 
@@ -284,19 +279,6 @@ void layout_workspace(mt_model* m) {
   m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
   // tanh pooler outputs of the tasks of one head launch: fp32 [kMaxGroups][max_batch][H]
   m->ws_pooled = take(static_cast<size_t>(kMaxGroups) * m->max_batch * H * sizeof(float));
-  {
-    // counters of the fused layer-tail launches: every launch of a forward has its own, so one memset at
-    // the start of the forward clears them all.  Launches per forward: per wave the chunks of at most
-    // n_slots layers, plus the first-token tails (at most one more step per wave and chunk of tasks).
-    int32_t max_branch = 0;
-    for (const TaskEntry& t : m->tasks) max_branch = std::max(max_branch, t.cfg.branch_layers);
-    const size_t T = m->tasks.size();
-    const size_t per_wave = (T + 1 + std::max<int32_t>(m->max_groups, 1) - 1) / std::max<int32_t>(m->max_groups, 1) +
-                            (T + kMaxGroups - 1) / kMaxGroups;
-    const size_t launches = static_cast<size_t>(m->trunk.trunk_layers + max_branch + 1) * per_wave;
-    m->sync_bytes = launches * pad256(chain_sync_bytes(kMaxGroups, static_cast<int64_t>(M)));
-    m->ws_sync = take(m->sync_bytes);
-  }
   m->ws_trunk[0] = take(m->state_bytes);
   m->ws_trunk[1] = take(m->state_bytes);
   m->ws_task0 = off;
@@ -407,16 +389,6 @@ void choose_block_n(const mt_model* m, GemmParams* g, int epilogue, bool all_row
   g->block_n = gemm_block_n(g->N, epilogue, rows, groups < 1 ? 1 : groups, g->pair != 0, m->sm_count);
 }
 
-// Whether the part of `groups` layers after attention runs as one persistent launch (see ChainParams).  Its
-// tiles hand over to one another through global memory, two to three microseconds per hand-over and four
-// hand-overs per layer; measured on the 32 x 128 batch that costs more than the four kernel boundaries it
-// removes (which programmatic dependent launch already hides in part), so it is off unless asked for.
-bool use_fused_tail(const mt_model* m, int32_t groups) {
-  if (groups < 1 || !chain_supported(m->trunk.hidden, m->trunk.ffn)) return false;
-  if (m->fused_tail != 2) return m->fused_tail != 0;
-  return groups >= m->fused_min_groups;
-}
-
 // Whether the residual GEMMs of `groups` layers carry their LayerNorm (see GemmLnParams).
 // (mode 2: few layers in the launch; optionally also launches of few rows per layer, the first-token tails,
 // which measured 0.3 % slower that way on the 32 x 128 batch; all ways give the same bits)
@@ -426,7 +398,6 @@ bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) {
 }
 // Launches of steps 3-7 for `groups` layers.
 int32_t tail_launches(const mt_model* m, int32_t groups, int64_t rows) {
-  if (use_fused_tail(m, groups)) return 1;
   return use_fused_ln(m, groups, rows) ? 3 : 5;
 }
 
@@ -452,8 +423,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.hidden = t->ln2.hidden = H;
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
-  t->fused = use_fused_tail(m, groups);
-  t->ln_fused = !t->fused && use_fused_ln(m, groups, rows);
+  t->ln_fused = use_fused_ln(m, groups, rows);
   if (t->ln_fused) {
     auto init_ln = [&](GemmLnParams* g, int32_t K) {
       memset(g, 0, sizeof(*g));
@@ -464,23 +434,6 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
     };
     init_ln(&t->attn_out_ln, H);
     init_ln(&t->ffn_down_ln, F);
-  }
-  if (t->fused) {
-    memset(&t->chain, 0, sizeof(t->chain));
-    const GemmParams* like[3] = {&t->attn_out, &t->ffn_up, &t->ffn_down};
-    int64_t rows_used = rows;
-    if (!all_rows_valid && m->pack_tokens && m->expected_tokens > 0 && m->expected_tokens < rows) rows_used = m->expected_tokens;
-    for (int ph = 0; ph < 3; ++ph) {
-      GemmParams* g = &t->chain.gemm[ph];
-      g->M = like[ph]->M; g->N = like[ph]->N; g->K = like[ph]->K;
-      g->pair = 0;
-      g->block_n = chain_block_n(ph, g->N, rows_used, groups, m->sm_count);
-      if (m->tail_bn[ph] != 0 && g->N % m->tail_bn[ph] == 0) g->block_n = m->tail_bn[ph];
-      g->m_valid = rows_valid;
-      g->status = like[ph]->status;
-    }
-    t->chain.sync = nullptr;   // assigned by build_plan
-    t->chain.sync_blocks = (rows + kGemmBlockM - 1) / kGemmBlockM;
   }
 }
 
@@ -522,18 +475,6 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
     float* out32_home = out32 != nullptr ? out32 : f32_of(m, out);
     if ((e = set_ln(&t->attn_out_ln, ctx, lo->wo, lo->bo, lo->ln1_g, lo->ln1_b, residual, h1, h1_32)) != cudaSuccess) return e;
     if ((e = set_ln(&t->ffn_down_ln, f, lo->w2, lo->b2, lo->ln2_g, lo->ln2_b, h1_32, out, out32_home)) != cudaSuccess) return e;
-  }
-  if (t->fused) {
-    ChainParams* c = &t->chain;
-    if ((e = set_gemm_group(&c->gemm[0], i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) != cudaSuccess)
-      return e;
-    if ((e = set_gemm_group(&c->gemm[1], i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) != cudaSuccess)
-      return e;
-    if ((e = set_gemm_group(&c->gemm[2], i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) != cudaSuccess)
-      return e;
-    c->gemm[0].n_groups = c->gemm[1].n_groups = c->gemm[2].n_groups = t->count;
-    c->ln[0] = t->ln1;
-    c->ln[1] = t->ln2;
   }
   return cudaSuccess;
 }
@@ -666,16 +607,6 @@ std::vector<int32_t> cls_tasks_after_wave(const mt_model* m, const Schedule& s, 
 cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int32_t seq, Plan* plan) {
   plan->steps.clear();
   plan->launches = 2;  // row starts, embedding
-  plan->sync_bytes = 0;
-  // gives a fused layer tail its own counters
-  auto assign_sync = [&](LayerTail* t) -> cudaError_t {
-    if (!t->fused || t->count == 0) return cudaSuccess;
-    const size_t bytes = pad256(chain_sync_bytes(t->count, t->chain.gemm[0].M));
-    if (plan->sync_bytes + bytes > m->sync_bytes) return cudaErrorMemoryAllocation;
-    t->chain.sync = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_sync + plan->sync_bytes);
-    plan->sync_bytes += bytes;
-    return cudaSuccess;
-  };
   // Pooler + head of a set of tasks.  Tasks whose final state is compact ([B, H], one row per sequence:
   // the last branch layer was evaluated on first tokens only) get their pooler as one grouped GEMM on
   // the tensor cores, Y_t = tanh(X_t . Wp_t^T + bp_t) in fp32, followed by the head kernel; the others
@@ -764,7 +695,6 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
       st.kind = 0;
       cudaError_t e = build_chunk(m, ops, first, count, batch, seq, &st.chunk);
       if (e != cudaSuccess) return e;
-      if ((e = assign_sync(&st.chunk.full)) != cudaSuccess) return e;
       plan->steps.push_back(std::move(st));
       plan->launches += chunk_launches(m, ops, first, count, static_cast<int64_t>(batch) * seq);
     }
@@ -776,7 +706,6 @@ cudaError_t build_plan(const mt_model* m, const Schedule& s, int32_t batch, int3
         st.kind = 2;
         cudaError_t e = build_cls_tail(m, tasks, first, std::min<size_t>(kMaxGroups, tasks.size() - first), batch, &st);
         if (e != cudaSuccess) return e;
-        if ((e = assign_sync(&st.tail)) != cudaSuccess) return e;
         plan->launches += tail_launches(m, st.tail.count, batch);
         plan->steps.push_back(std::move(st));
       }
@@ -819,6 +748,8 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->max_batch = max_batch;
   m->max_seq = max_seq;
   m->max_groups = kMaxGroups;
+  m->plan_cache = 32;
+  m->use_clock = 0;
   m->debug_capture = false;
   m->pack_tokens = true;
   m->cls_only = true;
@@ -826,7 +757,6 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->gemm_pair = 2;
   m->attention_tc = true;
   m->expected_tokens = 0;
-  m->fused_tail = 0;
   m->pool_gemm = true;
   m->overlap_cls = true;
   m->side_stream = nullptr;
@@ -834,8 +764,6 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->fused_ln = 2;
   m->fused_ln_max_groups = 2;
   m->fused_ln_max_rows = 0;
-  m->fused_min_groups = 3;
-  m->tail_bn[0] = m->tail_bn[1] = m->tail_bn[2] = 0;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
   m->ws_bytes_bound = 0;
@@ -921,12 +849,6 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     m->expected_tokens = value;
     return MT_OK;
   }
-  if (strcmp(key, "fused_tail") == 0) {
-    if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_tail must be 0, 1 or 2");
-    m->fused_tail = static_cast<int32_t>(value);
-    m->plans.clear();
-    return MT_OK;
-  }
   if (strcmp(key, "fused_ln") == 0) {
     if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1 or 2");
     m->fused_ln = static_cast<int32_t>(value);
@@ -952,24 +874,18 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     m->plans.clear();
     return MT_OK;
   }
+  if (strcmp(key, "plan_cache") == 0) {
+    if (value < 1) return fail(m, MT_ERR_INVALID_ARG, "plan_cache must be >= 1");
+    m->plan_cache = static_cast<int32_t>(value > 4096 ? 4096 : value);
+    m->plans.clear();
+    return MT_OK;
+  }
   if (strcmp(key, "overlap_cls") == 0) {
     m->overlap_cls = value != 0;
     return MT_OK;
   }
   if (strcmp(key, "pool_gemm") == 0) {
     m->pool_gemm = value != 0;
-    m->plans.clear();
-    return MT_OK;
-  }
-  if (strcmp(key, "fused_min_groups") == 0) {
-    if (value < 1) return fail(m, MT_ERR_INVALID_ARG, "fused_min_groups must be >= 1");
-    m->fused_min_groups = static_cast<int32_t>(value);
-    m->plans.clear();
-    return MT_OK;
-  }
-  if (strncmp(key, "tail_bn", 7) == 0 && key[7] >= '0' && key[7] <= '2' && key[8] == 0) {
-    if (value != 0 && value != 128 && value != 192) return fail(m, MT_ERR_INVALID_ARG, "tail_bn must be 0, 128 or 192");
-    m->tail_bn[key[7] - '0'] = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
   }
@@ -1042,6 +958,14 @@ int mt_bind_memory(mt_model* m, void* d_weights, size_t weights_bytes, void* d_w
   for (TaskEntry& t : m->tasks) t.loaded = false;
   e = cudaMemset(m->d_workspace + m->ws_status, 0, 256);
   if (e != cudaSuccess) return fail_cuda(m, e, "clearing the status word");
+  // the stream beside the caller's (option "overlap_cls") and its fork/join events: created here, once, so
+  // that a forward never creates anything
+  if (m->side_stream == nullptr) {
+    if ((e = cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming)) != cudaSuccess)
+      return fail_cuda(m, e, "creating the side stream");
+  }
   return MT_OK;
 }
 
@@ -1122,6 +1046,8 @@ int mt_plan_summary(const mt_model* m, uint64_t task_mask, int32_t* n_layers, in
   return MT_OK;
 }
 
+int mt_plan_cache_size(const mt_model* m) { return m == nullptr ? MT_ERR_INVALID_ARG : static_cast<int>(m->plans.size()); }
+
 int mt_plan_launches(const mt_model* m, uint64_t task_mask, int32_t* n_launches) {
   if (m == nullptr || n_launches == nullptr) return MT_ERR_INVALID_ARG;
   Schedule s;
@@ -1194,9 +1120,17 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     Plan plan;
     cudaError_t e = build_plan(m, s, batch, seq, &plan);
     if (e != cudaSuccess) return fail_cuda(m, e, "building the launch plan");
+    // a plan holds hundreds of tensor maps: keep the most recently used ones only
+    while (static_cast<int32_t>(m->plans.size()) >= m->plan_cache) {
+      auto oldest = m->plans.begin();
+      for (auto p = m->plans.begin(); p != m->plans.end(); ++p)
+        if (p->second.last_use < oldest->second.last_use) oldest = p;
+      m->plans.erase(oldest);
+    }
     it = m->plans.emplace(key, std::move(plan)).first;
   }
   Plan& plan = it->second;
+  plan.last_use = ++m->use_clock;
   uint32_t* status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   const size_t act_used = static_cast<size_t>(batch) * seq * m->trunk.hidden * sizeof(bf16);
   cudaError_t e;
@@ -1224,13 +1158,11 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     }                                                                                        \
   } while (0)
 
-  // Steps 3-7 of the layers of a wave: one persistent launch, or the five separate ones.
+  // Steps 3-7 of the layers of a wave: three launches (each residual GEMM carries its LayerNorm) or five.
 #define MT_TAIL(tail)                                                                                                  \
   do {                                                                                                                 \
     LayerTail* t_ = (tail);                                                                                            \
-    if (t_->fused) {                                                                                                   \
-      MT_TIMED(MT_CLASS_TAIL, launch_chain(t_->chain, m->sm_count, stream), "fused layer-tail kernel");                \
-    } else if (t_->ln_fused) {                                                                                         \
+    if (t_->ln_fused) {                                                                                         \
       MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm_ln(t_->attn_out_ln, stream), "attention output GEMM + LayerNorm");       \
       MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");            \
       MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm_ln(t_->ffn_down_ln, stream), "FFN down GEMM + LayerNorm");               \
@@ -1243,8 +1175,6 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     }                                                                                                                  \
   } while (0)
 
-  if (plan.sync_bytes > 0)
-    MT_LAUNCH(cudaMemsetAsync(m->d_workspace + m->ws_sync, 0, plan.sync_bytes, stream), "clearing the tile counters");
   int32_t* row_start = reinterpret_cast<int32_t*>(m->d_workspace + m->ws_row_start);
   MT_LAUNCH(launch_row_starts(d_lengths, batch, seq, m->pack_tokens ? 1 : 0, row_start,
                               reinterpret_cast<int32_t*>(m->d_workspace + m->ws_rows_valid), stream),
@@ -1275,13 +1205,8 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
       ck.attn.lengths = d_lengths;
       ck.attn_cls.lengths = d_lengths;
       MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
-      const bool beside = m->overlap_cls && !m->profile && ck.n_cls > 0 && ck.full.count > 0;
+      const bool beside = m->overlap_cls && m->side_stream != nullptr && !m->profile && ck.n_cls > 0 && ck.full.count > 0;
       if (beside) {
-        if (m->side_stream == nullptr) {
-          MT_LAUNCH(cudaStreamCreateWithFlags(&m->side_stream, cudaStreamNonBlocking), "creating the side stream");
-          MT_LAUNCH(cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming), "creating an event");
-          MT_LAUNCH(cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming), "creating an event");
-        }
         MT_LAUNCH(cudaEventRecord(m->ev_fork, stream), "forking the side stream");
         MT_LAUNCH(cudaStreamWaitEvent(m->side_stream, m->ev_fork, 0), "forking the side stream");
         MT_LAUNCH(launch_cls_attention(ck.attn_cls, m->side_stream), "first-token attention kernel");
@@ -1416,12 +1341,14 @@ int mt_debug_copy_hidden(mt_model* m, int32_t task, int32_t layer, void* d_out, 
       reinterpret_cast<const bf16*>(m->d_workspace + m->ws_dump0 + m->act_bytes * dump_slot(m, task, layer)),
       m->last_lengths, reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_row_start),
       static_cast<bf16*>(d_out), m->last_batch, m->last_seq, m->trunk.hidden,
-      (m->cls_only && task >= 0 && layer == m->tasks[task].cfg.branch_layers) ? 1 : 0, as_stream(stream_));
+      (task >= 0 && is_compact_task(m, task) && layer == m->tasks[task].cfg.branch_layers) ? 1 : 0, as_stream(stream_));
   if (e != cudaSuccess) return fail_cuda(m, e, "copying a captured hidden state");
   return MT_OK;
 }
 
 // ---- single steps ------------------------------------------------------------------------------
+
+void mt_kernel_linear_force_block_n(int32_t block_n) { g_force_block_n = block_n; }
 
 int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual, void* d_y, int32_t M,
                      int32_t N, int32_t K, int32_t epilogue, int32_t cta_pair, uint32_t* d_status, void* stream) {
@@ -1437,6 +1364,7 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
   p.pair = cta_pair != 0 ? 1 : 0;
   p.block_n = gemm_block_n(N, epilogue, M, 1, p.pair != 0, sms);
+  if (g_force_block_n > 0 && N % g_force_block_n == 0) p.block_n = g_force_block_n;
   if (set_gemm_group(&p, 0, epilogue, d_x, d_w, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
                      d_y) != cudaSuccess)
     return MT_ERR_CUDA;

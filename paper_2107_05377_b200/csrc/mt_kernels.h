@@ -144,31 +144,6 @@ struct LayerNormParams {
 };
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream);
 
-// Steps 3-7 of the encoder layer for the layers of one wave in ONE persistent launch:
-//   phase 0  u  = ctx . Wo^T + bo + x        (fp32)      then h1  = LN(u)   per block of 128 rows
-//   phase 1  f  = GELU(h1 . W1^T + b1)       (bf16)
-//   phase 2  u  = f . W2^T + b2 + h1         (fp32)      then out = LN(u)   per block of 128 rows
-// The tiles of all three GEMMs form one ordered list that the CTAs walk through; a tile waits (bounded)
-// on counters in global memory until the row block it reads has been produced by earlier tiles, and
-// warps set aside for it normalise the rows of a row block of phase 0 or 2 once all its tiles have arrived.  `sync` points at 4 zeroed words
-// per (group, row block): arrivals of phase 0, "h1 ready", arrivals of phase 1, arrivals of phase 2.
-// The arithmetic of every element is that of launch_gemm / launch_layernorm, so the results are
-// bit-identical to the five separate launches.
-constexpr int kChainMaxBlockN = 192;   // widest tile of the fused kernel (its stages hold 128 + 192 rows)
-struct alignas(64) ChainParams {
-  GemmParams gemm[3];        // attn_out, ffn_up, ffn_down: same M, m_valid, n_groups; pair = 0; block_n <= 192
-  LayerNormParams ln[2];     // after phase 0 and after phase 2
-  uint32_t* sync;            // [n_groups][sync_blocks][4], zero before the launch
-  int32_t sync_blocks;       // row blocks per group the sync array is laid out for (>= ceil(M / 128))
-};
-// Bytes of `sync` for a launch of `groups` layers over `rows` rows.
-size_t chain_sync_bytes(int groups, int64_t rows);
-// Whether the fused kernel handles this shape (hidden 768 or 1024, tile widths that divide N).
-bool chain_supported(int hidden, int ffn);
-// Tile width of phase `phase` (0..2) for output width N.
-int chain_block_n(int phase, int N, int64_t rows, int groups, int sm_count);
-cudaError_t launch_chain(const ChainParams& p, int sm_count, cudaStream_t stream);
-
 // Residual GEMM with the LayerNorm that follows it, in one launch:
 //   Y_g = LN( X_g[M,K] . W_g[N,K]^T + bias_g + residual_g ) * gamma_g + beta_g      N = hidden
 // written twice, bf16 (the next GEMM's operand) and fp32 (the next residual).  The N / 128 CTAs that hold

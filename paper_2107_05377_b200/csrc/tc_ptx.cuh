@@ -216,7 +216,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v 
 // precision.  Seven arithmetic instructions and two special-function ones (ex2, rcp) per element: the
 // epilogue of the FFN-up projection is bound by instruction issue, not by the accumulator loads.
 // The coefficients carry the factor -2 log2(e) so that the exponential is a bare ex2.
-__device__ __forceinline__ float gelu_erf(float x) {
+__device__ __forceinline__ float gelu_fitted(float x) {
   constexpr float kScale = -2.0f * 1.4426950408889634f;
   constexpr float a = 0.7975078774044234f * kScale;
   constexpr float b = 0.03700565178082531f * kScale;

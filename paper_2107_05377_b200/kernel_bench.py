@@ -138,6 +138,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--flush", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
+    ap.add_argument("--block-n", type=int, default=0, help="linear: force the tile width (0 = automatic)")
     ap.add_argument("--pair", action="store_true", help="linear: pairs of CTAs on 256-row tiles (cta_group::2)")
     ap.add_argument("--mma-sync", action="store_true", help="attention: the mma.sync kernel also where seq <= 128")
     a = ap.parse_args()
@@ -145,6 +146,7 @@ def main():
     USE_GRAPH = a.graph
     CTA_PAIR = a.pair
     TENSOR_MEMORY = not a.mma_sync
+    mt.lib().mt_kernel_linear_force_block_n(a.block_n)
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
@@ -155,7 +157,7 @@ def main():
     elif a.kernel == "layernorm":
         print(json.dumps(bench_layernorm(a.rows, a.hidden, a.iters, a.warmup, a.flush)))
     else:
-        for m in (4096, 24576):   # one layer, and six layers' worth of rows
+        for m in (2409, 4096, 24576):   # the valid tokens of the 32 x 128 batch, its padded rows, six layers of them
             for (n, k, e) in ((2304, 768, 0), (768, 768, 2), (3072, 768, 1), (768, 3072, 2)):
                 print(json.dumps(bench_linear(m, n, k, e, a.iters, a.warmup, a.flush)))
             for (n, k) in ((768, 768), (768, 3072)):

@@ -17,16 +17,11 @@ LOGIT_MAX_ABS = 2e-2   # tolerance on logits
 
 
 def run_model(cfg, blob, batch, mask=None, max_groups=None, debug=False, fill=None, pack_tokens=None, cls_only=None,
-              gemm_pair=None, attention_tc=None, expected_tokens=None, fused_tail=None, tail_bn=None, fused_ln=None):
+              gemm_pair=None, attention_tc=None, expected_tokens=None, fused_ln=None):
     B, S = batch.token_ids.shape
     model = mt.MTModel(cfg, B, S, max_groups=max_groups, debug_capture=debug)
     if fused_ln is not None:
         model.set_option("fused_ln", fused_ln)
-    if fused_tail is not None:
-        model.set_option("fused_tail", fused_tail)
-    if tail_bn is not None:
-        for i, bn in enumerate(tail_bn):
-            model.set_option(f"tail_bn{i}", bn)
     if attention_tc is not None:
         model.set_option("attention_tc", attention_tc)
     if expected_tokens is not None:
@@ -151,45 +146,6 @@ def test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches():
     torch.cuda.synchronize()
     assert m8.poll_status() == 0
     assert torch.equal(again, first)
-    check_against_oracle(big, wf8, b8, m8, again, rows=[0, 13, 31], check_hidden=False)
-
-
-def test_fused_layer_tail_matches_oracle_and_separate_launches_bits():
-    """The part of a layer after attention as one persistent launch per wave (option "fused_tail", the
-    default) against the five separate launches: every element is the same arithmetic, so hidden
-    states and logits are bit-identical, for every tile-width choice; and both match the oracle."""
-    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
-                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
-    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
-    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
-    m_sep, separate = run_model(cfg, blob, batch, debug=True, fused_tail=0, fused_ln=0)
-    m_fus, fused = run_model(cfg, blob, batch, debug=True, fused_tail=1)
-    check_against_oracle(cfg, wf, batch, m_fus, fused, rows=range(6))
-    assert torch.equal(fused, separate)
-    B, S = batch.token_ids.shape
-    for t, layer in ((-1, 1), (-1, 3), (1, 1), (1, 2), (3, 1)):
-        assert torch.equal(m_fus.debug_hidden(t, layer, B, S), m_sep.debug_hidden(t, layer, B, S)), (t, layer)
-    for bn in ((128, 128, 128), (192, 192, 192), (192, 128, 192)):
-        _, got = run_model(cfg, blob, batch, fused_tail=1, tail_bn=bn)
-        assert torch.equal(got, separate), bn
-    # every token in the last branch layers too (more rows in the fused launches), and the padded layout
-    _, full_sep = run_model(cfg, blob, batch, cls_only=0, pack_tokens=0, fused_tail=0, fused_ln=0)
-    _, full_fus = run_model(cfg, blob, batch, cls_only=0, pack_tokens=0, fused_tail=1)
-    assert torch.equal(full_fus, full_sep)
-    big = synth.config_glue8()
-    w8, blob8, wf8 = cached_weights(big, 0)
-    b8 = synth.batch_glue8(big)
-    _, s8 = run_model(big, blob8, b8, fused_tail=0, fused_ln=0)
-    for _ in range(3):   # repeated forwards reuse the counters after the memset
-        m8, f8 = run_model(big, blob8, b8, fused_tail=1)
-        assert torch.equal(f8, s8)
-    tok, seg, lens = dev_batch(b8)
-    again = torch.zeros_like(f8)
-    for _ in range(4):
-        m8.forward(tok, seg, lens, again)
-    torch.cuda.synchronize()
-    assert m8.poll_status() == 0
-    assert torch.equal(again, s8)
     check_against_oracle(big, wf8, b8, m8, again, rows=[0, 13, 31], check_hidden=False)
 
 
@@ -584,3 +540,98 @@ def test_two_batches_in_flight_over_one_weights_arena():
     other = mt.MTModel(synth.config_tiny(), 2, 32)
     with pytest.raises(mt.MTError):
         mt._check(mt.lib().mt_adopt_weights(other.handle, first.handle), "mt_adopt_weights", other.handle)
+
+
+def test_bad_lengths_are_clamped_the_same_way_by_every_kernel():
+    """A length of 0 or beyond seq is flagged and clamped to [1, seq] by every kernel of the path: logits are
+    finite and both attention kernels, and both token layouts, agree to rounding."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 5, 100, 1, 100, seed=9)
+    lengths = batch.lengths.copy()
+    lengths[1], lengths[3] = 0, 1000
+    bad = synth.Batch(batch.token_ids, batch.segment_ids, lengths)
+    B, S = bad.token_ids.shape
+    outs = {}
+    for tc in (1, 0):
+        for pack in (1, 0):
+            model = mt.MTModel(cfg, B, S)
+            model.set_option("attention_tc", tc)
+            model.set_option("pack_tokens", pack)
+            model.load_weights(blob)
+            logits = torch.full((B, cfg.total_classes), float("nan"), device="cuda")
+            model.forward(*dev_batch(bad), logits)
+            torch.cuda.synchronize()
+            assert model.poll_status() == mt.FLAG_BAD_LENGTH
+            assert torch.isfinite(logits).all()
+            outs[(tc, pack)] = logits
+    base = outs[(1, 1)]
+    for key, got in outs.items():
+        assert float((got - base).abs().max()) <= 3e-3, key
+    # the clamped lengths are what the oracle sees
+    clamped = synth.Batch(batch.token_ids, batch.segment_ids, np.clip(lengths, 1, S).astype(np.int32))
+    want = orc.forward_batch_mt(clamped.token_ids, clamped.segment_ids, clamped.lengths, wf, task_triples(cfg),
+                                cfg.heads, cfg.ln_eps)
+    assert np.max(np.abs(base.cpu().numpy().astype(np.float64) - want)) <= LOGIT_MAX_ABS
+
+
+def test_task_reload_on_a_second_stream_while_other_tasks_are_served():
+    """Sections 1 and 5.1, Appendix E: a task is replaced while the model keeps serving the others.  Forwards
+    whose mask excludes task 1 run on one stream while task 1's weights are copied in on another; the other
+    tasks' logits keep their bits, and afterwards task 1 answers with the new weights."""
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 16, 128, 20, 128, seed=2)
+    model, base = run_model(cfg, blob, batch)
+    new_task = synth.make_task_weights(cfg, 1, seed=78)
+    task_blob = torch.from_numpy(synth.pack_task_weights(cfg, 1, new_task)).pin_memory()
+    tok, seg, lens = dev_batch(batch)
+    serve, load = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = [torch.full_like(base, -7.0) for _ in range(12)]
+    for i, out in enumerate(outs):
+        model.forward(tok, seg, lens, out, task_mask=0b101, stream=serve)
+        if i == 3:
+            mt._check(mt.lib().mt_load_task_weights(model.handle, 1, task_blob.data_ptr(), task_blob.numel(),
+                                                    load.cuda_stream), "mt_load_task_weights", model.handle)
+    torch.cuda.synchronize()
+    assert model.poll_status() == 0
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    for out in outs:
+        assert torch.equal(out[:, offs[0]:offs[1]], base[:, offs[0]:offs[1]])
+        assert torch.equal(out[:, offs[2]:offs[3]], base[:, offs[2]:offs[3]])
+        assert torch.all(out[:, offs[1]:offs[2]] == -7.0)
+    after = torch.empty_like(base)
+    model.forward(tok, seg, lens, after)
+    torch.cuda.synchronize()
+    assert torch.equal(after[:, offs[0]:offs[1]], base[:, offs[0]:offs[1]])
+    wf2 = dict(wf)
+    wf2["tasks"] = list(wf["tasks"])
+    wf2["tasks"][1] = synth.widen(new_task)
+    check_against_oracle(cfg, wf2, batch, model, after, rows=[0, 7], check_hidden=False)
+
+
+def test_plan_cache_is_bounded_and_evicts_the_least_recently_used():
+    """More distinct (mask, batch, seq) keys than the cache holds: the count stays at the cap, an evicted
+    plan is rebuilt on its next use and every result keeps its bits."""
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 3, 64, 20, 64, seed=2)
+    model, base = run_model(cfg, blob, batch)
+    model.set_option("plan_cache", 3)
+    assert model.plan_cache_size() == 0
+    tok, seg, lens = dev_batch(batch)
+    masks = [0b111, 0b001, 0b010, 0b100, 0b011, 0b111, 0b110, 0b001]
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    for i, mask in enumerate(masks):
+        out = torch.full_like(base, -3.0)
+        model.forward(tok, seg, lens, out, task_mask=mask)
+        torch.cuda.synchronize()
+        assert model.plan_cache_size() == min(i + 1, 3)
+        for t in range(3):
+            cols = slice(offs[t], offs[t + 1])
+            assert torch.equal(out[:, cols], base[:, cols]) if (mask >> t) & 1 else torch.all(out[:, cols] == -3.0)
+    assert model.poll_status() == 0

@@ -128,7 +128,8 @@ def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
     (6, 128, 12, [128, 37, 1, 64, 65, 127], True),
     (3, 100, 2, [100, 65, 9], True),        # the 128-row tile reaches into the next sequence and past the buffer
     (1, 1, 1, [1], True),
-    (5, 128, 16, [0, 128, 0, 16, 113], True),   # empty sequences
+    (5, 128, 16, [0, 128, 0, 16, 113], True),   # a length of 0 is clamped to 1, as by every kernel of the path
+    (5, 128, 16, [0, 128, 0, 16, 113], False),
 ])
 def test_attention_matches_oracle(B, S, heads, lengths, tensor_memory):
     H = heads * 64
@@ -136,6 +137,7 @@ def test_attention_matches_oracle(B, S, heads, lengths, tensor_memory):
     # poison the padded rows of the input: they must not leak into valid rows
     qkv_dev = to_dev_bf16(qb)
     lens = torch.tensor(lengths, dtype=torch.int32, device="cuda")
+    lengths = [max(n, 1) for n in lengths]
     for b, n in enumerate(lengths):
         qkv_dev[b * S + n:(b + 1) * S] = float("nan")
     ctx = torch.full((B * S, H), float("nan"), dtype=torch.bfloat16, device="cuda")
@@ -229,3 +231,23 @@ def test_pooler_head_matches_oracle(B, S, H, C):
         want = orc.pooler_head(h[i * S:(i + 1) * S], tw)
         assert np.max(np.abs(got[i, 2:2 + C] - want)) <= 1e-4
     assert np.all(got[:, :2] == -77.0) and np.all(got[:, 2 + C:] == -77.0), "other tasks' columns must be untouched"
+
+
+def test_gelu_epilogue_stays_within_its_stated_fit_error():
+    """The FFN-up epilogue evaluates the exact-form GELU x * Phi(x) through a fitted sigmoid argument whose
+    stated largest absolute error is 2.6e-5; the result is then rounded once to bf16.  Pre-activations on a
+    grid over [-8, 8] are produced exactly (one non-zero weight of 1 per output, zero bias)."""
+    M, N, K = 128, 128, 64
+    grid = np.linspace(-8.0, 8.0, M * K, dtype=np.float32).reshape(M, K)
+    xb = synth.f32_to_bf16_bits(grid)
+    x = synth.bf16_bits_to_f64(xb)
+    w = np.zeros((N, K), dtype=np.float32)
+    w[np.arange(N), np.arange(N) % K] = 1.0          # output n of row m is x[m, n % 64]
+    y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    mt.mt_kernel_linear(to_dev_bf16(xb), to_dev_bf16(synth.f32_to_bf16_bits(w)),
+                        to_dev_bf16(synth.f32_to_bf16_bits(np.zeros(N, dtype=np.float32))), None, y, 1)
+    torch.cuda.synchronize()
+    got = dev_bf16_to_f64(y)
+    want = orc.gelu(x[:, np.arange(N) % K])
+    half_ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 1e-30))) - 8)
+    assert np.all(np.abs(got - want) <= 2.6e-5 + half_ulp + 1e-9)

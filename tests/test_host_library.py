@@ -92,14 +92,6 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     m.set_option("fused_ln_max_rows", 128)   # also the first-token tail (32 rows per layer)
     assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 3 + 2
     m.set_option("fused_ln", 0)
-    # fused_tail = 1: the part of a layer after attention is one launch, so a wave is projection + attention
-    # + fused tail (+ first-token attention where a branch ends); one fused first-token tail; pooler + head
-    m.set_option("fused_tail", 1)
-    assert m.plan_launches(0xFF) == 2 + 3 * 6 + 4 * 3 + 2 + 1 + 2
-    # fused_tail = 2: fused where at least three layers share the launch: waves 6, 7, 8 and the first-token tail
-    m.set_option("fused_tail", 2)
-    assert m.plan_launches(0xFF) == 2 + 7 * 5 + 3 + 4 + 4 + 8 + 2 + 1 + 2
-    m.set_option("fused_tail", 0)   # the default
     # waves 7, 8, 9 mix layers on all tokens (7 launches) with last branch layers, which only add the
     # first-token attention there; wave 10 holds a last layer alone (projection + first-token attention);
     # the rest of the eight last layers is one grouped pass of 5 launches before the pooler/head pair
