@@ -39,11 +39,27 @@ N_INPUT_BATCHES = 4
 REFERENCE_SAMPLE = 8          # sequences per step of the oracle arm
 L2_FLUSH_BYTES = 256 << 20    # larger than the 126 MB L2
 
-# DRAM traffic of the dominant kernel from one ncu capture (bytes per launch, averaged over the GEMM
-# launches of the forwards of `bench.py --steps 2`), valid only for the kernel sources it was taken on.
+# DRAM traffic of the dominant kernel comes from one ncu capture (bytes per launch, averaged over the GEMM
+# launches of the forwards of `bench.py --steps 2`); the figure and the digest of the kernel sources it was
+# taken on are two lines of the launch-list summary under profiles/, and it is reported only while the
+# sources still have that digest.
 GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_ln_tcgen05.cu", "tc_ptx.cuh", "rowwise.cuh")
-NCU_TRAFFIC = {"gemm_sources_sha256": "1457216e3c5239c21e5e0f4e4d50ef58209ed737064abc18998f6314587531a7",
-               "bytes_per_launch": 25192291}  # profiles/bench_glue8_b32_s128_launch_list.md
+TRAFFIC_SUMMARY = os.path.join("profiles", "bench_glue8_b32_s128_launch_list.md")
+NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16 of the part, for context beside the measured peak
+STEADY_SECONDS = 2.0
+
+
+def ncu_traffic():
+    """(digest, bytes per GEMM launch) as recorded in the launch-list summary, or (None, None)."""
+    import re
+    try:
+        with open(os.path.join(ROOT, TRAFFIC_SUMMARY)) as f:
+            text = f.read()
+    except OSError:
+        return None, None
+    d = re.search(r"gemm_sources_sha256:\s*`?([0-9a-f]{64})", text)
+    b = re.search(r"gemm_dram_bytes_per_launch:\s*`?(\d+)", text)
+    return (d.group(1), int(b.group(1))) if d and b else (None, None)
 
 
 def gemm_sources_digest():
@@ -301,6 +317,27 @@ def main():
     total_ms = sum(step_ms)
     assert model.poll_status() == 0, "device status word set during the timed region"
 
+    # steady state: at least STEADY_SECONDS of forwards back to back (graph replays, no flush: a forward streams
+    # 340 MB of weights, more than L2), one timed region, with clock samples of its own - whatever --steps is,
+    # the record shows sustained behaviour
+    steady = None
+    if graphs is not None:
+        reps = max(int(STEADY_SECONDS * 1e3 / (total_ms / args.steps)) + 1, args.steps)
+        steady_sampler = ClockSampler(local_rank) if rank == 0 else None
+        t_s, t_e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync_all()
+        t_s.record(stream)
+        for i in range(reps):
+            graphs[i % N_INPUT_BATCHES].replay()
+        t_e.record(stream)
+        sync_all()
+        steady_ms = max_over_ranks([t_s.elapsed_time(t_e)], device)[0]
+        steady = {"value": aggregate_throughput(world, BATCH, reps, steady_ms * 1e-3), "unit": UNIT, "steps": reps,
+                  "ms_per_step": steady_ms / reps, "seconds": steady_ms * 1e-3,
+                  "how": "forwards back to back on one stream, one timed region, no L2 flush",
+                  "clocks": steady_sampler.stop() if steady_sampler else None}
+        assert model.poll_status() == 0, "device status word set during the steady-state leg"
+
     # end to end through the host entry point: pinned host inputs -> device, forward, logits -> pinned host
     # buffer, and the host waits for every step's logits before it issues the next step.  Eagerly:
     # mt_forward_host.  Otherwise the same call without its final wait (mt_forward_host_async) is
@@ -389,7 +426,8 @@ def main():
         n_first = sum(1 for t in cfg.tasks if t.branch_layers > 0)   # last branch layers: first token only
         gemm_flops = sum(gemm_flops_per_forward(cfg, plan["layers"], t, n_first, BATCH) for t in step_tokens)
         achieved = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
-        traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["gemm_sources_sha256"] == gemm_sources_digest() else None
+        traffic_digest, traffic_bytes = ncu_traffic()
+        traffic = traffic_bytes if traffic_digest == gemm_sources_digest() else None
         valid_tokens = float(np.mean(step_tokens))
         padded_flops = gemm_flops_per_forward(cfg, plan["layers"], m_rows) + \
             plan["layers"] * BATCH * 4.0 * cfg.hidden * SEQ * SEQ
@@ -415,13 +453,22 @@ def main():
             "e2e": {"value": aggregate_throughput(world, BATCH, args.steps, e2e_s), "unit": UNIT,
                     "h2d_bytes_per_step": 2 * BATCH * SEQ * 4 + BATCH * 4,
                     "d2h_bytes_per_step": BATCH * cfg.total_classes * 4},
-            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 and gemm_ln_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches; where a "
-                                   "single layer is in the launch the two residual GEMMs include the LayerNorm after them)",
+            "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05 and gemm_ln_tcgen05 (QKV, attention-out, FFN-up, FFN-down launches; the two "
+                                   "residual GEMMs include the LayerNorm after them)",
                          "flops": "valid tokens only; the last layer of each branch counts its Q/K/V projection on all "
                                   "tokens and the rest on one token per sequence",
                          "achieved": achieved, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                         "frac": achieved / peaks["tflops"], "peak_source": peaks["source"], "traffic": traffic,
+                         "frac": achieved / peaks["tflops"], "peak_source": peaks["source"],
+                         "peak_nominal": NOMINAL_BF16_TFLOPS, "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+                         "traffic": traffic,
                          "launches": int(gemm_launches), "avg_launch_us": 1e3 * gemm_ms / max(gemm_launches, 1)},
+            "roofline_forward": {"what": "all algorithmic FLOPs of a forward (GEMMs and attention, valid tokens only) over "
+                                         "the whole step time, every kernel and every launch gap included",
+                                 "achieved": valid_flops / (total_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                                 "peak": peaks["tflops"], "frac": valid_flops / (total_ms * 1e-3) / 1e12 / peaks["tflops"],
+                                 "peak_source": peaks["source"], "peak_nominal": NOMINAL_BF16_TFLOPS,
+                                 "frac_of_nominal": valid_flops / (total_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
+            "steady_state": steady,
             "forward_tflops_valid": valid_flops / (total_ms * 1e-3) / 1e12,
             "forward_tflops_padded_equivalent": padded_flops * args.steps / (total_ms * 1e-3) / 1e12,
             "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
