@@ -541,8 +541,8 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
       ck->attn.ctx[a] = ctx;
       ck->attn.n_groups = a + 1;
       if (ck->attn.tensor_memory &&
-          ((e = make_tmap(&ck->attn.tmap_qkv[a], qkv, M, 3 * H, kAttnTensorMemoryMaxSeq, kHeadDim, false)) != cudaSuccess ||
-           (e = make_tmap(&ck->attn.tmap_qkv64[a], qkv, M, 3 * H, kAttnTensorMemoryMaxSeq / 2, kHeadDim, false)) != cudaSuccess))
+          ((e = make_tmap(&ck->attn.tmap_qkv[a], qkv, M, 3 * H, kAttnTileRows, kHeadDim, false)) != cudaSuccess ||
+           (e = make_tmap(&ck->attn.tmap_qkv64[a], qkv, M, 3 * H, kAttnTileRows / 2, kHeadDim, false)) != cudaSuccess))
         return e;
       if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f32_of(m, h1), f, out, f32_of(m, out))) !=
           cudaSuccess)
@@ -1408,9 +1408,9 @@ int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx
   if (tensor_memory != 0) {
     p.tensor_memory = 1;
     if (make_tmap(&p.tmap_qkv[0], d_qkv, static_cast<int64_t>(batch) * seq, 3 * static_cast<int64_t>(heads) * kHeadDim,
-                  kAttnTensorMemoryMaxSeq, kHeadDim, false) != cudaSuccess ||
+                  kAttnTileRows, kHeadDim, false) != cudaSuccess ||
         make_tmap(&p.tmap_qkv64[0], d_qkv, static_cast<int64_t>(batch) * seq, 3 * static_cast<int64_t>(heads) * kHeadDim,
-                  kAttnTensorMemoryMaxSeq / 2, kHeadDim, false) != cudaSuccess)
+                  kAttnTileRows / 2, kHeadDim, false) != cudaSuccess)
       return MT_ERR_CUDA;
   }
   return launch_attention(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;

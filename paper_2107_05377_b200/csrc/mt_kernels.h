@@ -111,8 +111,10 @@ struct alignas(64) AttnParams {
   int32_t tensor_memory;        // 1: the tcgen05 kernel (seq <= 128, tmap_qkv filled); 0: the mma.sync kernel
   uint32_t* status;             // sticky device status word (may be null)
 };
-// Longest sequence the tensor-memory attention kernel handles (one CTA holds all keys of a sequence).
-constexpr int kAttnTensorMemoryMaxSeq = 128;
+// Longest sequence the tensor-memory attention kernels handle (up to 128 tokens: one CTA holds all keys of a
+// sequence; longer: tiles of 128 queries walk the keys in tiles of 128).
+constexpr int kAttnTensorMemoryMaxSeq = 512;
+constexpr int kAttnTileRows = 128;   // rows of the Q/K/V boxes of the tensor maps
 cudaError_t launch_attention(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attention_tc(const AttnParams& p, cudaStream_t stream);
 

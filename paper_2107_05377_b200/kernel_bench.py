@@ -102,7 +102,7 @@ def bench_attention(batch, seq, heads, len_lo, iters, warmup, flush):
     qkv = torch.randn(batch * seq, 3 * hidden, device="cuda").to(torch.bfloat16)
     lengths = torch.randint(len_lo, seq + 1, (batch,), device="cuda", dtype=torch.int32)
     ctx = torch.empty(batch * seq, hidden, device="cuda", dtype=torch.bfloat16)
-    ms = _time(lambda: mt.mt_kernel_attention(qkv, lengths, ctx, batch, seq, heads, tensor_memory=TENSOR_MEMORY and seq <= 128), iters, warmup, flush)
+    ms = _time(lambda: mt.mt_kernel_attention(qkv, lengths, ctx, batch, seq, heads, tensor_memory=TENSOR_MEMORY and seq <= 512), iters, warmup, flush)
     bytes_ = 2.0 * 4 * batch * seq * hidden
     n = lengths.double()
     flops = float((4.0 * hidden * n * n).sum())

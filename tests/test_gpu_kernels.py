@@ -130,6 +130,9 @@ def oracle_attention_from_qkv(qkv, lengths, B, S, heads):
     (1, 1, 1, [1], True),
     (5, 128, 16, [0, 128, 0, 16, 113], True),   # a length of 0 is clamped to 1, as by every kernel of the path
     (5, 128, 16, [0, 128, 0, 16, 113], False),
+    (2, 512, 16, [512, 300], True),           # more than 128 tokens: tiles of 128 queries walk tiles of 128 keys
+    (3, 200, 2, [200, 129, 64], True),        # seq not a multiple of the tile; one key in the second tile
+    (5, 384, 12, [1, 128, 257, 384, 0], True),
 ])
 def test_attention_matches_oracle(B, S, heads, lengths, tensor_memory):
     H = heads * 64
