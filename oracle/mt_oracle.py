@@ -159,7 +159,7 @@ class LayerCounter:
 def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weights: Dict,
                         tasks: Sequence[TaskTriple], heads: int, eps: float,
                         task_mask: Optional[int] = None, hidden_out: Optional[Dict] = None,
-                        counter: Optional[LayerCounter] = None) -> Dict[int, np.ndarray]:
+                        counter: Optional[LayerCounter] = None, layer_fn=None) -> Dict[int, np.ndarray]:
     """Merged multi-task forward of ONE sequence with ``n`` valid tokens.
 
     The trunk is evaluated once up to D = max fork depth over the active
@@ -167,7 +167,9 @@ def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weight
     each active task runs its branch from its fork state.  Returns
     {task: logits[C_t]}.  ``hidden_out`` (if given) receives
     ("trunk", depth) -> [n, H] for every depth 0..D and ("task", t, j) ->
-    [n, H] after branch layer j (1-based) of task t."""
+    [n, H] after branch layer j (1-based) of task t.  ``layer_fn`` replaces encoder_layer (same
+    signature) for variants of the layer arithmetic, such as the reduced-precision one."""
+    layer_fn = layer_fn or encoder_layer
     act = active_tasks(len(tasks), task_mask)
     if not act:
         raise ValueError("task_mask selects no task")
@@ -183,7 +185,7 @@ def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weight
     if hidden_out is not None:
         hidden_out[("trunk", 0)] = h
     for l in range(1, depth + 1):
-        h = encoder_layer(h, weights["trunk"][l - 1], heads, eps)
+        h = layer_fn(h, weights["trunk"][l - 1], heads, eps)
         if counter is not None:
             counter.count += 1
         if l in fork_depths:
@@ -196,7 +198,7 @@ def forward_sequence_mt(tokens: np.ndarray, segments: np.ndarray, n: int, weight
         x, y = tasks[t][0], tasks[t][1]
         g = forks[x]
         for j in range(1, y + 1):
-            g = encoder_layer(g, weights["tasks"][t]["layers"][j - 1], heads, eps)
+            g = layer_fn(g, weights["tasks"][t]["layers"][j - 1], heads, eps)
             if counter is not None:
                 counter.count += 1
             if hidden_out is not None:
@@ -228,7 +230,7 @@ def forward_batch_mt(token_ids: np.ndarray, segment_ids: np.ndarray, lengths: np
                      tasks: Sequence[TaskTriple], heads: int, eps: float,
                      task_mask: Optional[int] = None, rows: Optional[Iterable[int]] = None,
                      hidden_out: Optional[List[Dict]] = None,
-                     token_logits_out: Optional[List[np.ndarray]] = None) -> np.ndarray:
+                     token_logits_out: Optional[List[np.ndarray]] = None, layer_fn=None) -> np.ndarray:
     """Merged forward of a padded batch.  Returns float64 logits
     [B, sum C_t over the sequence-level tasks]; task t occupies columns
     [off_t, off_t + C_t); columns of inactive tasks and rows not in ``rows``
@@ -247,7 +249,7 @@ def forward_batch_mt(token_ids: np.ndarray, segment_ids: np.ndarray, lengths: np
     for b in (range(B) if rows is None else rows):
         hid = {} if hidden_out is not None else None
         res = forward_sequence_mt(token_ids[b], segment_ids[b], int(lengths[b]), weights, tasks, heads, eps,
-                                  task_mask=task_mask, hidden_out=hid)
+                                  task_mask=task_mask, hidden_out=hid, layer_fn=layer_fn)
         for t, lg in res.items():
             if head_kind(tasks[t]) == 1:
                 token_logits[b, :lg.shape[0], tok_offs[t]:tok_offs[t + 1]] = lg
