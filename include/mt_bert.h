@@ -299,6 +299,20 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
  * result: every output element is one fixed-order sum over K whatever the tile. */
 void mt_kernel_linear_force_block_n(int32_t block_n);
 
+/* Reduced precision (Appendix E: the production model ran at reduced precision; the paper gives no recipe, the
+ * reading here is 8-bit E4M3 operands with one fp32 scale per operand row).  Row-wise quantisation of a bf16
+ * matrix X[rows, cols] (cols % 256 == 0): d_scale[r] = max|X[r,:]| / 448 (1 for a row of zeros), d_q[r,c] = the
+ * E4M3 value nearest to X[r,c] / d_scale[r] (ties to even, saturating at +-448), decided in fp32.  Used for
+ * activations (a scale per token) and, once at load time, for weights [N, K] (a scale per output channel). */
+int mt_kernel_quantize_rows(const void* d_x, void* d_q, float* d_scale, int32_t rows, int32_t cols, void* stream);
+/* Y[M,N] = epilogue((Xq[M,K] . Wq[N,K]^T) * scale_x[row] * scale_w[column] + bias[N]) on tcgen05 (kind::f8f6f4,
+ * fp32 accumulate): Xq, Wq E4M3 bytes as written by mt_kernel_quantize_rows, scales fp32, bias bf16.  Epilogues
+ * as mt_kernel_linear (0: bf16; 1: GELU, bf16; 2: + fp32 residual, fp32).  K % 128 == 0; N % 256 == 0 (N % 128 == 0
+ * for epilogue 2); pointers 16-byte aligned. */
+int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d_wq, const float* d_scale_w,
+                         const void* d_bias, const void* d_residual, void* d_y, int32_t M, int32_t N, int32_t K,
+                         int32_t epilogue, uint32_t* d_status, void* stream);
+
 /* Y = LN(X[M,K] . W[N,K]^T + bias[N] + residual[M,N]) * gamma[N] + beta[N] in one launch: the residual
  * sub-layer followed by LayerNorm, as the encoder layer has it twice (after attention, after the FFN).
  * X, W, bias, gamma, beta bf16; residual fp32; Y is written twice, d_y bf16 [M,N] and d_y_f32 fp32 [M,N].

@@ -60,6 +60,8 @@ SIGNATURES = {
     "mt_last_error_string": (C.c_char_p, [_P]),
     "mt_kernel_linear_force_block_n": (None, [C.c_int32]),
     "mt_kernel_linear": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_kernel_quantize_rows": (C.c_int, [_P, _P, _P, _I32, _I32, _P]),
+    "mt_kernel_linear_fp8": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_linear_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
@@ -122,6 +124,19 @@ def mt_kernel_linear(x, w, bias, residual, y, epilogue: int, status=None, stream
     N = w.shape[0]
     _check(lib().mt_kernel_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), M, N, K, epilogue,
                                   1 if cta_pair else 0, _ptr(status), _stream(stream)), "mt_kernel_linear")
+
+
+def mt_kernel_quantize_rows(x, q, scale, stream=None) -> None:
+    rows, cols = x.shape
+    _check(lib().mt_kernel_quantize_rows(_ptr(x), _ptr(q), _ptr(scale), rows, cols, _stream(stream)),
+           "mt_kernel_quantize_rows")
+
+
+def mt_kernel_linear_fp8(xq, scale_x, wq, scale_w, bias, residual, y, epilogue: int, status=None, stream=None) -> None:
+    M, K = xq.shape
+    N = wq.shape[0]
+    _check(lib().mt_kernel_linear_fp8(_ptr(xq), _ptr(scale_x), _ptr(wq), _ptr(scale_w), _ptr(bias), _ptr(residual),
+                                      _ptr(y), M, N, K, epilogue, _ptr(status), _stream(stream)), "mt_kernel_linear_fp8")
 
 
 def mt_kernel_linear_layernorm(x, w, bias, residual, gamma, beta, y, y_f32, eps: float, status=None, stream=None) -> None:

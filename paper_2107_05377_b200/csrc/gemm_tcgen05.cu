@@ -67,8 +67,13 @@ __host__ __device__ constexpr int gemm_smem_bytes(int bn, bool pair, int epi) {
 // and stages half of the W tile; the MMA, issued by rank 0, reads both halves.  Per 128 x BN x 64
 // of tensor work a CTA then pulls 16 KB + BN/2 x 128 B from L2 instead of 16 KB + BN x 128 B, which
 // is what bounds the single-CTA kernel (an SM takes in roughly 64 bytes per clock).
-template <int BN, int EPI, bool PAIR>
+// FP8: the operands are E4M3 bytes with one fp32 scale per row of X and per row of W (GemmParams::scale_x,
+// scale_w); a shared-memory row of 128 bytes then holds 128 elements of K, an instruction covers 32 of them,
+// and the epilogue multiplies the accumulator by scale_x[row] * scale_w[column] before the bias.
+template <int BN, int EPI, bool PAIR, bool FP8 = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __grid_constant__ GemmParams p) {
+  static_assert(!FP8 || !PAIR, "the 8-bit operands run as single CTAs");
+  constexpr int KB_ELEMS = FP8 ? 2 * kGemmBlockK : kGemmBlockK;   // elements of K in a 128-byte row
   constexpr int STAGES = gemm_stages(BN, PAIR, EPI);
   constexpr int A_BYTES = gemm_a_bytes();
   constexpr int B_BYTES = gemm_b_bytes(BN, PAIR);   // this CTA's part of the W tile
@@ -101,7 +106,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
   const int n_tiles_n = p.N / BN;
-  const int k_blocks = p.K / kGemmBlockK;
+  const int k_blocks = p.K / KB_ELEMS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -147,10 +152,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       if (PAIR) {
         // rank 0 announces the bytes of both CTAs' W parts on its barrier; either CTA's copy may land first
         if (rank == 0) mbar_add_tx(bar_full + 8 * s, 2 * B_BYTES);
-        tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full_count + 8 * s);
+        tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full_count + 8 * s);
       } else {
         mbar_add_tx(bar_full + 8 * s, B_BYTES);
-        tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * kGemmBlockK, n0, bar_full + 8 * s);
+        tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full + 8 * s);
       }
     }
   }
@@ -193,14 +198,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           if (PAIR) {
             if (rank == 0)
               mbar_expect_tx(bar_full + 8 * stage, 2 * A_BYTES + (w_on_its_way ? 0 : 2 * B_BYTES));
-            tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full_count + 8 * stage);
+            tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], kb * KB_ELEMS, m0, bar_full_count + 8 * stage);
             if (!w_on_its_way)
-              tma_load_2d_pair(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full_count + 8 * stage);
+              tma_load_2d_pair(sB + stage * B_BYTES, &p.tmap_w[g], kb * KB_ELEMS, n0, bar_full_count + 8 * stage);
           } else {
             mbar_expect_tx(bar_full + 8 * stage, A_BYTES + (w_on_its_way ? 0 : B_BYTES));
-            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * KB_ELEMS, m0, bar_full + 8 * stage);
             if (!w_on_its_way)
-              tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+              tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * KB_ELEMS, n0, bar_full + 8 * stage);
           }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -226,7 +231,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(TILE_M, BN);
+      constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(TILE_M, BN) : umma_idesc_bf16(TILE_M, BN);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -244,8 +249,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           const uint64_t db = smem_desc_sw128(sB + stage * B_BYTES);
 #pragma unroll
           for (int k = 0; k < kGemmBlockK / 16; ++k) {
-            // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the address field
-            if (PAIR) umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            // advancing one instruction along K (16 bf16 or 32 E4M3 = 32 bytes) inside the swizzled row: +2 in the address field
+            if (FP8) umma_e4m3(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else if (PAIR) umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
             else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
@@ -301,6 +307,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       tc_fence_after();
       const bf16* bias = p.group[g].bias;
       const bool rows_in_range = m0 + quarter * 32 < m_rows;
+      float row_scale = 1.0f;          // (8-bit operands) scale of this thread's row of X
+      const float* col_scale = nullptr;
+      if (FP8) {
+        const int row = m0 + quarter * 32 + lane;
+        row_scale = row < p.M ? __ldg(p.group[g].scale_x + row) : 0.0f;
+        col_scale = p.group[g].scale_w;
+      }
 #pragma unroll 1
       for (int chunk = col_group; chunk < CHUNKS; chunk += COL_GROUPS) {
         const int col = n0 + chunk * CHUNK_COLS;
@@ -324,6 +337,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
             break;
           }
           res_phase[buf] ^= 1u;
+          if (FP8) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 sc = __ldg(reinterpret_cast<const float4*>(col_scale + col) + q);
+              v[q * 4 + 0] = __float_as_uint(__uint_as_float(v[q * 4 + 0]) * (row_scale * sc.x));
+              v[q * 4 + 1] = __float_as_uint(__uint_as_float(v[q * 4 + 1]) * (row_scale * sc.y));
+              v[q * 4 + 2] = __float_as_uint(__uint_as_float(v[q * 4 + 2]) * (row_scale * sc.z));
+              v[q * 4 + 3] = __float_as_uint(__uint_as_float(v[q * 4 + 3]) * (row_scale * sc.w));
+            }
+          }
           const uint4* bias4 = reinterpret_cast<const uint4*>(bias + col);
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -380,6 +403,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
             uint32_t v[32];
             tmem_ld_32x32(taddr + half * 32, v);
             tmem_ld_wait();
+            if (FP8) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 sc = __ldg(reinterpret_cast<const float4*>(col_scale + col + half * 32) + q);
+                v[q * 4 + 0] = __float_as_uint(__uint_as_float(v[q * 4 + 0]) * (row_scale * sc.x));
+                v[q * 4 + 1] = __float_as_uint(__uint_as_float(v[q * 4 + 1]) * (row_scale * sc.y));
+                v[q * 4 + 2] = __float_as_uint(__uint_as_float(v[q * 4 + 2]) * (row_scale * sc.z));
+                v[q * 4 + 3] = __float_as_uint(__uint_as_float(v[q * 4 + 3]) * (row_scale * sc.w));
+              }
+            }
             const uint4* bias4 = reinterpret_cast<const uint4*>(bias + col + half * 32);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -436,9 +469,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   }
 }
 
-template <int BN, int EPI, bool PAIR>
+template <int BN, int EPI, bool PAIR, bool FP8 = false>
 cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
-  auto kernel = gemm_bf16_tcgen05<BN, EPI, PAIR>;
+  auto kernel = gemm_bf16_tcgen05<BN, EPI, PAIR, FP8>;
   static bool configured = false;  // per instantiation; the attribute is per function and per device
   static int configured_device = -1;
   int dev = 0;
@@ -522,6 +555,13 @@ cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStr
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.block_n < 1 || p.N % p.block_n != 0 ||
       p.M < 1)
     return cudaErrorInvalidValue;
+  if (p.fp8) {
+    if (p.pair || p.K % (2 * kGemmBlockK) != 0) return cudaErrorInvalidValue;
+    if (epilogue == kEpiBias && p.block_n == 256) return launch_one<256, kEpiBias, false, true>(p, sm_count, stream);
+    if (epilogue == kEpiBiasGelu && p.block_n == 256) return launch_one<256, kEpiBiasGelu, false, true>(p, sm_count, stream);
+    if (epilogue == kEpiBiasResidual && p.block_n == 128) return launch_one<128, kEpiBiasResidual, false, true>(p, sm_count, stream);
+    return cudaErrorInvalidValue;
+  }
   return p.pair ? launch_any<true>(p, epilogue, sm_count, stream) : launch_any<false>(p, epilogue, sm_count, stream);
 }
 

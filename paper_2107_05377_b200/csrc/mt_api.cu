@@ -157,6 +157,21 @@ cudaError_t make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t 
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// Tensor map of a row-major matrix [rows, cols] of bytes (E4M3 operands) accessed in boxes of box_rows x 128.
+cudaError_t make_tmap_u8(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn enc = nullptr;
+  cudaError_t err = get_encoder(&enc);
+  if (err != cudaSuccess) return err;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols)};
+  const cuuint32_t box[2] = {128u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t elem[2] = {1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 // Fills group i of a grouped GEMM Y = epi(X[M,K] . W[N,K]^T + bias (+ residual)): operand maps, the
 // output map (bf16, or fp32 for the residual epilogue) and the fp32 residual map.
 cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, const void* w, const bf16* bias,
@@ -165,8 +180,13 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
   const bool res = epilogue == kEpiBiasResidual;
   const bool f32_out = res || epilogue == kEpiBiasTanhF32;
   cudaError_t e;
-  if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
-  if ((e = make_tmap(&g->tmap_w[i], w, N, K, g->block_n / (g->pair != 0 ? 2 : 1), kGemmBlockK, false)) != cudaSuccess) return e;
+  if (g->fp8 != 0) {
+    if ((e = make_tmap_u8(&g->tmap_x[i], x, M, K, kGemmBlockM)) != cudaSuccess) return e;
+    if ((e = make_tmap_u8(&g->tmap_w[i], w, N, K, g->block_n)) != cudaSuccess) return e;
+  } else {
+    if ((e = make_tmap(&g->tmap_x[i], x, M, K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return e;
+    if ((e = make_tmap(&g->tmap_w[i], w, N, K, g->block_n / (g->pair != 0 ? 2 : 1), kGemmBlockK, false)) != cudaSuccess) return e;
+  }
   if ((e = make_tmap(&g->tmap_out[i], y, M, N, 32, gemm_out_box_cols(epilogue), f32_out)) != cudaSuccess) return e;
   if (res && (e = make_tmap(&g->tmap_res[i], residual, M, N, 32, 32, true)) != cudaSuccess) return e;
   g->group[i].bias = bias;
@@ -1368,6 +1388,41 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   if (set_gemm_group(&p, 0, epilogue, d_x, d_w, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
                      d_y) != cudaSuccess)
     return MT_ERR_CUDA;
+  return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_quantize_rows(const void* d_x, void* d_q, float* d_scale, int32_t rows, int32_t cols, void* stream) {
+  if (d_x == nullptr || d_q == nullptr || d_scale == nullptr || rows < 1 || cols < 256 || cols % 256 != 0)
+    return MT_ERR_INVALID_ARG;
+  QuantParams p;
+  memset(&p, 0, sizeof(p));
+  p.x[0] = static_cast<const bf16*>(d_x); p.q[0] = static_cast<uint8_t*>(d_q); p.scale[0] = d_scale;
+  p.n_groups = 1; p.rows = rows; p.cols = cols;
+  return launch_quantize_rows(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d_wq, const float* d_scale_w,
+                         const void* d_bias, const void* d_residual, void* d_y, int32_t M, int32_t N, int32_t K,
+                         int32_t epilogue, uint32_t* d_status, void* stream) {
+  if (d_xq == nullptr || d_scale_x == nullptr || d_wq == nullptr || d_scale_w == nullptr || d_bias == nullptr ||
+      d_y == nullptr || M < 1 || K < 128 || K % 128 != 0 || epilogue < 0 || epilogue > 2 ||
+      (epilogue == 2 && d_residual == nullptr))
+    return MT_ERR_INVALID_ARG;
+  if (N < 128 || N % (epilogue == 2 ? 128 : 256) != 0) return MT_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MT_ERR_CUDA;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
+  p.fp8 = 1;
+  p.block_n = epilogue == 2 ? 128 : 256;
+  if (set_gemm_group(&p, 0, epilogue, d_xq, d_wq, static_cast<const bf16*>(d_bias), static_cast<const float*>(d_residual),
+                     d_y) != cudaSuccess)
+    return MT_ERR_CUDA;
+  p.group[0].scale_x = d_scale_x;
+  p.group[0].scale_w = d_scale_w;
   return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 

@@ -70,6 +70,8 @@ enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2, kEpiBi
 // The output and the residual are reached through the tensor maps of GemmParams.
 struct GemmGroup {
   const bf16* bias;
+  const float* scale_x;  // (8-bit operands) one scale per row of X, [M]
+  const float* scale_w;  // (8-bit operands) one scale per row of W, [N]
 };
 
 struct alignas(64) GemmParams {
@@ -83,6 +85,8 @@ struct alignas(64) GemmParams {
   const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
   int32_t pair;            // 1: run as pairs of CTAs on 256-row tiles (the W maps then fetch half a tile's rows)
   int32_t block_n;         // tile width along N: 128, 192 or 256 (gemm_block_n); N % block_n == 0
+  int32_t fp8;             // 1: X and W are E4M3 bytes (maps of uint8, boxes of 128 bytes of K) with row scales;
+                           // single CTAs, block_n 256 (128 for the residual epilogue), K % 128 == 0
   uint32_t* status;        // sticky device status word (may be null)
 };
 
@@ -212,6 +216,17 @@ struct TokenHeadParams {
   int32_t n_tasks, batch, seq, hidden, logits_stride;
 };
 cudaError_t launch_token_heads(const TokenHeadParams& p, cudaStream_t stream);
+
+// Row-wise quantisation to E4M3 for the 8-bit GEMMs: scale[r] = max|x[r, :]| * (1 / 448) (1 for a row of zeros),
+// q[r, c] = the E4M3 value nearest to x[r, c] / scale[r] (ties to even, saturating), all in fp32.
+struct QuantParams {
+  const bf16* x[kMaxGroups];   // [rows, cols]
+  uint8_t* q[kMaxGroups];      // [rows, cols]
+  float* scale[kMaxGroups];    // [rows]
+  int32_t n_groups, rows, cols;   // cols a multiple of 256
+  const int32_t* rows_valid;   // device scalar: rows actually in use (<= rows); null = all
+};
+cudaError_t launch_quantize_rows(const QuantParams& p, cudaStream_t stream);
 
 // row_start[b] for b = 0..batch and *rows_valid = row_start[batch]: b * seq (padded) or the running sum
 // of the lengths clamped to [1, seq] (packed).

@@ -183,6 +183,48 @@ __global__ void __launch_bounds__(kHeadThreads) head_kernel(const HeadParams p) 
   }
 }
 
+// Row-wise E4M3 quantisation (QuantParams): one warp per row; the row is read twice (bf16 from L2), first for
+// its largest magnitude, then to scale and convert.  Every decision is taken in fp32 with IEEE operations
+// that no compiler option can change: scale = amax * (1/448), y = x / scale, code = cvt.rn.satfinite.e4m3.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const QuantParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.y;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  int rows = p.rows;
+  if (p.rows_valid != nullptr) rows = min(rows, *p.rows_valid);
+  const int row = blockIdx.x * (kRowThreads / 32) + warp;
+  if (row >= rows) return;
+  const bf16* x = p.x[g] + static_cast<size_t>(row) * p.cols;
+  float amax = 0.f;
+  for (int c = lane * 8; c < p.cols; c += 256) {
+    float f[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(x + c)), f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  const float scale = amax == 0.f ? 1.0f : __fmul_rn(amax, 1.0f / 448.0f);
+  if (lane == 0) p.scale[g][row] = scale;
+  uint8_t* q = p.q[g] + static_cast<size_t>(row) * p.cols;
+  for (int c = lane * 8; c < p.cols; c += 256) {
+    float f[8];
+    unpack8(__ldg(reinterpret_cast<const uint4*>(x + c)), f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = __fdiv_rn(f[i], scale);
+    uint2 out;
+    out.x = cvt_e4m3x2(f[1], f[0]) | (cvt_e4m3x2(f[3], f[2]) << 16);
+    out.y = cvt_e4m3x2(f[5], f[4]) | (cvt_e4m3x2(f[7], f[6]) << 16);
+    *reinterpret_cast<uint2*>(q + c) = out;
+  }
+}
+
 // One warp: inclusive scan of the clamped lengths in chunks of 32.
 __global__ void row_starts_kernel(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed,
                                   int32_t* row_start, int32_t* rows_valid) {
@@ -233,6 +275,13 @@ __global__ void __launch_bounds__(kRowThreads) unpack_rows_kernel(const bf16* pa
 }
 
 }  // namespace
+
+cudaError_t launch_quantize_rows(const QuantParams& p, cudaStream_t stream) {
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1 || p.cols < 256 || p.cols % 256 != 0) return cudaErrorInvalidValue;
+  const int rows_per_cta = kRowThreads / 32;
+  dim3 grid((p.rows + rows_per_cta - 1) / rows_per_cta, p.n_groups);
+  return launch_kernel(quantize_rows_kernel, grid, dim3(kRowThreads), 0, stream, p);
+}
 
 cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,
                               int32_t* rows_valid, cudaStream_t stream) {
