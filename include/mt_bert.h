@@ -236,6 +236,15 @@ int mt_plan_cache_size(const mt_model* m);
  * used for every longer seq).  key "expected_tokens" (>= 0, default 0 = every row, any time): the caller's
  * estimate of the valid tokens per batch; with the packed layout the GEMM tile widths are chosen for
  * that many rows instead of batch*seq; it never changes a result.
+ * key "fp8_gemm" (0/1, default 0; before mt_bind_memory, it enlarges both arenas): reduced precision in the
+ * sense of Appendix E.  The Q/K/V, FFN-up and FFN-down projections run on E4M3 operands (tcgen05 kind::f8f6f4,
+ * fp32 accumulation) with one fp32 scale per operand row: weights are quantised once per output channel when
+ * they are loaded (8-bit copies behind the bf16 payload in the weights arena), activations per token by a
+ * row-wise kernel before each of those projections; see mt_kernel_quantize_rows.  Everything else (attention,
+ * the attention-output projection, LayerNorm, the fp32 residual stream, pooler, heads) is unchanged.  Against
+ * the unquantised fp64 definition the hidden states then agree to about 4e-2 relative L2 and the logits to
+ * about 3e-2 (measured on the 8-task tree; the tests state the bounds); merged == stand-alone still holds bit
+ * for bit.
  * key "sm_limit" (>= 0, default 0 = all; any time): size the persistent GEMM grids for at most this many SMs
  * (for callers that share the GPU between several streams and want to leave room; measured no gain).
  * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 2) layers
@@ -272,7 +281,8 @@ int mt_set_option(mt_model* m, const char* key, int64_t value);
 #define MT_CLASS_FFN_DOWN  6  /* GEMM: FFN down projection + residual               */
 #define MT_CLASS_LN2       7  /* LayerNorm after the FFN                            */
 #define MT_CLASS_HEAD      8  /* pooler + head                                      */
-#define MT_NUM_CLASSES     9
+#define MT_CLASS_QUANT     9  /* row-wise E4M3 quantisation (option "fp8_gemm")        */
+#define MT_NUM_CLASSES     10
 int mt_profile_read(mt_model* m, double* ms_by_class, int64_t* launches_by_class);
 
 /* Copies the hidden state [batch*seq, hidden] bf16 captured by the LAST mt_forward to d_out (padded

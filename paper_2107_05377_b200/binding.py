@@ -18,7 +18,7 @@ MT_OK = 0
 ERRORS = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "NOT_BOUND", -4: "NOT_LOADED", -5: "BLOB_MISMATCH",
           -6: "CUDA", -7: "UNSUPPORTED", -8: "DEVICE_FLAG"}
 FLAG_BAD_TOKEN, FLAG_BAD_SEGMENT, FLAG_BAD_LENGTH, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head")
+KERNEL_CLASSES = ("embed", "qkv", "attention", "attn_out", "ln1", "ffn_up", "ffn_down", "ln2", "head", "quant")
 
 
 class TrunkConfig(C.Structure):
@@ -196,7 +196,8 @@ class MTModel:
     """mt_create + mt_bind_memory + mt_load_weights + mt_forward around torch-owned memory."""
 
     def __init__(self, cfg, max_batch: int, max_seq: int, max_groups: Optional[int] = None,
-                 debug_capture: bool = False, device: str = "cuda:0", bind: bool = True, share_weights_with=None):
+                 debug_capture: bool = False, device: str = "cuda:0", bind: bool = True, share_weights_with=None,
+                 fp8_gemm: bool = False):
         """``share_weights_with``: another MTModel of the same configuration whose weights arena this one
         uses too (mt_adopt_weights) - a second batch in flight needs a workspace of its own, not a second
         copy of the weights."""
@@ -213,6 +214,8 @@ class MTModel:
             self.set_option("max_groups", max_groups)
         if debug_capture:
             self.set_option("debug_capture", 1)
+        if fp8_gemm:
+            self.set_option("fp8_gemm", 1)
         self.c_total = cfg.total_classes
         self.weights = self.workspace = None
         self._shared_from = share_weights_with

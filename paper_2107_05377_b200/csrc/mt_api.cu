@@ -40,6 +40,8 @@ inline size_t pad256(size_t n) { return (n + kAlign - 1) / kAlign * kAlign; }
 // Offsets (bytes from the start of the arena = start of the blob payload) of one layer's tensors.
 struct LayerOffsets {
   size_t wq, wk, wv, bq, bk, bv, wo, bo, ln1_g, ln1_b, w1, b1, w2, b2, ln2_g, ln2_b;
+  // 8-bit copies (option "fp8_gemm"), behind the payload of the blob: E4M3 bytes and one fp32 scale per output row
+  size_t q_qkv, s_qkv, q_w1, s_w1, q_w2, s_w2;
 };
 
 struct TaskEntry {
@@ -80,7 +82,11 @@ struct LayerTail {
   int32_t count = 0;
   // each residual GEMM together with the LayerNorm after it, as one cluster launch (option "fused_ln")
   bool ln_fused = false;
+  bool down_fused = false;   // the FFN-down projection too (not with 8-bit operands: that GEMM is the plain kernel)
   GemmLnParams attn_out_ln, ffn_down_ln;
+  // 8-bit operands: the inputs of the FFN-up and FFN-down projections are quantised row by row first
+  bool fp8 = false;
+  QuantParams q_h1, q_f;
 };
 struct DumpCopy {
   const bf16* src;
@@ -93,6 +99,7 @@ struct DumpCopy {
 // and values of all tokens) and the first-token attention (`attn_cls`, `n_cls` groups); the rest of
 // those layers, a few rows each, is run for all tasks together after the last wave (a `cls tail` step).
 struct Chunk {
+  QuantParams q_in;   // 8-bit operands: the layers' inputs, quantised row by row before the Q/K/V projection
   GemmParams qkv;
   AttnParams attn;
   ClsAttnParams attn_cls;
@@ -203,7 +210,8 @@ struct mt_model {
   // arena
   size_t emb_word, emb_pos, emb_type, emb_ln_g, emb_ln_b;
   std::vector<LayerOffsets> trunk_layers;
-  size_t weights_bytes;
+  size_t payload_bytes;   // the blob's payload = the bf16 part of the arena
+  size_t weights_bytes;   // payload + (option "fp8_gemm") the 8-bit copies
   bool trunk_loaded;
 
   // options
@@ -225,6 +233,7 @@ struct mt_model {
   bool overlap_cls;
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
+  bool fp8;          // Q/K/V, FFN-up and FFN-down projections on E4M3 operands (set before mt_bind_memory)
   bool pool_gemm;    // the pooler of tasks with a compact final state runs as a grouped GEMM on the tensor cores
 
   // device memory (caller-owned)
@@ -237,6 +246,7 @@ struct mt_model {
   // workspace layout (byte offsets)
   size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
       ws_slot0, ws_cls0, ws_dump0;
+  size_t slot_q_off, cls_q_off;   // 8-bit scratch inside a slot / inside a task's first-token scratch
   size_t cls_bytes, cls_h_bytes, cls_h32_bytes;  // per-task first-token scratch and its [B,H] bf16 / fp32 pieces
   size_t act_bytes;    // max_batch*max_seq*hidden bf16
   size_t act32_bytes;  // the same tensor in fp32
@@ -282,6 +292,52 @@ size_t place_layer(const mt_trunk_config& c, size_t off, LayerOffsets* lo) {
   return off;
 }
 
+// The 8-bit copies live behind the blob's payload, so the bf16 part of the arena stays a verbatim copy of it.
+void layout_fp8_weights(mt_model* m) {
+  size_t off = m->payload_bytes;
+  if (m->fp8) {
+    const size_t H = m->trunk.hidden, F = m->trunk.ffn;
+    auto take = [&](size_t bytes) { size_t at = off; off += pad256(bytes); return at; };
+    auto place = [&](LayerOffsets* lo) {
+      lo->q_qkv = take(3 * H * H); lo->s_qkv = take(3 * H * 4);
+      lo->q_w1 = take(F * H); lo->s_w1 = take(F * 4);
+      lo->q_w2 = take(H * F); lo->s_w2 = take(H * 4);
+    };
+    for (LayerOffsets& lo : m->trunk_layers) place(&lo);
+    for (TaskEntry& t : m->tasks)
+      for (LayerOffsets& lo : t.layers) place(&lo);
+  }
+  m->weights_bytes = off;
+}
+
+// Quantises the Q/K/V, FFN-up and FFN-down matrices of `layers` (already in the arena as bf16) into their 8-bit
+// copies: one scale per output channel = per row of W[N, K].  Grouped launches of up to kMaxGroups layers.
+cudaError_t quantize_layer_weights(const mt_model* m, const std::vector<const LayerOffsets*>& layers, cudaStream_t stream) {
+  const int32_t H = m->trunk.hidden, F = m->trunk.ffn;
+  for (size_t first = 0; first < layers.size(); first += kMaxGroups) {
+    const size_t count = std::min<size_t>(kMaxGroups, layers.size() - first);
+    for (int which = 0; which < 3; ++which) {
+      QuantParams q;
+      memset(&q, 0, sizeof(q));
+      q.n_groups = static_cast<int32_t>(count);
+      q.rows = which == 0 ? 3 * H : (which == 1 ? F : H);
+      q.cols = which == 2 ? F : H;
+      for (size_t i = 0; i < count; ++i) {
+        const LayerOffsets* lo = layers[first + i];
+        const size_t src = which == 0 ? lo->wq : (which == 1 ? lo->w1 : lo->w2);
+        const size_t dst = which == 0 ? lo->q_qkv : (which == 1 ? lo->q_w1 : lo->q_w2);
+        const size_t sc = which == 0 ? lo->s_qkv : (which == 1 ? lo->s_w1 : lo->s_w2);
+        q.x[i] = reinterpret_cast<const bf16*>(m->d_weights + src);
+        q.q[i] = m->d_weights + dst;
+        q.scale[i] = reinterpret_cast<float*>(m->d_weights + sc);
+      }
+      cudaError_t e = launch_quantize_rows(q, stream);
+      if (e != cudaSuccess) return e;
+    }
+  }
+  return cudaSuccess;
+}
+
 void layout_workspace(mt_model* m) {
   const size_t M = static_cast<size_t>(m->max_batch) * m->max_seq;
   const size_t H = m->trunk.hidden, F = m->trunk.ffn;
@@ -306,6 +362,9 @@ void layout_workspace(mt_model* m) {
   m->n_slots = std::min<int32_t>(m->max_groups, static_cast<int32_t>(m->tasks.size()) + 1);
   // slot = qkv [M,3H] bf16 + ctx [M,H] bf16 + u [M,H] fp32 + h1 [M,H] bf16 and fp32 + f [M,F] bf16
   m->slot_bytes = pad256(M * 3 * H * 2) + m->act_bytes + m->act32_bytes + m->state_bytes + pad256(M * F * 2);
+  m->slot_q_off = m->slot_bytes;
+  // 8-bit operands: E4M3 copies of the layer input and of h1 ([M,H]) and of f ([M,F]), each with a scale per row
+  if (m->fp8) m->slot_bytes += 2 * pad256(M * H) + pad256(M * F) + 3 * pad256(M * 4);
   m->ws_slot0 = off;
   off += m->slot_bytes * m->n_slots;
   // per task, for its last branch layer on first tokens: ctx bf16, residual fp32, u fp32, h1 bf16 + fp32 (all
@@ -313,6 +372,11 @@ void layout_workspace(mt_model* m) {
   m->cls_h_bytes = pad256(static_cast<size_t>(m->max_batch) * H * 2);
   m->cls_h32_bytes = pad256(static_cast<size_t>(m->max_batch) * H * 4);
   m->cls_bytes = 2 * m->cls_h_bytes + 3 * m->cls_h32_bytes + pad256(static_cast<size_t>(m->max_batch) * F * 2);
+  m->cls_q_off = m->cls_bytes;
+  if (m->fp8) {
+    const size_t B = static_cast<size_t>(m->max_batch);
+    m->cls_bytes += pad256(B * H) + pad256(B * F) + 2 * pad256(B * 4);
+  }
   m->ws_cls0 = off;
   off += m->cls_bytes * m->tasks.size();
   m->n_dump = 0;
@@ -383,6 +447,37 @@ float* f32_of(const mt_model* m, bf16* state) {
   return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(state) + m->act_bytes);
 }
 
+// 8-bit scratch of a slot (rows = max_batch * max_seq; xq/sx: the layer input) or of a task's first-token
+// scratch (rows = max_batch; no xq).
+struct QuantScratch {
+  uint8_t* xq; float* sx;
+  uint8_t* h1q; float* sh1;
+  uint8_t* fq; float* sf;
+};
+QuantScratch slot_quant(const mt_model* m, uint8_t* slot) {
+  const size_t M = static_cast<size_t>(m->max_batch) * m->max_seq, H = m->trunk.hidden, F = m->trunk.ffn;
+  uint8_t* p = slot + m->slot_q_off;
+  QuantScratch q;
+  q.xq = p; p += pad256(M * H);
+  q.sx = reinterpret_cast<float*>(p); p += pad256(M * 4);
+  q.h1q = p; p += pad256(M * H);
+  q.sh1 = reinterpret_cast<float*>(p); p += pad256(M * 4);
+  q.fq = p; p += pad256(M * F);
+  q.sf = reinterpret_cast<float*>(p);
+  return q;
+}
+QuantScratch cls_quant(const mt_model* m, uint8_t* cs) {
+  const size_t B = static_cast<size_t>(m->max_batch), H = m->trunk.hidden, F = m->trunk.ffn;
+  uint8_t* p = cs + m->cls_q_off;
+  QuantScratch q;
+  q.xq = nullptr; q.sx = nullptr;
+  q.h1q = p; p += pad256(B * H);
+  q.sh1 = reinterpret_cast<float*>(p); p += pad256(B * 4);
+  q.fq = p; p += pad256(B * F);
+  q.sf = reinterpret_cast<float*>(p);
+  return q;
+}
+
 // True when the final state of a task is [B, H], one row per sequence.
 bool is_token_task(const mt_model* m, int32_t task) { return m->tasks[task].cfg.head_kind == MT_HEAD_TOKEN; }
 bool is_compact_task(const mt_model* m, int32_t task) {
@@ -418,7 +513,9 @@ bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) {
 }
 // Launches of steps 3-7 for `groups` layers.
 int32_t tail_launches(const mt_model* m, int32_t groups, int64_t rows) {
-  return use_fused_ln(m, groups, rows) ? 3 : 5;
+  const bool fused = use_fused_ln(m, groups, rows);
+  // 8-bit operands: two quantisations, and the FFN-down projection keeps its LayerNorm as a launch of its own
+  return (fused ? 3 : 5) + (m->fp8 ? 2 + (fused ? 1 : 0) : 0);
 }
 
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
@@ -436,6 +533,20 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   init_gemm(&t->attn_out, H, H, kEpiBiasResidual);
   init_gemm(&t->ffn_up, F, H, kEpiBiasGelu);
   init_gemm(&t->ffn_down, H, F, kEpiBiasResidual);
+  t->fp8 = m->fp8;
+  if (m->fp8) {
+    // E4M3 operands: single CTAs, 256-wide tiles (128 with the residual epilogue)
+    t->ffn_up.fp8 = t->ffn_down.fp8 = 1;
+    t->ffn_up.pair = t->ffn_down.pair = 0;
+    t->ffn_up.block_n = 256;
+    t->ffn_down.block_n = 128;
+    memset(&t->q_h1, 0, sizeof(t->q_h1));
+    memset(&t->q_f, 0, sizeof(t->q_f));
+    t->q_h1.rows = t->q_f.rows = rows;
+    t->q_h1.cols = H;
+    t->q_f.cols = F;
+    t->q_h1.rows_valid = t->q_f.rows_valid = rows_valid;
+  }
   memset(&t->ln1, 0, sizeof(t->ln1));
   memset(&t->ln2, 0, sizeof(t->ln2));
   t->ln1.rows_valid = t->ln2.rows_valid = rows_valid;
@@ -444,6 +555,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
   t->ln_fused = use_fused_ln(m, groups, rows);
+  t->down_fused = t->ln_fused && !m->fp8;
   if (t->ln_fused) {
     auto init_ln = [&](GemmLnParams* g, int32_t K) {
       memset(g, 0, sizeof(*g));
@@ -460,7 +572,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
 // Steps 3-7 of a layer for one group of a tail: u = ctx Wo^T + bo + residual; h1 = LN(u);
 // f = GELU(h1 W1^T + b1); u = f W2^T + b2 + h1; out = LN(u).
 cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo, const bf16* ctx, const float* residual,
-                        float* u, bf16* h1, float* h1_32, bf16* f, bf16* out, float* out32) {
+                        float* u, bf16* h1, float* h1_32, bf16* f, bf16* out, float* out32, const QuantScratch* qs) {
   const int i = t->count;
   cudaError_t e;
   if ((e = set_gemm_group(&t->attn_out, i, kEpiBiasResidual, ctx, w_ptr(m, lo->wo), w_ptr(m, lo->bo), residual, u)) !=
@@ -468,12 +580,29 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
     return e;
   t->ln1.x[i] = u; t->ln1.gamma[i] = w_ptr(m, lo->ln1_g); t->ln1.beta[i] = w_ptr(m, lo->ln1_b);
   t->ln1.y[i] = h1; t->ln1.y32[i] = h1_32;
-  if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
-      cudaSuccess)
-    return e;
-  if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) !=
-      cudaSuccess)
-    return e;
+  if (t->fp8) {
+    // h1 and f are quantised row by row into the scratch; the projections read those and the 8-bit weights
+    t->q_h1.x[i] = h1; t->q_h1.q[i] = qs->h1q; t->q_h1.scale[i] = qs->sh1;
+    t->q_f.x[i] = f; t->q_f.q[i] = qs->fq; t->q_f.scale[i] = qs->sf;
+    t->q_h1.n_groups = t->q_f.n_groups = i + 1;
+    if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, qs->h1q, m->d_weights + lo->q_w1, w_ptr(m, lo->b1), nullptr, f)) !=
+        cudaSuccess)
+      return e;
+    t->ffn_up.group[i].scale_x = qs->sh1;
+    t->ffn_up.group[i].scale_w = reinterpret_cast<const float*>(m->d_weights + lo->s_w1);
+    if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, qs->fq, m->d_weights + lo->q_w2, w_ptr(m, lo->b2), h1_32,
+                            u)) != cudaSuccess)
+      return e;
+    t->ffn_down.group[i].scale_x = qs->sf;
+    t->ffn_down.group[i].scale_w = reinterpret_cast<const float*>(m->d_weights + lo->s_w2);
+  } else {
+    if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
+        cudaSuccess)
+      return e;
+    if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) !=
+        cudaSuccess)
+      return e;
+  }
   t->ln2.x[i] = u; t->ln2.gamma[i] = w_ptr(m, lo->ln2_g); t->ln2.beta[i] = w_ptr(m, lo->ln2_b);
   t->ln2.y[i] = out; t->ln2.y32[i] = out32;
   t->count = i + 1;
@@ -494,7 +623,9 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
     // (a state is its bf16 copy followed by room for its fp32 copy: the fp32 result always has a home)
     float* out32_home = out32 != nullptr ? out32 : f32_of(m, out);
     if ((e = set_ln(&t->attn_out_ln, ctx, lo->wo, lo->bo, lo->ln1_g, lo->ln1_b, residual, h1, h1_32)) != cudaSuccess) return e;
-    if ((e = set_ln(&t->ffn_down_ln, f, lo->w2, lo->b2, lo->ln2_g, lo->ln2_b, h1_32, out, out32_home)) != cudaSuccess) return e;
+    if (t->down_fused &&
+        (e = set_ln(&t->ffn_down_ln, f, lo->w2, lo->b2, lo->ln2_g, lo->ln2_b, h1_32, out, out32_home)) != cudaSuccess)
+      return e;
   }
   return cudaSuccess;
 }
@@ -510,6 +641,16 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
   ck->qkv.M = M; ck->qkv.N = 3 * H; ck->qkv.K = H;
   ck->qkv.pair = use_pair(m, M, static_cast<int64_t>(count));
   choose_block_n(m, &ck->qkv, kEpiBias, false, static_cast<int32_t>(count));
+  memset(&ck->q_in, 0, sizeof(ck->q_in));
+  if (m->fp8) {
+    ck->qkv.fp8 = 1;
+    ck->qkv.pair = 0;
+    ck->qkv.block_n = 256;
+    ck->q_in.n_groups = static_cast<int32_t>(count);
+    ck->q_in.rows = M;
+    ck->q_in.cols = H;
+    ck->q_in.rows_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
+  }
   ck->qkv.m_valid = reinterpret_cast<const int32_t*>(m->d_workspace + m->ws_rows_valid);
   ck->qkv.status = reinterpret_cast<uint32_t*>(m->d_workspace + m->ws_status);
   int32_t n_full = 0;
@@ -550,9 +691,18 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
     cudaError_t e;
     // 1. qkv = in . [Wq;Wk;Wv]^T + [bq;bk;bv] on every token (the three matrices and biases are
     //    contiguous in the arena); keys and values are needed for all tokens even in a `cls` layer
-    if ((e = set_gemm_group(&ck->qkv, static_cast<int>(i), kEpiBias, in, w_ptr(m, lo->wq), w_ptr(m, lo->bq), nullptr,
-                            qkv)) != cudaSuccess)
+    const QuantScratch qs = m->fp8 ? slot_quant(m, slot) : QuantScratch{};
+    if (m->fp8) {
+      ck->q_in.x[i] = in; ck->q_in.q[i] = qs.xq; ck->q_in.scale[i] = qs.sx;
+      if ((e = set_gemm_group(&ck->qkv, static_cast<int>(i), kEpiBias, qs.xq, m->d_weights + lo->q_qkv, w_ptr(m, lo->bq),
+                              nullptr, qkv)) != cudaSuccess)
+        return e;
+      ck->qkv.group[i].scale_x = qs.sx;
+      ck->qkv.group[i].scale_w = reinterpret_cast<const float*>(m->d_weights + lo->s_qkv);
+    } else if ((e = set_gemm_group(&ck->qkv, static_cast<int>(i), kEpiBias, in, w_ptr(m, lo->wq), w_ptr(m, lo->bq), nullptr,
+                                   qkv)) != cudaSuccess) {
       return e;
+    }
     const bool cls = is_cls_op(m, op);
     if (!cls) {
       // 2. ctx = attention(qkv) for every token; 3-7 on every token
@@ -564,7 +714,7 @@ cudaError_t build_chunk(const mt_model* m, const std::vector<OpDesc>& ops, size_
           ((e = make_tmap(&ck->attn.tmap_qkv[a], qkv, M, 3 * H, kAttnTileRows, kHeadDim, false)) != cudaSuccess ||
            (e = make_tmap(&ck->attn.tmap_qkv64[a], qkv, M, 3 * H, kAttnTileRows / 2, kHeadDim, false)) != cudaSuccess))
         return e;
-      if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f32_of(m, h1), f, out, f32_of(m, out))) !=
+      if ((e = add_to_tail(m, &ck->full, lo, ctx, f32_of(m, in), u, h1, f32_of(m, h1), f, out, f32_of(m, out), &qs)) !=
           cudaSuccess)
         return e;
       if (m->debug_capture) ck->dumps.push_back({out, dump_slot(m, op.task, op.layer), false});
@@ -599,7 +749,8 @@ cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks,
     float* h1_32 = reinterpret_cast<float*>(cs + 2 * m->cls_h_bytes + 2 * m->cls_h32_bytes);
     bf16* f = reinterpret_cast<bf16*>(cs + 2 * m->cls_h_bytes + 3 * m->cls_h32_bytes);
     bf16* out = task_buf(m, t);  // the task's state becomes [B, H]
-    cudaError_t e = add_to_tail(m, &st->tail, lo, ctx, res, u, h1, h1_32, f, out, nullptr);
+    const QuantScratch qs = m->fp8 ? cls_quant(m, cs) : QuantScratch{};
+    cudaError_t e = add_to_tail(m, &st->tail, lo, ctx, res, u, h1, h1_32, f, out, nullptr, &qs);
     if (e != cudaSuccess) return e;
     if (m->debug_capture) st->dumps.push_back({out, dump_slot(m, t, te.cfg.branch_layers), true});
   }
@@ -609,7 +760,8 @@ cudaError_t build_cls_tail(const mt_model* m, const std::vector<int32_t>& tasks,
 int32_t chunk_launches(const mt_model* m, const std::vector<OpDesc>& ops, size_t first, size_t count, int64_t rows) {
   size_t n_cls = 0;
   for (size_t i = 0; i < count; ++i) n_cls += is_cls_op(m, ops[first + i]) ? 1 : 0;
-  return 1 + (n_cls < count ? 1 + tail_launches(m, static_cast<int32_t>(count - n_cls), rows) : 0) + (n_cls > 0 ? 1 : 0);
+  return 1 + (m->fp8 ? 1 : 0) + (n_cls < count ? 1 + tail_launches(m, static_cast<int32_t>(count - n_cls), rows) : 0) +
+         (n_cls > 0 ? 1 : 0);
 }
 // Active tasks whose last branch layer is finished on first tokens right after wave w (1-based):
 // those whose last layer is in wave w with option early_heads, otherwise all of them after the last wave.
@@ -828,7 +980,9 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
     }
     te.loaded = false;
   }
-  m->weights_bytes = off;
+  m->payload_bytes = off;
+  m->fp8 = false;
+  layout_fp8_weights(m);
   m->c_total = col;
   m->ct_total = col_tok;
   layout_workspace(m);
@@ -847,7 +1001,7 @@ void mt_destroy(mt_model* m) {
 
 size_t mt_weights_bytes(const mt_model* m) { return m ? m->weights_bytes : 0; }
 size_t mt_workspace_bytes(const mt_model* m) { return m ? m->ws_total : 0; }
-size_t mt_blob_bytes(const mt_model* m) { return m ? m->weights_bytes + kHeaderBytes : 0; }
+size_t mt_blob_bytes(const mt_model* m) { return m ? m->payload_bytes + kHeaderBytes : 0; }
 size_t mt_task_blob_bytes(const mt_model* m, int32_t task) {
   if (m == nullptr || task < 0 || task >= static_cast<int32_t>(m->tasks.size())) return 0;
   return m->tasks[task].section_bytes + kHeaderBytes;
@@ -945,6 +1099,9 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     m->max_groups = static_cast<int32_t>(value);
   } else if (strcmp(key, "debug_capture") == 0) {
     m->debug_capture = value != 0;
+  } else if (strcmp(key, "fp8_gemm") == 0) {
+    m->fp8 = value != 0;
+    layout_fp8_weights(m);
   } else {
     return fail(m, MT_ERR_INVALID_ARG, std::string("unknown option ") + key);
   }
@@ -1015,11 +1172,18 @@ static int check_header(const mt_model* m, const void* blob, size_t bytes, uint3
 int mt_load_weights(mt_model* m, const void* host_blob, size_t bytes, void* stream) {
   if (m == nullptr) return MT_ERR_INVALID_ARG;
   if (m->d_weights == nullptr) return fail(m, MT_ERR_NOT_BOUND, "mt_bind_memory has not been called");
-  int rc = check_header(m, host_blob, bytes, 0, -1, m->weights_bytes);
+  int rc = check_header(m, host_blob, bytes, 0, -1, m->payload_bytes);
   if (rc != MT_OK) return rc;
-  cudaError_t e = cudaMemcpyAsync(m->d_weights, static_cast<const uint8_t*>(host_blob) + kHeaderBytes, m->weights_bytes,
+  cudaError_t e = cudaMemcpyAsync(m->d_weights, static_cast<const uint8_t*>(host_blob) + kHeaderBytes, m->payload_bytes,
                                   cudaMemcpyHostToDevice, as_stream(stream));
   if (e != cudaSuccess) return fail_cuda(m, e, "copying weights");
+  if (m->fp8) {
+    std::vector<const LayerOffsets*> layers;
+    for (const LayerOffsets& lo : m->trunk_layers) layers.push_back(&lo);
+    for (const TaskEntry& t : m->tasks)
+      for (const LayerOffsets& lo : t.layers) layers.push_back(&lo);
+    if ((e = quantize_layer_weights(m, layers, as_stream(stream))) != cudaSuccess) return fail_cuda(m, e, "quantising weights");
+  }
   m->trunk_loaded = true;
   for (TaskEntry& t : m->tasks) t.loaded = true;
   return MT_OK;
@@ -1029,7 +1193,7 @@ int mt_adopt_weights(mt_model* m, const mt_model* src) {
   if (m == nullptr || src == nullptr) return MT_ERR_INVALID_ARG;
   if (m->d_weights == nullptr || src->d_weights == nullptr) return fail(m, MT_ERR_NOT_BOUND, "both models must be bound");
   if (m->d_weights != src->d_weights) return fail(m, MT_ERR_INVALID_ARG, "the two models are bound to different weight arenas");
-  bool same = m->weights_bytes == src->weights_bytes && m->tasks.size() == src->tasks.size() &&
+  bool same = m->weights_bytes == src->weights_bytes && m->fp8 == src->fp8 && m->tasks.size() == src->tasks.size() &&
               memcmp(&m->trunk, &src->trunk, sizeof(m->trunk)) == 0;
   for (size_t t = 0; same && t < m->tasks.size(); ++t)
     same = memcmp(&m->tasks[t].cfg, &src->tasks[t].cfg, sizeof(mt_task_config)) == 0;
@@ -1049,6 +1213,11 @@ int mt_load_task_weights(mt_model* m, int32_t task, const void* host_blob, size_
   cudaError_t e = cudaMemcpyAsync(m->d_weights + te.section_begin, static_cast<const uint8_t*>(host_blob) + kHeaderBytes,
                                   te.section_bytes, cudaMemcpyHostToDevice, as_stream(stream));
   if (e != cudaSuccess) return fail_cuda(m, e, "copying task weights");
+  if (m->fp8) {
+    std::vector<const LayerOffsets*> layers;
+    for (const LayerOffsets& lo : te.layers) layers.push_back(&lo);
+    if ((e = quantize_layer_weights(m, layers, as_stream(stream))) != cudaSuccess) return fail_cuda(m, e, "quantising task weights");
+  }
   te.loaded = true;
   return MT_OK;
 }
@@ -1182,14 +1351,18 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
 #define MT_TAIL(tail)                                                                                                  \
   do {                                                                                                                 \
     LayerTail* t_ = (tail);                                                                                            \
-    if (t_->ln_fused) {                                                                                         \
+    if (t_->ln_fused) {                                                                                                \
       MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm_ln(t_->attn_out_ln, stream), "attention output GEMM + LayerNorm");       \
-      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");            \
-      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm_ln(t_->ffn_down_ln, stream), "FFN down GEMM + LayerNorm");               \
     } else {                                                                                                           \
       MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t_->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM"); \
       MT_TIMED(MT_CLASS_LN1, launch_layernorm(t_->ln1, stream), "LayerNorm 1");                                        \
-      MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");            \
+    }                                                                                                                  \
+    if (t_->fp8) MT_TIMED(MT_CLASS_QUANT, launch_quantize_rows(t_->q_h1, stream), "quantising the FFN input");         \
+    MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");              \
+    if (t_->fp8) MT_TIMED(MT_CLASS_QUANT, launch_quantize_rows(t_->q_f, stream), "quantising the FFN intermediate");   \
+    if (t_->down_fused) {                                                                                              \
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm_ln(t_->ffn_down_ln, stream), "FFN down GEMM + LayerNorm");               \
+    } else {                                                                                                           \
       MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t_->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");  \
       MT_TIMED(MT_CLASS_LN2, launch_layernorm(t_->ln2, stream), "LayerNorm 2");                                        \
     }                                                                                                                  \
@@ -1224,6 +1397,7 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
       Chunk& ck = st.chunk;
       ck.attn.lengths = d_lengths;
       ck.attn_cls.lengths = d_lengths;
+      if (m->fp8) MT_TIMED(MT_CLASS_QUANT, launch_quantize_rows(ck.q_in, stream), "quantising the layer inputs");
       MT_TIMED(MT_CLASS_QKV, launch_gemm(ck.qkv, kEpiBias, m->sm_count, stream), "QKV GEMM");
       const bool beside = m->overlap_cls && m->side_stream != nullptr && !m->profile && ck.n_cls > 0 && ck.full.count > 0;
       if (beside) {

@@ -81,6 +81,23 @@ def bench_linear(m, n, k, epilogue, iters, warmup, flush):
             "tflops": flops / ms / 1e9, "min_gbytes_per_s": bytes_ / ms / 1e6}
 
 
+def bench_linear_fp8(m, n, k, epilogue, iters, warmup, flush):
+    """The 8-bit GEMM on operands quantised by the library's own row-wise kernel (timed: the GEMM alone)."""
+    x = torch.randn(m, k, device="cuda").to(torch.bfloat16)
+    w = (0.02 * torch.randn(n, k, device="cuda")).to(torch.bfloat16)
+    b = (0.02 * torch.randn(n, device="cuda")).to(torch.bfloat16)
+    r = torch.randn(m, n, device="cuda") if epilogue == 2 else None
+    y = torch.empty(m, n, device="cuda", dtype=torch.float32 if epilogue == 2 else torch.bfloat16)
+    xq, wq = torch.empty(m, k, device="cuda", dtype=torch.uint8), torch.empty(n, k, device="cuda", dtype=torch.uint8)
+    sx, sw = torch.empty(m, device="cuda"), torch.empty(n, device="cuda")
+    mt.mt_kernel_quantize_rows(x, xq, sx)
+    mt.mt_kernel_quantize_rows(w, wq, sw)
+    ms = _time(lambda: mt.mt_kernel_linear_fp8(xq, sx, wq, sw, b, r, y, epilogue), iters, warmup, flush)
+    ms_q = _time(lambda: mt.mt_kernel_quantize_rows(x, xq, sx), iters, warmup, flush)
+    return {"kernel": "linear_fp8", "M": m, "N": n, "K": k, "epilogue": epilogue, "us": 1e3 * ms,
+            "tflops": 2.0 * m * n * k / ms / 1e9, "quantize_rows_us": 1e3 * ms_q}
+
+
 def bench_linear_ln(m, n, k, iters, warmup, flush):
     x = torch.randn(m, k, device="cuda").to(torch.bfloat16)
     w = (0.02 * torch.randn(n, k, device="cuda")).to(torch.bfloat16)
@@ -123,7 +140,7 @@ def bench_layernorm(rows, hidden, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["linear", "linear_ln", "attention", "layernorm", "suite"])
+    ap.add_argument("kernel", choices=["linear", "linear_fp8", "linear_ln", "attention", "layernorm", "suite"])
     ap.add_argument("--m", type=int, default=4096)
     ap.add_argument("--n", type=int, default=2304)
     ap.add_argument("--k", type=int, default=768)
@@ -150,6 +167,8 @@ def main():
     torch.manual_seed(0)
     if a.kernel == "linear":
         print(json.dumps(bench_linear(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
+    elif a.kernel == "linear_fp8":
+        print(json.dumps(bench_linear_fp8(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
     elif a.kernel == "linear_ln":
         print(json.dumps(bench_linear_ln(a.m, a.n, a.k, a.iters, a.warmup, a.flush)))
     elif a.kernel == "attention":
@@ -162,7 +181,10 @@ def main():
                 print(json.dumps(bench_linear(m, n, k, e, a.iters, a.warmup, a.flush)))
             for (n, k) in ((768, 768), (768, 3072)):
                 print(json.dumps(bench_linear_ln(m, n, k, a.iters, a.warmup, a.flush)))
+            for (n, k, e) in ((2304, 768, 0), (3072, 768, 1), (768, 3072, 2)):
+                print(json.dumps(bench_linear_fp8(m, n, k, e, a.iters, a.warmup, a.flush)))
         print(json.dumps(bench_linear(8192, 8192, 8192, 0, 10, 2, a.flush)))
+        print(json.dumps(bench_linear_fp8(8192, 8192, 8192, 0, 10, 2, a.flush)))
         print(json.dumps(bench_attention(32, 128, 12, 16, a.iters, a.warmup, a.flush)))
         print(json.dumps(bench_attention(16, 512, 12, 128, a.iters, a.warmup, a.flush)))
         print(json.dumps(bench_layernorm(4096, 768, a.iters, a.warmup, a.flush)))

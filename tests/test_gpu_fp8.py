@@ -72,3 +72,83 @@ def test_fp8_linear_matches_the_oracle_on_oracle_quantised_operands(M, N, K, epi
     exact = orc.linear(x, w, b)
     if epi == 0:
         assert rel_l2(got, exact) <= 0.06
+
+
+def fp8_forward(cfg, blob, batch, mask=None, debug=False):
+    B, S = batch.token_ids.shape
+    model = mt.MTModel(cfg, B, S, debug_capture=debug, fp8_gemm=True)
+    model.load_weights(blob)
+    logits = torch.full((B, cfg.total_classes), float("nan"), device="cuda")
+    model.forward(*dev_batch(batch), logits, task_mask=mask)
+    torch.cuda.synchronize()
+    assert model.poll_status() == 0
+    return model, logits
+
+
+# Bounds of the 8-bit path (E4M3 keeps 3 mantissa bits: 2^-4 relative rounding per operand element).  Against the
+# 8-bit ORACLE the GPU differs by its bf16/fp32 rounding plus the codes that flip where the two sides' inputs differ
+# in the last bits; against the UNQUANTISED fp64 definition it carries the quantisation noise itself.
+# Measured on the trees below: 2.9e-2 / 2.4e-2 against the 8-bit oracle, 3.8e-2 / 2.8e-2 against the exact one.
+FP8_HIDDEN_VS_FP8_ORACLE = 5e-2
+FP8_LOGITS_VS_FP8_ORACLE = 5e-2
+FP8_HIDDEN_VS_EXACT = 8e-2
+FP8_LOGITS_VS_EXACT = 1e-1
+
+
+def test_fp8_forward_against_the_fp8_oracle_and_the_exact_one():
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    batch = synth.make_batch(cfg, 6, 150, 1, 150, seed=4)
+    B, S = batch.token_ids.shape
+    model, logits = fp8_forward(cfg, blob, batch, debug=True)
+    got = logits.cpu().numpy().astype(np.float64)
+    worst = {}
+    for name, layer_fn, tol_h, tol_l in (("fp8 oracle", f8.encoder_layer_fp8, FP8_HIDDEN_VS_FP8_ORACLE, FP8_LOGITS_VS_FP8_ORACLE),
+                                        ("exact oracle", None, FP8_HIDDEN_VS_EXACT, FP8_LOGITS_VS_EXACT)):
+        hid = []
+        want = orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, wf, task_triples(cfg), cfg.heads,
+                                    cfg.ln_eps, hidden_out=hid, layer_fn=layer_fn)
+        err_l = float(np.max(np.abs(got - want)))
+        err_h = 0.0
+        for key in hid[0]:
+            t, layer = (-1, key[1]) if key[0] == "trunk" else (key[1], key[2])
+            state = dev_bf16_to_f64(model.debug_hidden(t, layer, B, S)).reshape(B, S, cfg.hidden)
+            for b in range(B):
+                n = int(batch.lengths[b])
+                if key[0] == "task" and key[2] == cfg.tasks[key[1]].branch_layers:
+                    n = 1
+                err_h = max(err_h, rel_l2(state[b, :n], hid[b][key][:n]))
+        worst[name] = (err_h, err_l)
+        assert err_h <= tol_h and err_l <= tol_l, (name, err_h, err_l)
+    print("fp8 forward, worst (hidden rel-L2, logits max-abs):", worst)
+    # deterministic, and masking keeps the bits
+    _, again = fp8_forward(cfg, blob, batch)
+    assert torch.equal(again, logits)
+    offs = cfg.logit_offsets + [cfg.total_classes]
+    _, one = fp8_forward(cfg, blob, batch, mask=0b0010)
+    assert torch.equal(one[:, offs[1]:offs[2]], logits[:, offs[1]:offs[2]])
+
+
+def test_fp8_glue8_tree_32x128_sampled_rows_and_merged_equals_standalone():
+    cfg = synth.config_glue8()
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.batch_glue8(cfg)
+    model, logits = fp8_forward(cfg, blob, batch)
+    got = logits.cpu().numpy().astype(np.float64)
+    order = np.argsort(batch.lengths)
+    rows = [int(order[0]), int(order[-1])]
+    for name, layer_fn, tol in (("fp8 oracle", f8.encoder_layer_fp8, FP8_LOGITS_VS_FP8_ORACLE), ("exact oracle", None, FP8_LOGITS_VS_EXACT)):
+        want = orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, wf, task_triples(cfg), cfg.heads,
+                                    cfg.ln_eps, rows=rows, layer_fn=layer_fn)
+        err = max(float(np.max(np.abs(got[b] - want[b]))) for b in rows)
+        print(name, "logits max-abs", err)
+        assert err <= tol, (name, err)
+    assert torch.isfinite(logits).all()
+    # Section 3.3 under reduced precision: a task's stand-alone student gives the bits of its merged columns
+    offs = cfg.logit_offsets
+    for t in (3, 6):
+        st_cfg = synth.config_single_task(cfg, t)
+        st_blob = synth.pack_weights(st_cfg, synth.select_task_weights(w, t))
+        _, single = fp8_forward(st_cfg, st_blob, batch)
+        assert torch.equal(single, logits[:, offs[t]:offs[t] + cfg.tasks[t].num_classes]), t
