@@ -247,13 +247,16 @@ int mt_plan_cache_size(const mt_model* m);
  * for bit.
  * key "sm_limit" (>= 0, default 0 = all; any time): size the persistent GEMM grids for at most this many SMs
  * (for callers that share the GPU between several streams and want to leave room; measured no gain).
- * key "fused_ln" (0 never; 1 always; 2 = for launches of at most "fused_ln_max_groups" (default 2) layers
- * and for launches of at most "fused_ln_max_rows" (default 0) rows per layer, the default; any time): the attention-output and FFN-down projections carry the LayerNorm that follows
- * them: the CTAs holding the column blocks of the same 128 rows form a thread-block cluster and exchange
- * per-row statistics through distributed shared memory, so the pre-normalisation sum never goes to global
- * memory and no LayerNorm launch follows.  Results have the same bits as the separate launches
- * (every LayerNorm of the library sums its row statistics over the same 64-column segments in the same order).  Measured: a few microseconds faster for one or two layers, slower than the wider
- * paired tiles of the plain GEMM where more layers share a launch.
+ * key "fused_ln" (0 never; 1 always, on 128-column tiles; 3 always, on 256-column tiles; 2 = chosen per launch, the
+ * default: launches of at most "fused_ln_max_groups" (default 2) layers on all tokens - one layer on 128-column
+ * tiles, more on 256-column tiles - and launches of at most "fused_ln_max_rows" (default 0) rows per layer; any
+ * time): the attention-output and FFN-down projections carry the LayerNorm that follows them: the CTAs holding the
+ * column blocks of the same 128 rows form a thread-block cluster and exchange per-row statistics through
+ * distributed shared memory, so the pre-normalisation sum never goes to global memory and no LayerNorm launch
+ * follows.  All settings give the same bits (every LayerNorm of the library sums its row statistics over the same
+ * 64-column segments in the same order, every projection sums over K in one sequence).  Measured: faster than the
+ * separate launches while the launch is a single round of tiles (one or two layers of the 32 x 128 batch), slower
+ * beyond, where the separate LayerNorm hides the same latencies behind full occupancy.
  * key "overlap_cls" (0/1, default 1, any time): where a wave holds layers on all tokens and last branch
  * layers, the first-token attention of the latter runs on a stream the library creates for itself (in
  * mt_bind_memory), forked from the caller's stream after the wave's Q/K/V projection and joined before the next
@@ -332,6 +335,11 @@ int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d
 int mt_kernel_linear_layernorm(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
                                const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32, int32_t M,
                                int32_t N, int32_t K, float eps, uint32_t* d_status, void* stream);
+/* The same with the accumulator tile width chosen by the caller: 128 (clusters of N / 128 CTAs, as above) or 256
+ * (clusters of N / 256 CTAs; tcgen05.mma at its full rate, for launches with many row blocks).  Identical bits. */
+int mt_kernel_linear_layernorm_tiles(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
+                                     const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32, int32_t M,
+                                     int32_t N, int32_t K, float eps, int32_t tile_cols, uint32_t* d_status, void* stream);
 
 /* ctx[B*S, heads*64] = softmax(QK^T/8 masked to keys < length) V per (sequence, head), from the
  * packed projection qkv[B*S, 3*heads*64] = [Q | K | V].  Rows at positions >= length are written as 0.

@@ -63,6 +63,7 @@ SIGNATURES = {
     "mt_kernel_quantize_rows": (C.c_int, [_P, _P, _P, _I32, _I32, _P]),
     "mt_kernel_linear_fp8": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_linear_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _P, _P]),
+    "mt_kernel_linear_layernorm_tiles": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _I32, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
@@ -139,12 +140,13 @@ def mt_kernel_linear_fp8(xq, scale_x, wq, scale_w, bias, residual, y, epilogue: 
                                       _ptr(y), M, N, K, epilogue, _ptr(status), _stream(stream)), "mt_kernel_linear_fp8")
 
 
-def mt_kernel_linear_layernorm(x, w, bias, residual, gamma, beta, y, y_f32, eps: float, status=None, stream=None) -> None:
+def mt_kernel_linear_layernorm(x, w, bias, residual, gamma, beta, y, y_f32, eps: float, status=None, stream=None,
+                               tile_cols: int = 128) -> None:
     M, K = x.shape
     N = w.shape[0]
-    _check(lib().mt_kernel_linear_layernorm(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta), _ptr(y),
-                                            _ptr(y_f32), M, N, K, eps, _ptr(status), _stream(stream)),
-           "mt_kernel_linear_layernorm")
+    _check(lib().mt_kernel_linear_layernorm_tiles(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(gamma), _ptr(beta),
+                                                  _ptr(y), _ptr(y_f32), M, N, K, eps, tile_cols, _ptr(status),
+                                                  _stream(stream)), "mt_kernel_linear_layernorm_tiles")
 
 
 def mt_kernel_attention(qkv, lengths, ctx, batch: int, seq: int, heads: int, stream=None,

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmt_bert.so")
-SOURCES = ["mt_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "gemm_ln_tcgen05.cu", "rowwise.cu", "noalloc.cu"]
+SOURCES = ["mt_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "gemm_ln_tcgen05.cu", "gemm_ln_wide_tcgen05.cu", "rowwise.cu", "noalloc.cu"]
 
 
 def sources():
@@ -23,7 +23,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, "mt_kernels.h"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "rowwise.cuh"), os.path.join(HERE, "..", "include", "mt_bert.h")]
+    deps = sources() + [os.path.join(CSRC, "mt_kernels.h"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "rowwise.cuh"), os.path.join(CSRC, "cluster_ptx.cuh"), os.path.join(HERE, "..", "include", "mt_bert.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -29,8 +29,8 @@
 // flag and the status word, all roles leave their loops, the peers' waits run out in turn, and every
 // CTA reaches the closing cluster barrier, after which tensor memory is freed.
 
+#include "cluster_ptx.cuh"
 #include "rowwise.cuh"
-#include "tc_ptx.cuh"
 
 namespace mt {
 namespace {
@@ -47,54 +47,6 @@ constexpr int kLnStatsBytes = 2 * kLnMaxCluster * 2 * kGemmBlockM * 8;   // [par
 constexpr uint32_t kLnTmemCols = 256;
 constexpr int kLnSmemBytes = kLnStages * (kLnABytes + kLnBBytes) + kLnEpilogueWarps * 2 * kLnStagingBytes +
                              kLnStatsBytes + 512 + 1024;
-
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait that also makes the peers' shared-memory writes (released at cluster scope) visible.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  unsigned long long t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((it & 0xFFu) == 0xFFu) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ void st_cluster_f2(uint32_t cluster_addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(cluster_addr), "f"(a), "f"(b) : "memory");
-}
-// Release at cluster scope once, then arrivals that carry no ordering of their own: one fence instead of
-// one per peer.
-__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
-__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ uint32_t cluster_id_x() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t cluster_count_x() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
-  return r;
-}
 
 __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_constant__ GemmLnParams p) {
   extern __shared__ uint8_t smem_raw[];

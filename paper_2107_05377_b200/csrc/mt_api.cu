@@ -82,6 +82,7 @@ struct LayerTail {
   int32_t count = 0;
   // each residual GEMM together with the LayerNorm after it, as one cluster launch (option "fused_ln")
   bool ln_fused = false;
+  bool ln_wide = false;      // ... on 128 x 256 accumulator tiles (clusters of N / 256): launches with many row blocks
   bool down_fused = false;   // the FFN-down projection too (not with 8-bit operands: that GEMM is the plain kernel)
   GemmLnParams attn_out_ln, ffn_down_ln;
   // 8-bit operands: the inputs of the FFN-up and FFN-down projections are quantised row by row first
@@ -223,8 +224,8 @@ struct mt_model {
   bool attention_tc;  // attention on tcgen05 with tensor-memory accumulators when seq <= 128 (else mma.sync)
   int32_t gemm_pair;  // GEMMs as pairs of CTAs on 256-row tiles (cta_group::2): 0 never, 1 always, 2 by launch size
   bool early_heads;  // every task's head (and first-token tail) runs right after the wave that finishes its branch
-  int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always,
-                     // 2 for launches of at most fused_ln_max_groups layers
+  int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always on
+                     // 128-column tiles, 3 always on 256-column tiles, 2 by the launch (fused_ln_kind)
   int32_t fused_ln_max_groups;
   int32_t fused_ln_max_rows;
   // The first-token attention of the branches that end in a wave depends on the wave's QKV projection only
@@ -504,13 +505,24 @@ void choose_block_n(const mt_model* m, GemmParams* g, int epilogue, bool all_row
   g->block_n = gemm_block_n(g->N, epilogue, rows, groups < 1 ? 1 : groups, g->pair != 0, m->sm_count);
 }
 
-// Whether the residual GEMMs of `groups` layers carry their LayerNorm (see GemmLnParams).
-// (mode 2: few layers in the launch; optionally also launches of few rows per layer, the first-token tails,
-// which measured 0.3 % slower that way on the 32 x 128 batch; all ways give the same bits)
-bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) {
-  if (groups < 1 || !gemm_ln_supported(m->trunk.hidden) || m->fused_ln == 0) return false;
-  return m->fused_ln == 1 || groups <= m->fused_ln_max_groups || rows <= m->fused_ln_max_rows;
+// Whether the residual GEMMs of `groups` layers carry their LayerNorm (see GemmLnParams): 0 no, 1 on 128-column
+// tiles (clusters of N / 128 CTAs), 2 on 256-column tiles (clusters of N / 256).  All three ways give the same bits,
+// so the default chooses by the launch.  The fused epilogue is a chain of latencies (statistics through the
+// cluster, staged stores) run by eight warps per CTA; it only beats the separate LayerNorm launch, which hides the
+// same latencies behind full occupancy, while the whole launch is a single round of tiles.  Measured on the
+// 32 x 128 batch (about 2409 valid rows per layer): one layer per launch - narrow tiles, 12.5 + 23.4 us against
+// 8.8 + 6 + 20.1 + 6 us; two layers - wide tiles, 18.2 + 32.8 us against 18.9 + 40.1 us for the narrow ones; three
+// layers - separate launches, 15 + 8 + 40 + 8 us against 25 + 60 us (narrow) or 31 + 62 us (wide).
+// The first-token tails (a few rows per layer) keep the separate launches unless fused_ln_max_rows says otherwise.
+int fused_ln_kind(const mt_model* m, int32_t groups, int64_t rows) {
+  if (groups < 1 || !gemm_ln_supported(m->trunk.hidden) || m->fused_ln == 0) return 0;
+  if (m->fused_ln == 1) return 1;
+  if (m->fused_ln == 3) return 2;
+  if (rows <= m->fused_ln_max_rows) return 1;
+  if (rows <= m->max_batch || groups > m->fused_ln_max_groups) return 0;   // a first-token tail, or many layers
+  return groups == 1 ? 1 : 2;
 }
+bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) { return fused_ln_kind(m, groups, rows) != 0; }
 // Launches of steps 3-7 for `groups` layers.
 int32_t tail_launches(const mt_model* m, int32_t groups, int64_t rows) {
   const bool fused = use_fused_ln(m, groups, rows);
@@ -555,6 +567,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->ln1.eps = t->ln2.eps = m->trunk.ln_eps;
   t->count = 0;
   t->ln_fused = use_fused_ln(m, groups, rows);
+  t->ln_wide = fused_ln_kind(m, groups, rows) == 2;
   t->down_fused = t->ln_fused && !m->fp8;
   if (t->ln_fused) {
     auto init_ln = [&](GemmLnParams* g, int32_t K) {
@@ -613,6 +626,8 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
       cudaError_t err;
       if ((err = make_tmap(&g->tmap_x[i], x, g->M, g->K, kGemmBlockM, kGemmBlockK, false)) != cudaSuccess) return err;
       if ((err = make_tmap(&g->tmap_w[i], w_ptr(m, w), g->N, g->K, 128, kGemmBlockK, false)) != cudaSuccess) return err;
+      if ((err = make_tmap(&g->tmap_w256[i], w_ptr(m, w), g->N, g->K, 256, kGemmBlockK, false)) != cudaSuccess) return err;
+      g->residual[i] = res;
       if ((err = make_tmap(&g->tmap_res[i], res, g->M, g->N, 32, 32, true)) != cudaSuccess) return err;
       if ((err = make_tmap(&g->tmap_y[i], y, g->M, g->N, 32, 64, false)) != cudaSuccess) return err;
       if ((err = make_tmap(&g->tmap_y32[i], y32, g->M, g->N, 32, 32, true)) != cudaSuccess) return err;
@@ -1024,7 +1039,7 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
     return MT_OK;
   }
   if (strcmp(key, "fused_ln") == 0) {
-    if (value < 0 || value > 2) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1 or 2");
+    if (value < 0 || value > 3) return fail(m, MT_ERR_INVALID_ARG, "fused_ln must be 0, 1, 2 or 3");
     m->fused_ln = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
@@ -1352,7 +1367,9 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
   do {                                                                                                                 \
     LayerTail* t_ = (tail);                                                                                            \
     if (t_->ln_fused) {                                                                                                \
-      MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm_ln(t_->attn_out_ln, stream), "attention output GEMM + LayerNorm");       \
+      MT_TIMED(MT_CLASS_ATTN_OUT, t_->ln_wide ? launch_gemm_ln_wide(t_->attn_out_ln, stream)                          \
+                                              : launch_gemm_ln(t_->attn_out_ln, stream),                              \
+               "attention output GEMM + LayerNorm");                                                                   \
     } else {                                                                                                           \
       MT_TIMED(MT_CLASS_ATTN_OUT, launch_gemm(t_->attn_out, kEpiBiasResidual, m->sm_count, stream), "attention output GEMM"); \
       MT_TIMED(MT_CLASS_LN1, launch_layernorm(t_->ln1, stream), "LayerNorm 1");                                        \
@@ -1361,7 +1378,9 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
     MT_TIMED(MT_CLASS_FFN_UP, launch_gemm(t_->ffn_up, kEpiBiasGelu, m->sm_count, stream), "FFN up GEMM");              \
     if (t_->fp8) MT_TIMED(MT_CLASS_QUANT, launch_quantize_rows(t_->q_f, stream), "quantising the FFN intermediate");   \
     if (t_->down_fused) {                                                                                              \
-      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm_ln(t_->ffn_down_ln, stream), "FFN down GEMM + LayerNorm");               \
+      MT_TIMED(MT_CLASS_FFN_DOWN, t_->ln_wide ? launch_gemm_ln_wide(t_->ffn_down_ln, stream)                          \
+                                              : launch_gemm_ln(t_->ffn_down_ln, stream),                              \
+               "FFN down GEMM + LayerNorm");                                                                           \
     } else {                                                                                                           \
       MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t_->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");  \
       MT_TIMED(MT_CLASS_LN2, launch_layernorm(t_->ln2, stream), "LayerNorm 2");                                        \
@@ -1603,6 +1622,14 @@ int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d
 int mt_kernel_linear_layernorm(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
                                const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32, int32_t M, int32_t N,
                                int32_t K, float eps, uint32_t* d_status, void* stream) {
+  return mt_kernel_linear_layernorm_tiles(d_x, d_w, d_bias, d_residual, d_gamma, d_beta, d_y, d_y_f32, M, N, K, eps, 128,
+                                          d_status, stream);
+}
+
+int mt_kernel_linear_layernorm_tiles(const void* d_x, const void* d_w, const void* d_bias, const void* d_residual,
+                                     const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32, int32_t M,
+                                     int32_t N, int32_t K, float eps, int32_t tile_cols, uint32_t* d_status, void* stream) {
+  if (tile_cols != 128 && tile_cols != 256) return MT_ERR_INVALID_ARG;
   if (d_x == nullptr || d_w == nullptr || d_bias == nullptr || d_residual == nullptr || d_gamma == nullptr ||
       d_beta == nullptr || d_y == nullptr || d_y_f32 == nullptr || M < 1 || !gemm_ln_supported(N) || K < 64 || K % 64 != 0 ||
       !(eps >= 0.f))
@@ -1612,6 +1639,7 @@ int mt_kernel_linear_layernorm(const void* d_x, const void* d_w, const void* d_b
   p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.eps = eps; p.status = d_status;
   if (make_tmap(&p.tmap_x[0], d_x, M, K, kGemmBlockM, kGemmBlockK, false) != cudaSuccess ||
       make_tmap(&p.tmap_w[0], d_w, N, K, 128, kGemmBlockK, false) != cudaSuccess ||
+      make_tmap(&p.tmap_w256[0], d_w, N, K, 256, kGemmBlockK, false) != cudaSuccess ||
       make_tmap(&p.tmap_res[0], d_residual, M, N, 32, 32, true) != cudaSuccess ||
       make_tmap(&p.tmap_y[0], d_y, M, N, 32, 64, false) != cudaSuccess ||
       make_tmap(&p.tmap_y32[0], d_y_f32, M, N, 32, 32, true) != cudaSuccess)
@@ -1619,7 +1647,9 @@ int mt_kernel_linear_layernorm(const void* d_x, const void* d_w, const void* d_b
   p.bias[0] = static_cast<const bf16*>(d_bias);
   p.gamma[0] = static_cast<const bf16*>(d_gamma);
   p.beta[0] = static_cast<const bf16*>(d_beta);
-  return launch_gemm_ln(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+  p.residual[0] = static_cast<const float*>(d_residual);
+  const cudaError_t e = tile_cols == 256 ? launch_gemm_ln_wide(p, as_stream(stream)) : launch_gemm_ln(p, as_stream(stream));
+  return e == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
 int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx, int32_t batch, int32_t seq,

@@ -158,9 +158,11 @@ cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream);
 struct alignas(64) GemmLnParams {
   CUtensorMap tmap_x[kMaxGroups];     // X_g: dims {K, M}, box {64, 128}
   CUtensorMap tmap_w[kMaxGroups];     // W_g: dims {K, N}, box {64, 128}
+  CUtensorMap tmap_w256[kMaxGroups];  // W_g with a box of 256 rows (the kernel on 256-column tiles)
   CUtensorMap tmap_res[kMaxGroups];   // residual_g fp32: dims {N, M}, box {32, 32}
   CUtensorMap tmap_y[kMaxGroups];     // Y_g bf16: dims {N, M}, box {64, 32}
   CUtensorMap tmap_y32[kMaxGroups];   // Y_g fp32: dims {N, M}, box {32, 32}
+  const float* residual[kMaxGroups];  // the same residual by pointer (fp32 [M, N]; the kernel on 256-column tiles)
   const bf16* bias[kMaxGroups];
   const bf16* gamma[kMaxGroups];
   const bf16* beta[kMaxGroups];
@@ -173,6 +175,10 @@ struct alignas(64) GemmLnParams {
 // N must be 768 or 1024 (clusters of 6 or 8 CTAs), K a multiple of 64.
 bool gemm_ln_supported(int N);
 cudaError_t launch_gemm_ln(const GemmLnParams& p, cudaStream_t stream);
+// The same on 128 x 256 accumulator tiles, clusters of N / 256 CTAs (tmap_w256 and residual filled): identical bits,
+// half the CTAs per row block and full-rate tcgen05.mma - for launches with many row blocks.
+bool gemm_ln_wide_supported(int N);
+cudaError_t launch_gemm_ln_wide(const GemmLnParams& p, cudaStream_t stream);
 
 struct EmbedParams {
   const int32_t* token_ids;

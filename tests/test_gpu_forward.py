@@ -129,6 +129,10 @@ def test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches():
         assert torch.equal(m_fus.debug_hidden(t, layer, B, S), m_sep.debug_hidden(t, layer, B, S)), (t, layer)
     _, auto = run_model(cfg, blob, batch, fused_ln=2)
     assert torch.equal(auto, separate)
+    m_wide, wide = run_model(cfg, blob, batch, debug=True, fused_ln=3)   # 256-column tiles, clusters of three
+    assert torch.equal(wide, separate)
+    for t, layer in ((-1, 1), (-1, 3), (1, 1), (1, 2), (3, 1)):
+        assert torch.equal(m_wide.debug_hidden(t, layer, B, S), m_sep.debug_hidden(t, layer, B, S)), (t, layer)
     # all rows in the last layers, padded layout: more and fuller row blocks
     m_full, full = run_model(cfg, blob, batch, debug=True, cls_only=0, pack_tokens=0, fused_ln=1)
     check_against_oracle(cfg, wf, batch, m_full, full, rows=range(6), cls_only=False)
@@ -138,6 +142,10 @@ def test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches():
     b8 = synth.batch_glue8(big)
     _, sep8 = run_model(big, blob8, b8, fused_ln=0)
     m8, first = run_model(big, blob8, b8, fused_ln=1)
+    assert torch.equal(first, sep8)
+    _, wide8 = run_model(big, blob8, b8, fused_ln=3)
+    assert torch.equal(wide8, sep8)
+    m8, first = run_model(big, blob8, b8)            # the default: chosen per launch
     assert torch.equal(first, sep8)
     tok, seg, lens = dev_batch(b8)
     again = torch.zeros_like(first)

@@ -67,8 +67,10 @@ def test_linear_matches_oracle(M, N, K, epi, pair):
     (2409, 768, 3072),        # FFN down + LayerNorm at the valid-token count of the 32 x 128 batch
     (4096, 768, 768),         # more row blocks than clusters fit the GPU at once: several tiles per cluster
     (700, 1024, 4096),        # BERT-large width: clusters of eight
+    (7227, 768, 768),         # three layers' worth of valid tokens: several tiles per cluster
 ])
-def test_linear_layernorm_cluster_matches_oracle_and_separate_kernels(M, N, K):
+@pytest.mark.parametrize("tile_cols", [128, 256])
+def test_linear_layernorm_cluster_matches_oracle_and_separate_kernels(M, N, K, tile_cols):
     """Residual GEMM + LayerNorm in one cluster launch (row statistics through distributed shared memory):
     against the oracle's linear + residual + layer_norm, and bit for bit against the plain residual GEMM
     followed by the LayerNorm kernel, which sums the row statistics in the same order."""
@@ -84,7 +86,7 @@ def test_linear_layernorm_cluster_matches_oracle_and_separate_kernels(M, N, K):
     y32 = torch.full((M + 8, N), float("nan"), dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     xd, wd, bd, bed = to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(bb), to_dev_bf16(beb)
-    mt.mt_kernel_linear_layernorm(xd, wd, bd, res, g_dev, bed, y[:M], y32[:M], 1e-12, status=status)
+    mt.mt_kernel_linear_layernorm(xd, wd, bd, res, g_dev, bed, y[:M], y32[:M], 1e-12, status=status, tile_cols=tile_cols)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert torch.isnan(y[M:].float()).all() and torch.isnan(y32[M:]).all(), "rows beyond M were written"

@@ -91,6 +91,8 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 5 + 2
     m.set_option("fused_ln_max_rows", 128)   # also the first-token tail (32 rows per layer)
     assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 3 + 2
+    m.set_option("fused_ln", 3)
+    assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 3 + 2
     m.set_option("fused_ln", 0)
     # waves 7, 8, 9 mix layers on all tokens (7 launches) with last branch layers, which only add the
     # first-token attention there; wave 10 holds a last layer alone (projection + first-token attention);
