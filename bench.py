@@ -43,7 +43,8 @@ L2_FLUSH_BYTES = 256 << 20    # larger than the 126 MB L2
 # launches of the forwards of `bench.py --steps 2`); the figure and the digest of the kernel sources it was
 # taken on are two lines of the launch-list summary under profiles/, and it is reported only while the
 # sources still have that digest.
-GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_ln_tcgen05.cu", "tc_ptx.cuh", "rowwise.cuh")
+GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_ln_tcgen05.cu", "gemm_ln_wide_tcgen05.cu", "cluster_ptx.cuh", "tc_ptx.cuh",
+                "rowwise.cuh")
 TRAFFIC_SUMMARY = os.path.join("profiles", "bench_glue8_b32_s128_launch_list.md")
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16 of the part, for context beside the measured peak
 STEADY_SECONDS = 2.0

@@ -4,6 +4,8 @@
     python -m paper_2107_05377_b200.kernel_bench linear_ln --m 4096 --n 768 --k 3072   # residual GEMM + LayerNorm, one launch
     python -m paper_2107_05377_b200.kernel_bench attention --batch 32 --seq 128 --heads 12
     python -m paper_2107_05377_b200.kernel_bench layernorm --rows 4096 --hidden 768
+    python -m paper_2107_05377_b200.kernel_bench embed --batch 256 --seq 128
+    python -m paper_2107_05377_b200.kernel_bench linear_fp8 --m 4096 --n 2304 --k 768            # E4M3 operands
     python -m paper_2107_05377_b200.kernel_bench suite          # the shapes of the 32 x 128 workload
 
 Times `--iters` launches between CUDA events on the launching stream after `--warmup` launches; with
@@ -98,7 +100,7 @@ def bench_linear_fp8(m, n, k, epilogue, iters, warmup, flush):
             "tflops": 2.0 * m * n * k / ms / 1e9, "quantize_rows_us": 1e3 * ms_q}
 
 
-def bench_linear_ln(m, n, k, iters, warmup, flush):
+def bench_linear_ln(m, n, k, iters, warmup, flush, tile_cols=128):
     x = torch.randn(m, k, device="cuda").to(torch.bfloat16)
     w = (0.02 * torch.randn(n, k, device="cuda")).to(torch.bfloat16)
     b = (0.02 * torch.randn(n, device="cuda")).to(torch.bfloat16)
@@ -107,10 +109,10 @@ def bench_linear_ln(m, n, k, iters, warmup, flush):
     r = torch.randn(m, n, device="cuda")
     y = torch.empty(m, n, device="cuda", dtype=torch.bfloat16)
     y32 = torch.empty(m, n, device="cuda")
-    ms = _time(lambda: mt.mt_kernel_linear_layernorm(x, w, b, r, g, be, y, y32, 1e-12), iters, warmup, flush)
+    ms = _time(lambda: mt.mt_kernel_linear_layernorm(x, w, b, r, g, be, y, y32, 1e-12, tile_cols=tile_cols), iters, warmup, flush)
     flops = 2.0 * m * n * k
     bytes_ = 2.0 * (m * k + n * k) + (4.0 + 2.0 + 4.0) * m * n
-    return {"kernel": "linear_ln", "M": m, "N": n, "K": k, "us": 1e3 * ms, "tflops": flops / ms / 1e9,
+    return {"kernel": "linear_ln", "tile_cols": tile_cols, "M": m, "N": n, "K": k, "us": 1e3 * ms, "tflops": flops / ms / 1e9,
             "min_gbytes_per_s": bytes_ / ms / 1e6}
 
 
@@ -127,6 +129,24 @@ def bench_attention(batch, seq, heads, len_lo, iters, warmup, flush):
             "gbytes_per_s": bytes_ / ms / 1e6, "valid_tflops": flops / ms / 1e9}
 
 
+def bench_embed(batch, seq, hidden, iters, warmup, flush):
+    vocab = 30522
+    tok = torch.randint(1000, vocab, (batch, seq), device="cuda", dtype=torch.int32)
+    seg = torch.randint(0, 2, (batch, seq), device="cuda", dtype=torch.int32)
+    lens = torch.full((batch,), seq, device="cuda", dtype=torch.int32)
+    word = (0.02 * torch.randn(vocab, hidden, device="cuda")).to(torch.bfloat16)
+    pos = (0.02 * torch.randn(512, hidden, device="cuda")).to(torch.bfloat16)
+    typ = (0.02 * torch.randn(2, hidden, device="cuda")).to(torch.bfloat16)
+    g = torch.ones(hidden, device="cuda", dtype=torch.bfloat16)
+    b = torch.zeros(hidden, device="cuda", dtype=torch.bfloat16)
+    h0 = torch.empty(batch * seq, hidden, device="cuda", dtype=torch.bfloat16)
+    h32 = torch.empty(batch * seq, hidden, device="cuda")
+    ms = _time(lambda: mt.mt_kernel_embed(tok, seg, lens, word, pos, typ, g, b, h0, 1e-12, h0_f32=h32), iters, warmup, flush)
+    # per token: one word row and one position row read (bf16), the bf16 and the fp32 state written
+    return {"kernel": "embed", "batch": batch, "seq": seq, "hidden": hidden, "us": 1e3 * ms,
+            "gbytes_per_s": 10.0 * batch * seq * hidden / ms / 1e6}
+
+
 def bench_layernorm(rows, hidden, iters, warmup, flush):
     x = torch.randn(rows, hidden, device="cuda")
     g = torch.ones(hidden, device="cuda", dtype=torch.bfloat16)
@@ -140,7 +160,7 @@ def bench_layernorm(rows, hidden, iters, warmup, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["linear", "linear_fp8", "linear_ln", "attention", "layernorm", "suite"])
+    ap.add_argument("kernel", choices=["linear", "linear_fp8", "linear_ln", "attention", "layernorm", "embed", "suite"])
     ap.add_argument("--m", type=int, default=4096)
     ap.add_argument("--n", type=int, default=2304)
     ap.add_argument("--k", type=int, default=768)
@@ -155,6 +175,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--flush", action="store_true")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
+    ap.add_argument("--tile-cols", type=int, default=128, help="linear_ln: accumulator tile width, 128 or 256")
     ap.add_argument("--block-n", type=int, default=0, help="linear: force the tile width (0 = automatic)")
     ap.add_argument("--pair", action="store_true", help="linear: pairs of CTAs on 256-row tiles (cta_group::2)")
     ap.add_argument("--mma-sync", action="store_true", help="attention: the mma.sync kernel also where seq <= 128")
@@ -170,11 +191,13 @@ def main():
     elif a.kernel == "linear_fp8":
         print(json.dumps(bench_linear_fp8(a.m, a.n, a.k, a.epilogue, a.iters, a.warmup, a.flush)))
     elif a.kernel == "linear_ln":
-        print(json.dumps(bench_linear_ln(a.m, a.n, a.k, a.iters, a.warmup, a.flush)))
+        print(json.dumps(bench_linear_ln(a.m, a.n, a.k, a.iters, a.warmup, a.flush, a.tile_cols)))
     elif a.kernel == "attention":
         print(json.dumps(bench_attention(a.batch, a.seq, a.heads, a.len_lo, a.iters, a.warmup, a.flush)))
     elif a.kernel == "layernorm":
         print(json.dumps(bench_layernorm(a.rows, a.hidden, a.iters, a.warmup, a.flush)))
+    elif a.kernel == "embed":
+        print(json.dumps(bench_embed(a.batch, a.seq, a.hidden, a.iters, a.warmup, a.flush)))
     else:
         for m in (2409, 4096, 24576):   # the valid tokens of the 32 x 128 batch, its padded rows, six layers of them
             for (n, k, e) in ((2304, 768, 0), (768, 768, 2), (3072, 768, 1), (768, 3072, 2)):
