@@ -507,17 +507,13 @@ __global__ void __launch_bounds__(kTcThreads, 2) attention_tc_tiled_kernel(const
 cudaError_t launch_attention_tc(const AttnParams& p, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.batch < 1 || p.seq < 1 || p.seq > kAttnTensorMemoryMaxSeq)
     return cudaErrorInvalidValue;
-  static int configured_device = -1;   // the attributes are per function and per device
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  static PerDeviceOnce once;
+  cudaError_t e = per_device_once(once, [&](int) {
+    cudaError_t r = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    if (r != cudaSuccess) return r;
+    return cudaFuncSetAttribute(attention_tc_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTlSmemBytes);
+  });
   if (e != cudaSuccess) return e;
-  if (configured_device != dev) {
-    e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attention_tc_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTlSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured_device = dev;
-  }
   if (p.seq <= kTcRows) {
     dim3 grid(p.heads, p.batch, p.n_groups);
     return launch_kernel(attention_tc_kernel, grid, dim3(kTcThreads), kTcSmemBytes, stream, p);

@@ -374,37 +374,36 @@ cudaError_t launch_gemm_ln(const GemmLnParams& p, cudaStream_t stream) {
       p.M < 1)
     return cudaErrorInvalidValue;
   const int cluster_size = p.N / kLnBlockN;
+  // per device: shared-memory opt-in and, per cluster size, the number of clusters that fit the GPU at once
+  static PerDeviceOnce once;
+  static int max_clusters[kMaxDevices][2] = {};
   int dev = 0;
-  cudaError_t err = cudaGetDevice(&dev);
+  cudaError_t err = per_device_once(once, [&](int d) {
+    cudaError_t r = cudaFuncSetAttribute(gemm_ln_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnSmemBytes);
+    if (r != cudaSuccess) return r;
+    for (int which = 0; which < 2; ++which) {
+      const int cs = which == 0 ? 6 : 8;
+      cudaLaunchConfig_t q = {};
+      q.gridDim = dim3(cs * 64);
+      q.blockDim = dim3(kLnThreads);
+      q.dynamicSmemBytes = kLnSmemBytes;
+      cudaLaunchAttribute a[1];
+      a[0].id = cudaLaunchAttributeClusterDimension;
+      a[0].val.clusterDim.x = cs;
+      a[0].val.clusterDim.y = 1;
+      a[0].val.clusterDim.z = 1;
+      q.attrs = a;
+      q.numAttrs = 1;
+      int n = 0;
+      r = cudaOccupancyMaxActiveClusters(&n, gemm_ln_tcgen05, &q);
+      if (r != cudaSuccess) return r;
+      max_clusters[d][which] = n;
+    }
+    return cudaSuccess;
+  }, &dev);
   if (err != cudaSuccess) return err;
-  // per device and cluster size: shared-memory opt-in and the number of clusters that fit the GPU at once
-  static int max_clusters[64][2] = {};
-  static bool configured[64] = {};
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!configured[dev]) {
-    err = cudaFuncSetAttribute(gemm_ln_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, kLnSmemBytes);
-    if (err != cudaSuccess) return err;
-    configured[dev] = true;
-  }
-  int& fit = max_clusters[dev][cluster_size == 8 ? 1 : 0];
-  if (fit == 0) {
-    cudaLaunchConfig_t q = {};
-    q.gridDim = dim3(cluster_size * 64);
-    q.blockDim = dim3(kLnThreads);
-    q.dynamicSmemBytes = kLnSmemBytes;
-    cudaLaunchAttribute a[1];
-    a[0].id = cudaLaunchAttributeClusterDimension;
-    a[0].val.clusterDim.x = cluster_size;
-    a[0].val.clusterDim.y = 1;
-    a[0].val.clusterDim.z = 1;
-    q.attrs = a;
-    q.numAttrs = 1;
-    int n = 0;
-    err = cudaOccupancyMaxActiveClusters(&n, gemm_ln_tcgen05, &q);
-    if (err != cudaSuccess) return err;
-    if (n < 1) return cudaErrorLaunchOutOfResources;
-    fit = n;
-  }
+  const int fit = max_clusters[dev][cluster_size == 8 ? 1 : 0];
+  if (fit < 1) return cudaErrorLaunchOutOfResources;
   const int tiles = ((p.M + kGemmBlockM - 1) / kGemmBlockM) * p.n_groups;
   const int clusters = tiles < fit ? tiles : fit;
   return launch_kernel(gemm_ln_tcgen05, dim3(clusters * cluster_size), dim3(kLnThreads), kLnSmemBytes, stream, p,

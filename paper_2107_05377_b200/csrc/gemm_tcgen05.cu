@@ -472,17 +472,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 template <int BN, int EPI, bool PAIR, bool FP8 = false>
 cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
   auto kernel = gemm_bf16_tcgen05<BN, EPI, PAIR, FP8>;
-  static bool configured = false;  // per instantiation; the attribute is per function and per device
-  static int configured_device = -1;
-  int dev = 0;
-  cudaError_t err = cudaGetDevice(&dev);
+  static PerDeviceOnce once;   // per instantiation
+  cudaError_t err = per_device_once(once, [&](int) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN, PAIR, EPI));
+  });
   if (err != cudaSuccess) return err;
-  if (!configured || configured_device != dev) {
-    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(BN, PAIR, EPI));
-    if (err != cudaSuccess) return err;
-    configured = true;
-    configured_device = dev;
-  }
   constexpr int tile_m = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
   const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN) * p.n_groups;
   const int workers_max = PAIR ? sm_count / 2 : sm_count;

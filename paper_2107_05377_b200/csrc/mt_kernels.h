@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 namespace mt {
 
 typedef __nv_bfloat16 bf16;
@@ -31,6 +33,30 @@ extern bool g_use_pdl;
 #ifdef __CUDACC__
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Per-function launch set-up (the opt-in to large dynamic shared memory, occupancy queries) is per device: this runs
+// `setup(dev)` once per device and call site, under a lock, so that launches from several host threads or on
+// several devices of one process never race on it.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+  std::mutex mu;
+  bool done[kMaxDevices] = {};
+};
+template <typename F>
+cudaError_t per_device_once(PerDeviceOnce& state, F&& setup, int* device_out = nullptr) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (device_out != nullptr) *device_out = dev;
+  std::lock_guard<std::mutex> lock(state.mu);
+  if (!state.done[dev]) {
+    e = setup(dev);
+    if (e != cudaSuccess) return e;
+    state.done[dev] = true;
+  }
+  return cudaSuccess;
+}
 
 // cluster_x > 1 launches the grid as thread-block clusters of that many CTAs along x.
 template <typename Param>
