@@ -152,3 +152,44 @@ def test_fp8_glue8_tree_32x128_sampled_rows_and_merged_equals_standalone():
         st_blob = synth.pack_weights(st_cfg, synth.select_task_weights(w, t))
         _, single = fp8_forward(st_cfg, st_blob, batch)
         assert torch.equal(single, logits[:, offs[t]:offs[t] + cfg.tasks[t].num_classes]), t
+
+
+def test_fp8_task_reload_requantises_that_task_only():
+    """Per-task update under reduced precision: the reloaded task's 8-bit copies are rebuilt from its new bf16
+    weights, the other tasks keep their bits."""
+    cfg = synth.TreeConfig(trunk_layers=4, tasks=(synth.TaskSpec(4, 1, 2), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 1, 1, token_level=True)))
+    w, blob, wf = cached_weights(cfg, 0)
+    batch = synth.make_batch(cfg, 3, 64, 20, 64, seed=2)
+    B, S = batch.token_ids.shape
+    model = mt.MTModel(cfg, B, S, fp8_gemm=True)
+    model.load_weights(blob)
+    tok, seg, lens = dev_batch(batch)
+
+    def run():
+        logits = torch.full((B, cfg.total_classes), float("nan"), device="cuda")
+        tlog = torch.full((B, S, cfg.total_token_classes), float("nan"), device="cuda")
+        model.forward_tokens(tok, seg, lens, logits, tlog)
+        torch.cuda.synchronize()
+        assert model.poll_status() == 0
+        return logits, tlog
+
+    base, base_t = run()
+    new_task = synth.make_task_weights(cfg, 1, seed=77)
+    model.load_task_weights(1, synth.pack_task_weights(cfg, 1, new_task))
+    after, after_t = run()
+    offs = cfg.logit_offsets
+    assert torch.equal(after[:, offs[0]:offs[0] + 2], base[:, offs[0]:offs[0] + 2])
+    valid = torch.from_numpy(np.arange(S)[None, :] < batch.lengths[:, None]).cuda()
+    assert torch.equal(after_t[valid], base_t[valid])
+    assert not torch.equal(after[:, offs[1]:offs[1] + 3], base[:, offs[1]:offs[1] + 3])
+    wf2 = dict(wf)
+    wf2["tasks"] = list(wf["tasks"])
+    wf2["tasks"][1] = synth.widen(new_task)
+    tl = []
+    want = orc.forward_batch_mt(batch.token_ids, batch.segment_ids, batch.lengths, wf2, task_triples(cfg), cfg.heads,
+                                cfg.ln_eps, layer_fn=f8.encoder_layer_fp8, token_logits_out=tl)
+    assert np.max(np.abs(after.cpu().numpy().astype(np.float64) - want)) <= FP8_LOGITS_VS_FP8_ORACLE
+    got_t = after_t.cpu().numpy().astype(np.float64)
+    v = valid.cpu().numpy()
+    assert np.max(np.abs(got_t[v] - tl[0][v])) <= FP8_LOGITS_VS_FP8_ORACLE
