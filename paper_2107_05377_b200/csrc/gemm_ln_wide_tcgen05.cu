@@ -97,11 +97,16 @@ __global__ void __launch_bounds__(kLwThreads, 1) gemm_ln_wide_tcgen05(const __gr
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  grid_dependency_wait();
-  grid_launch_dependents();
-
+  // rows in use: all M, or fewer when the token layout is packed (a device-side count written by the forward's
+  // first kernel).  When this kernel starts, every kernel of the stream but its immediate predecessor has
+  // completed (each waits for its own predecessor before it lets its dependents start), and the immediate
+  // predecessor is never the one that writes the count: it is read before the dependency wait, off the
+  // critical path.
   int m_rows = p.M;
   if (p.m_valid != nullptr) m_rows = min(m_rows, *p.m_valid);
+
+  grid_dependency_wait();
+  grid_launch_dependents();
   const int total_tiles = ((m_rows + kGemmBlockM - 1) / kGemmBlockM) * p.n_groups;   // (row block, group) pairs
 
   if (warp == 0) {

@@ -159,11 +159,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       }
     }
   }
-  grid_dependency_wait();
-  grid_launch_dependents();
-  // rows in use: all M, or fewer when the token layout is packed (a device-side count)
+  // rows in use: all M, or fewer when the token layout is packed (a device-side count written by the forward's
+  // first kernel).  When this kernel starts, every kernel of the stream but its immediate predecessor has
+  // completed (each waits for its own predecessor before it lets its dependents start), and the immediate
+  // predecessor is never the one that writes the count: it is read before the dependency wait, off the
+  // critical path.
   int m_rows = p.M;
   if (p.m_valid != nullptr) m_rows = min(m_rows, *p.m_valid);
+  grid_dependency_wait();
+  grid_launch_dependents();
   const int n_tiles_m = (m_rows + TILE_M - 1) / TILE_M;
   const int total_tiles = n_tiles_m * tiles_per_m;
 

@@ -17,9 +17,12 @@ __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormP
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
   const int g = blockIdx.y;
+  // (the count of rows in use was written by the forward's first kernel, never by the immediate predecessor: it
+  // may be read before the dependency wait)
+  const int rows_in_use = p.rows_valid != nullptr ? min(p.rows, *p.rows_valid) : p.rows;
   grid_dependency_wait();
   grid_launch_dependents();
-  if (row >= p.rows || (p.rows_valid != nullptr && row >= *p.rows_valid)) return;
+  if (row >= rows_in_use) return;
   const float* xin = p.x[g] + static_cast<size_t>(row) * H;
   float x[V][8];
 #pragma unroll
@@ -194,10 +197,10 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo) {
 __global__ void __launch_bounds__(kRowThreads) quantize_rows_kernel(const QuantParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.y;
+  int rows = p.rows;
+  if (p.rows_valid != nullptr) rows = min(rows, *p.rows_valid);   // (readable before the wait, as in layernorm_kernel)
   grid_dependency_wait();
   grid_launch_dependents();
-  int rows = p.rows;
-  if (p.rows_valid != nullptr) rows = min(rows, *p.rows_valid);
   const int row = blockIdx.x * (kRowThreads / 32) + warp;
   if (row >= rows) return;
   const bf16* x = p.x[g] + static_cast<size_t>(row) * p.cols;
