@@ -61,9 +61,9 @@ def flops_padded(cfg, layers, batch, seq):
     return layers * (2.0 * m * (4 * cfg.hidden * cfg.hidden + 2 * cfg.hidden * cfg.ffn) + batch * 4.0 * cfg.hidden * seq * seq)
 
 
-def run_tree(name, cfg, blob, batch, masks, iters, out):
+def run_tree(name, cfg, blob, batch, masks, iters, out, fp8=False):
     B, S = batch.token_ids.shape
-    model = binding.MTModel(cfg, B, S)
+    model = binding.MTModel(cfg, B, S, fp8_gemm=fp8)
     model.load_weights(blob)
     tok, seg, lens = _dev(batch)
     logits = torch.zeros(B, max(cfg.total_classes, 1), dtype=torch.float32, device="cuda")
@@ -130,6 +130,11 @@ def main():
     run_tree("glue8 tree, long sequences", cfg, blob, synth.make_batch(cfg, 16, 512, 128, 512, seed=1),
              [("all 8", 0xFF)], 20, out)
     run_tree("glue8 tree, headline shape", cfg, blob, synth.batch_glue8(cfg), [("all 8", 0xFF)], 50, out)
+    # the 8-bit projections (option "fp8_gemm") beside bf16: where a forward is made of tensor work, not launches
+    for B in (32, 256):
+        hb8 = synth.batch_glue8(cfg, B, 128)
+        run_tree("glue8 tree, lengths U[16,128], bf16", cfg, blob, hb8, [("all 8", 0xFF)], 20, out)
+        run_tree("glue8 tree, lengths U[16,128], E4M3 projections", cfg, blob, hb8, [("all 8", 0xFF)], 20, out, fp8=True)
     # time to each task's logits with heads scheduled as early as possible (the latency limitation of Section 5.2)
     hb = synth.batch_glue8(cfg)
     for early in (0, 1):
