@@ -112,7 +112,9 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
+    // the warp stays converged (all lanes wait on the barriers); the elected lane issues the copies
+    const bool leader = elect_one();
+    {
       int stage = 0;
       uint32_t phase = 0;
       long long issued = 0;
@@ -122,14 +124,16 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
         const int g = tile % p.n_groups;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(bar_full + 8 * stage, kLnABytes + kLnBBytes);
-          tma_load_2d(sA + stage * kLnABytes, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
-          tma_load_2d(sB + stage * kLnBBytes, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+          if (leader) {
+            mbar_expect_tx(bar_full + 8 * stage, kLnABytes + kLnBBytes);
+            tma_load_2d(sA + stage * kLnABytes, &p.tmap_x[g], kb * kGemmBlockK, m0, bar_full + 8 * stage);
+            tma_load_2d(sB + stage * kLnBBytes, &p.tmap_w[g], kb * kGemmBlockK, n0, bar_full + 8 * stage);
+          }
           ++issued;
           if (++stage == kLnStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
+      if (!ok && leader) {
         // aborting: give the copies still in flight the same limit to land before the CTA retires
         int s = stage;
         uint32_t ph = phase;
@@ -146,7 +150,9 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
-    if (lane == 0) {
+    // (the same: a converged warp, the elected lane issues the MMAs and the commits)
+    const bool leader = elect_one();
+    {
       constexpr uint32_t idesc = umma_idesc_bf16(kGemmBlockM, kLnBlockN);
       int stage = 0;
       uint32_t phase = 0;
@@ -160,16 +166,18 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t da = smem_desc_sw128(sA + stage * kLnABytes);
-          const uint64_t db = smem_desc_sw128(sB + stage * kLnBBytes);
+          if (leader) {
+            const uint64_t da = smem_desc_sw128(sA + stage * kLnABytes);
+            const uint64_t db = smem_desc_sw128(sB + stage * kLnBBytes);
 #pragma unroll
-          for (int k = 0; k < kGemmBlockK / 16; ++k)
-            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit(bar_empty + 8 * stage);
+            for (int k = 0; k < kGemmBlockK / 16; ++k)
+              umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_commit(bar_empty + 8 * stage);
+          }
           if (++stage == kLnStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(bar_acc_full + 8 * acc);
+        if (leader) umma_commit(bar_acc_full + 8 * acc);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }

@@ -140,22 +140,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   // either: the producer thread starts the W tiles of this CTA's first tile before it waits for
   // that kernel, so their trip from HBM overlaps its tail.  From the wait on, the previous kernel
   // has completed and its writes are visible.
-  int prefetched = 0;   // stages whose W tile is already on its way (producer thread only)
-  if (warp == 0 && lane == 0) {
+  int prefetched = 0;   // stages whose W tile is already on its way (producer warp only)
+  bool producer_leader = false;
+  if (warp == 0) {
+    producer_leader = elect_one();   // the warp stays converged; this lane issues the copies
     const int rem = worker % tiles_per_m;
     const int g = rem / n_tiles_n;
     const int n0 = (rem - g * n_tiles_n) * BN + static_cast<int>(rank) * (PAIR ? BN / 2 : 0);
-    prefetch_tensormap(&p.tmap_x[g]);
-    prefetch_tensormap(&p.tmap_w[g]);
     prefetched = k_blocks < STAGES ? k_blocks : STAGES;
-    for (int s = 0; s < prefetched; ++s) {
-      if (PAIR) {
-        // rank 0 announces the bytes of both CTAs' W parts on its barrier; either CTA's copy may land first
-        if (rank == 0) mbar_add_tx(bar_full + 8 * s, 2 * B_BYTES);
-        tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full_count + 8 * s);
-      } else {
-        mbar_add_tx(bar_full + 8 * s, B_BYTES);
-        tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full + 8 * s);
+    if (producer_leader) {
+      prefetch_tensormap(&p.tmap_x[g]);
+      prefetch_tensormap(&p.tmap_w[g]);
+      for (int s = 0; s < prefetched; ++s) {
+        if (PAIR) {
+          // rank 0 announces the bytes of both CTAs' W parts on its barrier; either CTA's copy may land first
+          if (rank == 0) mbar_add_tx(bar_full + 8 * s, 2 * B_BYTES);
+          tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full_count + 8 * s);
+        } else {
+          mbar_add_tx(bar_full + 8 * s, B_BYTES);
+          tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full + 8 * s);
+        }
       }
     }
   }
@@ -173,12 +177,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
+    {
       int stage = 0;
       uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
-      if (worker >= total_tiles && rank == 0) {
+      if (worker >= total_tiles && rank == 0 && producer_leader) {
         // no tile for this CTA (pair) after all (fewer rows in use than the grid was sized for): let
         // the early W tiles land before the CTA retires (in a pair, rank 1 is held by the exit barrier)
         for (int s = 0; s < prefetched; ++s) {
@@ -199,7 +203,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           const bool w_on_its_way = prefetched > 0;
           if (w_on_its_way) --prefetched;
-          if (PAIR) {
+          if (!producer_leader) {
+            // the other lanes only keep the warp together
+          } else if (PAIR) {
             if (rank == 0)
               mbar_expect_tx(bar_full + 8 * stage, 2 * A_BYTES + (w_on_its_way ? 0 : 2 * B_BYTES));
             tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], kb * KB_ELEMS, m0, bar_full_count + 8 * stage);
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok && rank == 0) {
+      if (!ok && rank == 0 && producer_leader) {
         // Aborting: wait (bounded) until the copies still in flight have landed, so that the
         // CTA does not retire underneath them.  The last min(issued, STAGES) fills are the ones
         // that may be pending; walk back over them.
@@ -234,7 +240,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
-    if (lane == 0 && rank == 0) {
+    // The whole warp walks the loop and waits on the barriers (it stays converged); the elected lane issues.
+    const bool leader = elect_one();
+    if (rank == 0) {
       constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(TILE_M, BN) : umma_idesc_bf16(TILE_M, BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -249,20 +257,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t da = smem_desc_sw128(sA + stage * A_BYTES);
-          const uint64_t db = smem_desc_sw128(sB + stage * B_BYTES);
+          if (leader) {
+            const uint64_t da = smem_desc_sw128(sA + stage * A_BYTES);
+            const uint64_t db = smem_desc_sw128(sB + stage * B_BYTES);
 #pragma unroll
-          for (int k = 0; k < kGemmBlockK / 16; ++k) {
-            // advancing one instruction along K (16 bf16 or 32 E4M3 = 32 bytes) inside the swizzled row: +2 in the address field
-            if (FP8) umma_e4m3(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            else if (PAIR) umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-            else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < kGemmBlockK / 16; ++k) {
+              // advancing one instruction along K (16 bf16 or 32 E4M3 = 32 bytes) inside the swizzled row: +2 in the address field
+              if (FP8) umma_e4m3(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+              else if (PAIR) umma_bf16_pair(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+              else umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
           }
-          if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        if (PAIR) umma_commit_pair(bar_acc_full + 8 * acc); else umma_commit(bar_acc_full + 8 * acc);
+        if (leader) {
+          if (PAIR) umma_commit_pair(bar_acc_full + 8 * acc); else umma_commit(bar_acc_full + 8 * acc);
+        }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
