@@ -309,7 +309,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       tma_load_2d(my_stage + b * kStagingBytes, &p.tmap_res[g], col0, row0, my_res_bar + 8 * b);
     };
 
-    if (EPI == kEpiBiasResidual && lane == 0 && worker < total_tiles) prefetch_residual(worker, col_group, 0);
+    // (residual epilogue, lane 0) This warp's chunks, in the order it works through them, use the two staging
+    // buffers alternately.  A buffer can take the residual of the chunk two places on as soon as the store of
+    // its present chunk has read it, so up to two requests are kept in flight: both chunks of a 128-wide tile
+    // are asked for before the tile's main loop ends (at the kernel's start for a CTA's first tile) instead of
+    // the second one only when the first is being worked on.
+    int req_tile = worker, req_chunk = col_group;   // the next chunk to ask for
+    int n_req = 0, n_done = 0;                      // chunks asked for / chunks whose store has been issued
+    auto refill = [&]() {
+      while (n_req < n_done + 2 && req_tile < total_tiles) {
+        prefetch_residual(req_tile, req_chunk, n_req & 1);
+        ++n_req;
+        req_chunk += COL_GROUPS;
+        if (req_chunk >= CHUNKS) { req_chunk = col_group; req_tile += n_workers; }
+      }
+    };
+    if (EPI == kEpiBiasResidual && lane == 0) refill();
     // a pair's accumulator is free again when the epilogue warps of both CTAs are done with it
     const uint32_t bar_acc_empty_count = (PAIR && rank != 0) ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;
 
@@ -337,16 +352,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
                                static_cast<uint32_t>(acc * BN + chunk * CHUNK_COLS);
         uint8_t* sbuf = my_stage_ptr + buf * kStagingBytes;
         if (EPI == kEpiBiasResidual) {
-          // prefetch the residual of the chunk after this one (next chunk of this tile, or the first
-          // chunk of this CTA's next tile) into the other buffer
-          if (lane == 0) {
-            int nt = tile, nc = chunk + COL_GROUPS;
-            if (nc >= CHUNKS) { nt = tile + n_workers; nc = col_group; }
-            if (nt < total_tiles) prefetch_residual(nt, nc, buf ^ 1);
-          }
-          __syncwarp();
           uint32_t v[32];
           tmem_ld_32x32(taddr, v);
+          // the other buffer is free once the store before this chunk has read it
+          if (lane == 0) refill();
+          __syncwarp();
           tmem_ld_wait();
           if (!__all_sync(0xffffffffu, mbar_wait(my_res_bar + 8 * buf, res_phase[buf], abort_flag))) {
             ok = false;
@@ -455,6 +465,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           tma_store_2d(&p.tmap_out[g], my_stage + buf * kStagingBytes, col, m0 + quarter * 32);
           tma_store_commit();
         }
+        ++n_done;
         if (NBUF == 2) buf ^= 1;
       }
       tc_fence_before();
@@ -462,11 +473,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       if (lane == 0) {
         if (PAIR && rank != 0) mbar_arrive_cluster(bar_acc_empty_count + 8 * acc);
         else mbar_arrive(bar_acc_empty + 8 * acc);
+        // the tile's last store frees its buffer for the next tile's residual while that tile's main loop runs
+        if (EPI == kEpiBiasResidual) refill();
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-    // shared memory must outlive the stores that still read it
-    if (lane == 0) tma_store_wait_read<0>();
+    // shared memory must outlive the stores that still read it, and (when the CTA is giving up) the residual
+    // copies that were asked for and never used: those get the same limit to land
+    if (lane == 0) {
+      tma_store_wait_read<0>();
+      for (int i = n_done; i < n_req; ++i) {
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(my_res_bar + 8 * (i & 1), res_phase[i & 1])) {
+          if (global_timer_ns() - t0 > kWaitLimitNs) break;
+        }
+      }
+    }
     __syncwarp();
   }
 
