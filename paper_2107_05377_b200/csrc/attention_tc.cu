@@ -5,12 +5,12 @@
 //
 // One CTA of 128 threads = one (layer of the wave, sequence, head); thread t owns query row t, which
 // is lane t of tensor memory.  Steps:
-//   1. one thread fetches the 128 x 64 Q, K and V tiles with three TMA loads (128-byte swizzle; rows
+//   1. an elected lane fetches the 128 x 64 Q, K and V tiles with three TMA loads (128-byte swizzle; rows
 //      past the end of the buffer arrive as zeros, rows past the sequence's length are another
 //      sequence's finite data or stale memory and are masked: V rows >= length are overwritten with
 //      zeros in shared memory, score columns >= length never enter the softmax)
 //   2. S = Q . K^T: four tcgen05.mma 128 x N x 16 (N = 64 when length <= 64, else 128) into tensor
-//      memory columns [0, N)
+//      memory columns [0, N), issued by the lane that saw the copies land while the others clear V
 //   3. every thread reads its row of S twice with tcgen05.ld (maximum; then exponentials and their
 //      fp32 sum), rounds the probabilities to bf16 and stores them K-major, 128-byte swizzled, over
 //      the Q and K tiles, which are no longer needed
@@ -60,6 +60,8 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
   const int b = blockIdx.y;
   const int g = blockIdx.z;
   const int H = p.heads * kHeadDim;
+  // warp 1 is converged here: one of its lanes issues the copies and the MMAs (warp 0 allocates tensor memory)
+  const bool leader = warp == 1 && elect_one();
 
   if (tid == 0) {
     mbar_init(bar_load, 1);
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
   bool ok = true;
   bool loads_in_flight = false;
   {
-    if (tid == 0) {
+    if (leader) {
       // a sequence of at most 64 tokens needs only the first 64 rows of each tile (the rest of the tiles
       // keeps whatever shared memory held: query rows and keys >= length never reach a result, and the V
       // rows >= length are overwritten with zeros below)
@@ -101,22 +103,12 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
       tma_load_2d(sK, map, H + head * kHeadDim, row0, bar_load);
       tma_load_2d(sV, map, 2 * H + head * kHeadDim, row0, bar_load);
     }
-    ok = __syncthreads_and(mbar_wait(bar_load, 0, abort_flag)) != 0;
-    loads_in_flight = !ok;
-  }
-
-  if (ok) {
-    // keys >= length take no part: their probabilities are exactly 0, and 0 * V must stay finite
-    if (tid >= len) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(smem + 2 * kTcTileBytes + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-    }
-    fence_async_shared();
-    __syncthreads();
-
-    const int key_tiles = len > 64 ? 2 : 1;   // 64 keys each
-    if (tid == 0) {
+    const bool landed = mbar_wait(bar_load, 0, abort_flag);
+    if (leader && landed) {
+      // S = Q K^T at once: the thread that saw the barrier complete sees the tiles (no MMA is issued if
+      // the copies never landed)
       tc_fence_after();
+      const int key_tiles = len > 64 ? 2 : 1;   // 64 keys each
       const uint64_t dq = smem_desc_sw128(sQ);
       const uint64_t dk = smem_desc_sw128(sK);
       const uint32_t idesc = umma_idesc_bf16(kTcRows, 64 * key_tiles);
@@ -124,8 +116,16 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
       for (int k = 0; k < kHeadDim / 16; ++k) umma_bf16(tmem_base, dq + 2 * k, dk + 2 * k, idesc, k > 0 ? 1u : 0u);
       umma_commit(bar_mma);
     }
-    ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag)) != 0;
+    // meanwhile: keys >= length take no part (their probabilities are exactly 0), and 0 * V must stay finite;
+    // the proxy fence after the probabilities are written covers these stores too
+    if (landed && tid >= len) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(smem + 2 * kTcTileBytes + tid * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+    }
+    ok = __syncthreads_and(landed) != 0;
+    loads_in_flight = !ok;
   }
+  if (ok) ok = __syncthreads_and(mbar_wait(bar_mma, 0, abort_flag)) != 0;
 
   if (ok) {
     tc_fence_after();
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(kTcThreads, 4) attention_tc_kernel(const __gri
     tc_fence_before();
     __syncthreads();
 
-    if (tid == 0) {
+    if (leader) {
       tc_fence_after();
       const uint32_t idesc = umma_idesc_bf16_b_mn(kTcRows, kHeadDim);
       for (int t = 0; t < key_tiles; ++t) {
