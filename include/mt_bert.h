@@ -257,6 +257,14 @@ int mt_plan_cache_size(const mt_model* m);
  * 64-column segments in the same order, every projection sums over K in one sequence).  Measured: faster than the
  * separate launches while the launch is a single round of tiles (one or two layers of the 32 x 128 batch), slower
  * beyond, where the separate LayerNorm hides the same latencies behind full occupancy.
+ * key "ffn_down_split" (0/1, default 1, any time): launches of at most 512 rows per layer (batch x seq up to
+ * 4 x 128, and the first-token rows of the last branch layers for batches up to 512) run the FFN-down projection
+ * as partial sums over four ranges of K - four times as many tiles, each a quarter as long - and the LayerNorm
+ * kernel after it adds the ranges in order, then the bias and the residual.  Such a launch has so few tiles that
+ * the chain of k-blocks one CTA walks is what it costs.  The sum over K is then taken range by range: results
+ * differ in the last bits from the unsplit projection, within every tolerance of the tests; the choice depends on
+ * the rows of one layer and on options only, never on the tasks asked for or on how many layers share a launch,
+ * so a merged model and its tasks run alone still agree bit for bit.  Not with "fp8_gemm".
  * key "overlap_cls" (0/1, default 1, any time): where a wave holds layers on all tokens and last branch
  * layers, the first-token attention of the latter runs on a stream the library creates for itself (in
  * mt_bind_memory), forked from the caller's stream after the wave's Q/K/V projection and joined before the next
@@ -326,6 +334,15 @@ int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d
                          const void* d_bias, const void* d_residual, void* d_y, int32_t M, int32_t N, int32_t K,
                          int32_t epilogue, uint32_t* d_status, void* stream);
 
+/* Partial sums of X[M,K] . W[N,K]^T with K split into k_splits equal ranges (a launch of few rows then has
+ * k_splits times as many tiles, each walking a k_splits-th of K): range s writes its fp32 sum, without bias, to rows
+ * [s * split_pitch, s * split_pitch + M) of d_part (fp32 [k_splits * split_pitch, N], device).  X, W bf16;
+ * (K / 64) % k_splits == 0; split_pitch >= M and a multiple of 128; N % 128 == 0.  This is how the FFN-down
+ * projection (Section 3: the second linear map of the feed-forward sub-layer) runs for launches of at most 512
+ * rows per layer (option "ffn_down_split"); mt_kernel_layernorm_partial puts the row together. */
+int mt_kernel_linear_partial(const void* d_x, const void* d_w, void* d_part, int32_t M, int32_t N, int32_t K,
+                             int32_t k_splits, int32_t split_pitch, uint32_t* d_status, void* stream);
+
 /* Y = LN(X[M,K] . W[N,K]^T + bias[N] + residual[M,N]) * gamma[N] + beta[N] in one launch: the residual
  * sub-layer followed by LayerNorm, as the encoder layer has it twice (after attention, after the FFN).
  * X, W, bias, gamma, beta bf16; residual fp32; Y is written twice, d_y bf16 [M,N] and d_y_f32 fp32 [M,N].
@@ -354,6 +371,13 @@ int mt_kernel_attention(const void* d_qkv, const int32_t* d_lengths, void* d_ctx
  * written as bf16 to d_y and, when d_y_f32 is not NULL, as fp32 too.  hidden in {768, 1024}. */
 int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32,
                         int32_t rows, int32_t hidden, float eps, void* stream);
+
+/* The same LayerNorm on x = residual + ((part_0 + part_1 + ... + part_{n_parts-1}) + bias), the ranges added in
+ * this order: the residual sub-layer after a projection whose K was split (mt_kernel_linear_partial).  d_part fp32
+ * [n_parts * part_pitch, hidden] (range s at row s * part_pitch; n_parts <= 4), d_residual fp32 [rows, hidden], bias bf16. */
+int mt_kernel_layernorm_partial(const float* d_part, int32_t n_parts, int32_t part_pitch, const float* d_residual,
+                                const void* d_bias, const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32,
+                                int32_t rows, int32_t hidden, float eps, void* stream);
 
 /* h0[B*S, hidden] = LayerNorm(word[tok] + pos[position] + type[seg]), bf16 (and fp32 if d_h0_f32 != NULL). */
 int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,

@@ -66,6 +66,8 @@ SIGNATURES = {
     "mt_kernel_linear_layernorm_tiles": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, C.c_float, _I32, _P, _P]),
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
+    "mt_kernel_linear_partial": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_kernel_layernorm_partial": (C.c_int, [_P, _I32, _I32, _P, _P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
                                   _P]),
     "mt_kernel_pooler_head": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, _I32, _P]),
@@ -159,6 +161,23 @@ def mt_kernel_layernorm(x, gamma, beta, y, eps: float, y_f32=None, stream=None) 
     rows, hidden = x.shape
     _check(lib().mt_kernel_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), _ptr(y_f32), rows, hidden, eps,
                                      _stream(stream)), "mt_kernel_layernorm")
+
+
+def mt_kernel_linear_partial(x, w, part, k_splits: int, split_pitch: int, status=None, stream=None) -> None:
+    """part[s * split_pitch + i, :] = x[i, range s of K] . w[:, range s of K]^T (fp32, no bias)."""
+    M, K = x.shape
+    N = w.shape[0]
+    _check(lib().mt_kernel_linear_partial(_ptr(x), _ptr(w), _ptr(part), M, N, K, k_splits, split_pitch, _ptr(status),
+                                          _stream(stream)), "mt_kernel_linear_partial")
+
+
+def mt_kernel_layernorm_partial(part, n_parts: int, part_pitch: int, residual, bias, gamma, beta, y, eps: float,
+                                y_f32=None, stream=None) -> None:
+    """y = LayerNorm(residual + ((part_0 + part_1 + ...) + bias))."""
+    rows, hidden = residual.shape
+    _check(lib().mt_kernel_layernorm_partial(_ptr(part), n_parts, part_pitch, _ptr(residual), _ptr(bias), _ptr(gamma),
+                                             _ptr(beta), _ptr(y), _ptr(y_f32), rows, hidden, eps, _stream(stream)),
+           "mt_kernel_layernorm_partial")
 
 
 def mt_kernel_embed(token_ids, segment_ids, lengths, word, pos, type_, gamma, beta, h0, eps: float, h0_f32=None,

@@ -106,7 +106,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
   const int n_tiles_n = p.N / BN;
-  const int k_blocks = p.K / KB_ELEMS;
+  const int k_splits = p.k_splits > 1 ? p.k_splits : 1;   // ranges of K (> 1 only with the partial-sum epilogue)
+  const int k_blocks = p.K / KB_ELEMS / k_splits;         // k-blocks of one tile
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -133,9 +134,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   const uint32_t tmem_base = *tmem_slot;
   // where the "stage full" barriers are counted: in rank 0 of a pair
   const uint32_t bar_full_count = PAIR ? map_to_cta(bar_full, 0) : bar_full;
-  // Tiles are numbered m-tile outermost: tile = (m_tile * n_groups + g) * n_tiles_n + n_tile, so the
-  // group and the column block of a tile do not depend on the (device-side) number of rows.
-  const int tiles_per_m = p.n_groups * n_tiles_n;
+  // Tiles are numbered m-tile outermost: tile = ((m_tile * n_groups + g) * n_tiles_n + n_tile) * k_splits + range,
+  // so the group, the column block and the K range of a tile do not depend on the (device-side) number of rows.
+  const int tiles_per_m = p.n_groups * n_tiles_n * k_splits;
   // Everything above touched no global data.  The weights do not depend on the previous kernel
   // either: the producer thread starts the W tiles of this CTA's first tile before it waits for
   // that kernel, so their trip from HBM overlaps its tail.  From the wait on, the previous kernel
@@ -144,7 +145,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
   bool producer_leader = false;
   if (warp == 0) {
     producer_leader = elect_one();   // the warp stays converged; this lane issues the copies
-    const int rem = worker % tiles_per_m;
+    const int rem_s = worker % tiles_per_m;
+    const int kb0 = (rem_s % k_splits) * k_blocks;   // first k-block of the tile's range of K
+    const int rem = rem_s / k_splits;
     const int g = rem / n_tiles_n;
     const int n0 = (rem - g * n_tiles_n) * BN + static_cast<int>(rank) * (PAIR ? BN / 2 : 0);
     prefetched = k_blocks < STAGES ? k_blocks : STAGES;
@@ -155,10 +158,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
         if (PAIR) {
           // rank 0 announces the bytes of both CTAs' W parts on its barrier; either CTA's copy may land first
           if (rank == 0) mbar_add_tx(bar_full + 8 * s, 2 * B_BYTES);
-          tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full_count + 8 * s);
+          tma_load_2d_pair(sB + s * B_BYTES, &p.tmap_w[g], (kb0 + s) * KB_ELEMS, n0, bar_full_count + 8 * s);
         } else {
           mbar_add_tx(bar_full + 8 * s, B_BYTES);
-          tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], s * KB_ELEMS, n0, bar_full + 8 * s);
+          tma_load_2d(sB + s * B_BYTES, &p.tmap_w[g], (kb0 + s) * KB_ELEMS, n0, bar_full + 8 * s);
         }
       }
     }
@@ -195,7 +198,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
       }
       for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
         const int m0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM;
-        const int rem = tile % tiles_per_m;
+        const int rem_s = tile % tiles_per_m;
+        const int kb0 = (rem_s % k_splits) * k_blocks;
+        const int rem = rem_s / k_splits;
         const int g = rem / n_tiles_n;
         const int n0 = (rem - g * n_tiles_n) * BN + static_cast<int>(rank) * (PAIR ? BN / 2 : 0);
         for (int kb = 0; kb < k_blocks; ++kb) {
@@ -208,14 +213,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
           } else if (PAIR) {
             if (rank == 0)
               mbar_expect_tx(bar_full + 8 * stage, 2 * A_BYTES + (w_on_its_way ? 0 : 2 * B_BYTES));
-            tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], kb * KB_ELEMS, m0, bar_full_count + 8 * stage);
+            tma_load_2d_pair(sA + stage * A_BYTES, &p.tmap_x[g], (kb0 + kb) * KB_ELEMS, m0, bar_full_count + 8 * stage);
             if (!w_on_its_way)
-              tma_load_2d_pair(sB + stage * B_BYTES, &p.tmap_w[g], kb * KB_ELEMS, n0, bar_full_count + 8 * stage);
+              tma_load_2d_pair(sB + stage * B_BYTES, &p.tmap_w[g], (kb0 + kb) * KB_ELEMS, n0, bar_full_count + 8 * stage);
           } else {
             mbar_expect_tx(bar_full + 8 * stage, A_BYTES + (w_on_its_way ? 0 : B_BYTES));
-            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], kb * KB_ELEMS, m0, bar_full + 8 * stage);
+            tma_load_2d(sA + stage * A_BYTES, &p.tmap_x[g], (kb0 + kb) * KB_ELEMS, m0, bar_full + 8 * stage);
             if (!w_on_its_way)
-              tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], kb * KB_ELEMS, n0, bar_full + 8 * stage);
+              tma_load_2d(sB + stage * B_BYTES, &p.tmap_w[g], (kb0 + kb) * KB_ELEMS, n0, bar_full + 8 * stage);
           }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -286,7 +291,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
     const int quarter = warp & 3;                       // TMEM lanes this warp may read
     const int col_group = e >> 2;                       // which share of the column chunks
     constexpr int COL_GROUPS = kNumEpilogueWarps / 4;
-    constexpr int CHUNK_COLS = (EPI == kEpiBiasResidual || EPI == kEpiBiasTanhF32) ? 32 : 64;
+    constexpr int CHUNK_COLS = (EPI == kEpiBiasResidual || EPI == kEpiBiasTanhF32 || EPI == kEpiPartialF32) ? 32 : 64;
     constexpr int CHUNKS = BN / CHUNK_COLS;
     const uint32_t my_stage = sStage + static_cast<uint32_t>(e * NBUF * kStagingBytes);
     const uint32_t my_res_bar = bar_res + 16 * e;       // two barriers, one per staging buffer
@@ -299,7 +304,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
     // (residual epilogue) asks for the residual chunk `chunk` of tile `tile` into staging buffer b
     auto prefetch_residual = [&](int tile, int chunk, int b) {
-      const int rem = tile % tiles_per_m;
+      const int rem = (tile % tiles_per_m) / k_splits;
       const int g = rem / n_tiles_n;
       const int row0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM + quarter * 32;
       const int col0 = (rem - g * n_tiles_n) * BN + chunk * CHUNK_COLS;
@@ -330,9 +335,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
 
     for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
       const int m0 = (tile / tiles_per_m) * TILE_M + static_cast<int>(rank) * kGemmBlockM;
-      const int rem = tile % tiles_per_m;
+      const int rem_s = tile % tiles_per_m;
+      const int rem = rem_s / k_splits;
       const int g = rem / n_tiles_n;
       const int n0 = (rem - g * n_tiles_n) * BN;
+      // (partial sums) the tile's range of K writes its own rows of the output
+      const int out_row0 = m0 + quarter * 32 + (EPI == kEpiPartialF32 ? (rem_s % k_splits) * p.split_pitch : 0);
       // warp-uniform decisions: the TMEM loads below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag))) break;
       tc_fence_after();
@@ -392,6 +400,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
             *s0 = r0;
             *s1 = r1;
           }
+        } else if (EPI == kEpiPartialF32) {
+          // the store that last read this staging buffer must be done with it
+          if (lane == 0) {
+            if (NBUF == 2) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
+          }
+          __syncwarp();
+          uint32_t v[32];
+          tmem_ld_32x32(taddr, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            *reinterpret_cast<uint4*>(sbuf + staging_off(lane, q)) = make_uint4(v[q * 4 + 0], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
         } else if (EPI == kEpiBiasTanhF32) {
           // the store that last read this staging buffer must be done with it
           if (lane == 0) {
@@ -462,7 +482,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_tcgen05(const __gri
         fence_async_shared();
         __syncwarp();
         if (lane == 0 && rows_in_range) {
-          tma_store_2d(&p.tmap_out[g], my_stage + buf * kStagingBytes, col, m0 + quarter * 32);
+          tma_store_2d(&p.tmap_out[g], my_stage + buf * kStagingBytes, col, out_row0);
           tma_store_commit();
         }
         ++n_done;
@@ -516,7 +536,7 @@ cudaError_t launch_one(const GemmParams& p, int sm_count, cudaStream_t stream) {
   });
   if (err != cudaSuccess) return err;
   constexpr int tile_m = PAIR ? 2 * kGemmBlockM : kGemmBlockM;
-  const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN) * p.n_groups;
+  const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN) * p.n_groups * (p.k_splits > 1 ? p.k_splits : 1);
   const int workers_max = PAIR ? sm_count / 2 : sm_count;
   const int workers = tiles < workers_max ? tiles : workers_max;
   if (workers <= 0) return cudaSuccess;
@@ -534,6 +554,9 @@ cudaError_t launch_bn(const GemmParams& p, int epilogue, int sm_count, cudaStrea
       return cudaErrorInvalidValue;  // single CTAs: 256-wide stages and two fp32 staging buffers do not fit
     case kEpiBiasTanhF32:   // the pooler: a few rows, single CTAs on 128-wide tiles only
       if constexpr (BN == 128 && !PAIR) return launch_one<BN, kEpiBiasTanhF32, PAIR>(p, sm_count, stream);
+      return cudaErrorInvalidValue;
+    case kEpiPartialF32:    // partial sums of a split K: launches of few rows, single CTAs on 64- or 128-wide tiles
+      if constexpr ((BN == 128 || BN == 64) && !PAIR) return launch_one<BN, kEpiPartialF32, PAIR>(p, sm_count, stream);
       return cudaErrorInvalidValue;
     default: return cudaErrorInvalidValue;
   }
@@ -556,6 +579,12 @@ cudaError_t launch_any(const GemmParams& p, int epilogue, int sm_count, cudaStre
 
 int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int sm_count) {
   if (epilogue == kEpiBiasTanhF32) return 128;
+  if (epilogue == kEpiPartialF32) {
+    // (`groups` counts the ranges of K too) 64-wide tiles while they all run at once, else 128-wide (measured at
+    // N = 768, K = 3072 in four ranges: 128 rows 5.4 against 6.0 us, 512 rows 8.8 against 6.7 us)
+    const int64_t tiles64 = ((rows + kGemmBlockM - 1) / kGemmBlockM) * (N / 64) * groups;
+    return (N % 128 != 0 || tiles64 <= sm_count) ? 64 : 128;
+  }
   // (64: only ever the cheapest where a launch has so few rows that even 128-wide tiles leave most SMs
   // without work - the first-token tails - and each CTA would stream a long K by itself)
   const int candidates[4] = {256, 192, 128, 64};
@@ -581,11 +610,19 @@ int gemm_block_n(int N, int epilogue, int64_t rows, int groups, bool pair, int s
   }
   return best;
 }
-int gemm_out_box_cols(int epilogue) { return (epilogue == kEpiBiasResidual || epilogue == kEpiBiasTanhF32) ? 32 : 64; }
+int gemm_out_box_cols(int epilogue) {
+  return (epilogue == kEpiBiasResidual || epilogue == kEpiBiasTanhF32 || epilogue == kEpiPartialF32) ? 32 : 64;
+}
 
 cudaError_t launch_gemm(const GemmParams& p, int epilogue, int sm_count, cudaStream_t stream) {
   if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.K % kGemmBlockK != 0 || p.block_n < 1 || p.N % p.block_n != 0 ||
       p.M < 1)
+    return cudaErrorInvalidValue;
+  // a split K only with the partial-sum epilogue (single CTAs, bf16): equal ranges of whole k-blocks, and the
+  // ranges' outputs a whole number of row blocks apart so that no store box reaches into the next range's rows
+  if (p.k_splits > 1 &&
+      (epilogue != kEpiPartialF32 || p.fp8 || p.pair || (p.K / kGemmBlockK) % p.k_splits != 0 ||
+       p.split_pitch < p.M || p.split_pitch % kGemmBlockM != 0))
     return cudaErrorInvalidValue;
   if (p.fp8) {
     if (p.pair || p.K % (2 * kGemmBlockK) != 0) return cudaErrorInvalidValue;

@@ -34,6 +34,12 @@ constexpr uint32_t kBlobMagic = 0x4D544257u;
 constexpr uint32_t kBlobVersion = 1u;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;
+// rows between the partial sums of consecutive ranges of K: whole 128-row blocks
+constexpr size_t split_pitch(size_t rows) { return (rows + 127) / 128 * 128; }
+// The FFN-down projection of a launch of few rows is split into this many ranges of K (option "ffn_down_split").
+constexpr int32_t kDownSplits = 4;
+// "Few rows": at most this many per layer (batch 4 x 128 tokens; the first-token tails of batches up to 512).
+constexpr int32_t kSplitRowsMax = 512;
 
 inline size_t pad256(size_t n) { return (n + kAlign - 1) / kAlign * kAlign; }
 
@@ -84,6 +90,9 @@ struct LayerTail {
   bool ln_fused = false;
   bool ln_wide = false;      // ... on 128 x 256 accumulator tiles (clusters of N / 256): launches with many row blocks
   bool down_fused = false;   // the FFN-down projection too (not with 8-bit operands: that GEMM is the plain kernel)
+  // launches of few rows: the FFN-down projection as partial sums over `down_splits` ranges of K, put together
+  // (ranges in order, bias, residual) by the LayerNorm kernel after it
+  int32_t down_splits = 1;
   GemmLnParams attn_out_ln, ffn_down_ln;
   // 8-bit operands: the inputs of the FFN-up and FFN-down projections are quantised row by row first
   bool fp8 = false;
@@ -186,7 +195,7 @@ cudaError_t set_gemm_group(GemmParams* g, int i, int epilogue, const void* x, co
                            const float* residual, void* y) {
   const int M = g->M, N = g->N, K = g->K;
   const bool res = epilogue == kEpiBiasResidual;
-  const bool f32_out = res || epilogue == kEpiBiasTanhF32;
+  const bool f32_out = res || epilogue == kEpiBiasTanhF32 || epilogue == kEpiPartialF32;
   cudaError_t e;
   if (g->fp8 != 0) {
     if ((e = make_tmap_u8(&g->tmap_x[i], x, M, K, kGemmBlockM)) != cudaSuccess) return e;
@@ -227,6 +236,7 @@ struct mt_model {
   int32_t fused_ln;  // each residual GEMM and the LayerNorm after it as one cluster launch: 0 never, 1 always on
                      // 128-column tiles, 3 always on 256-column tiles, 2 by the launch (fused_ln_kind)
   int32_t fused_ln_max_groups;
+  int32_t ffn_down_split;   // 0: never; 1: launches of few rows split the K of the FFN-down projection (default)
   int32_t fused_ln_max_rows;
   // The first-token attention of the branches that end in a wave depends on the wave's QKV projection only
   // and feeds nothing before the first-token tails, so it runs on a stream of the library's own beside the
@@ -245,7 +255,7 @@ struct mt_model {
   int sm_device, sm_limit;
 
   // workspace layout (byte offsets)
-  size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_trunk[2], ws_task0,
+  size_t ws_status, ws_rows_valid, ws_row_start, ws_tok, ws_seg, ws_len, ws_logits, ws_pooled, ws_partial, ws_trunk[2], ws_task0,
       ws_slot0, ws_cls0, ws_dump0;
   size_t slot_q_off, cls_q_off;   // 8-bit scratch inside a slot / inside a task's first-token scratch
   size_t cls_bytes, cls_h_bytes, cls_h32_bytes;  // per-task first-token scratch and its [B,H] bf16 / fp32 pieces
@@ -356,6 +366,8 @@ void layout_workspace(mt_model* m) {
   m->ws_logits = take(static_cast<size_t>(m->max_batch) * m->c_total * 4);
   // tanh pooler outputs of the tasks of one head launch: fp32 [kMaxGroups][max_batch][H]
   m->ws_pooled = take(static_cast<size_t>(kMaxGroups) * m->max_batch * H * sizeof(float));
+  // partial sums of the FFN-down projection in launches of few rows: fp32 [group][range of K][row pitch][H]
+  m->ws_partial = take(static_cast<size_t>(kMaxGroups) * kDownSplits * split_pitch(std::min<size_t>(M, kSplitRowsMax)) * H * sizeof(float));
   m->ws_trunk[0] = take(m->state_bytes);
   m->ws_trunk[1] = take(m->state_bytes);
   m->ws_task0 = off;
@@ -528,11 +540,25 @@ int fused_ln_kind(const mt_model* m, int32_t groups, int64_t rows) {
   return groups == 1 ? 1 : 2;
 }
 bool use_fused_ln(const mt_model* m, int32_t groups, int64_t rows) { return fused_ln_kind(m, groups, rows) != 0; }
+// Ranges the K of the FFN-down projection is split into.  A launch of few rows has few tiles, and each walks
+// K = F by itself (48 k-blocks one after the other for BERT-base) while most SMs have none: four ranges, each a
+// tile of its own, shorten that chain fourfold, and the LayerNorm kernel that follows adds the four partial
+// sums in a fixed order.  The sum over K is then taken range by range, so the bits differ from the unsplit
+// projection; the choice depends only on the rows of one layer (batch x seq, or the batch for a first-token
+// tail) and on options, which are the same for a merged model and for its tasks run alone, never on how many
+// layers share the launch or on which tasks are asked for.
+// (Nor on option "fused_ln", whose settings all give the same bits: where the projection is split it keeps its
+// LayerNorm as a launch of its own, and only the attention-output projection is fused when that option says so.)
+int32_t down_split_count(const mt_model* m, int64_t rows) {
+  if (m->ffn_down_split == 0 || m->fp8 || rows > kSplitRowsMax) return 1;
+  return (m->trunk.ffn / kGemmBlockK) % kDownSplits == 0 ? kDownSplits : 1;
+}
 // Launches of steps 3-7 for `groups` layers.
 int32_t tail_launches(const mt_model* m, int32_t groups, int64_t rows) {
   const bool fused = use_fused_ln(m, groups, rows);
-  // 8-bit operands: two quantisations, and the FFN-down projection keeps its LayerNorm as a launch of its own
-  return (fused ? 3 : 5) + (m->fp8 ? 2 + (fused ? 1 : 0) : 0);
+  // 8-bit operands: two quantisations, and the FFN-down projection keeps its LayerNorm as a launch of its own;
+  // so does a projection whose K is split
+  return (fused ? 3 : 5) + (m->fp8 ? 2 + (fused ? 1 : 0) : 0) + (fused && down_split_count(m, rows) > 1 ? 1 : 0);
 }
 
 void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_valid, int32_t groups) {
@@ -549,7 +575,16 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   };
   init_gemm(&t->attn_out, H, H, kEpiBiasResidual);
   init_gemm(&t->ffn_up, F, H, kEpiBiasGelu);
-  init_gemm(&t->ffn_down, H, F, kEpiBiasResidual);
+  t->down_splits = down_split_count(m, rows);
+  if (t->down_splits > 1) {
+    init_gemm(&t->ffn_down, H, F, kEpiPartialF32);
+    t->ffn_down.k_splits = t->down_splits;
+    t->ffn_down.split_pitch = static_cast<int32_t>(split_pitch(rows));
+    t->ffn_down.block_n = gemm_block_n(H, kEpiPartialF32, rows, groups * t->down_splits, false, m->sm_count);
+    t->ffn_down.pair = 0;
+  } else {
+    init_gemm(&t->ffn_down, H, F, kEpiBiasResidual);
+  }
   t->fp8 = m->fp8;
   if (m->fp8) {
     // E4M3 operands: single CTAs, 256-wide tiles (128 with the residual epilogue)
@@ -573,7 +608,7 @@ void init_tail(const mt_model* m, LayerTail* t, int32_t rows, bool all_rows_vali
   t->count = 0;
   t->ln_fused = use_fused_ln(m, groups, rows);
   t->ln_wide = fused_ln_kind(m, groups, rows) == 2;
-  t->down_fused = t->ln_fused && !m->fp8;
+  t->down_fused = t->ln_fused && !m->fp8 && t->down_splits == 1;
   if (t->ln_fused) {
     auto init_ln = [&](GemmLnParams* g, int32_t K) {
       memset(g, 0, sizeof(*g));
@@ -617,9 +652,23 @@ cudaError_t add_to_tail(const mt_model* m, LayerTail* t, const LayerOffsets* lo,
     if ((e = set_gemm_group(&t->ffn_up, i, kEpiBiasGelu, h1, w_ptr(m, lo->w1), w_ptr(m, lo->b1), nullptr, f)) !=
         cudaSuccess)
       return e;
-    if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) !=
-        cudaSuccess)
+    if (t->down_splits > 1) {
+      // partial sums: range s of this group writes rows [s * pitch, s * pitch + rows) of the group's piece of the
+      // partial-sum scratch; the LayerNorm kernel adds the ranges, the bias and the residual
+      const size_t pitch = static_cast<size_t>(t->ffn_down.split_pitch);
+      float* part = reinterpret_cast<float*>(m->d_workspace + m->ws_partial) +
+                    static_cast<size_t>(i) * t->down_splits * pitch * m->trunk.hidden;
+      if ((e = set_gemm_group(&t->ffn_down, i, kEpiPartialF32, f, w_ptr(m, lo->w2), nullptr, nullptr, part)) != cudaSuccess)
+        return e;
+      if ((e = make_tmap(&t->ffn_down.tmap_out[i], part, static_cast<int>(t->down_splits * pitch), t->ffn_down.N, 32, 32,
+                         true)) != cudaSuccess)
+        return e;
+      t->ln2.part[i] = part; t->ln2.residual[i] = h1_32; t->ln2.bias[i] = w_ptr(m, lo->b2);
+      t->ln2.n_parts = t->down_splits; t->ln2.part_pitch = static_cast<int32_t>(pitch);
+    } else if ((e = set_gemm_group(&t->ffn_down, i, kEpiBiasResidual, f, w_ptr(m, lo->w2), w_ptr(m, lo->b2), h1_32, u)) !=
+               cudaSuccess) {
       return e;
+    }
   }
   t->ln2.x[i] = u; t->ln2.gamma[i] = w_ptr(m, lo->ln2_g); t->ln2.beta[i] = w_ptr(m, lo->ln2_b);
   t->ln2.y[i] = out; t->ln2.y32[i] = out32;
@@ -955,6 +1004,7 @@ int mt_create(const mt_trunk_config* trunk, const mt_task_config* tasks, int32_t
   m->ev_fork = m->ev_join = nullptr;
   m->fused_ln = 2;
   m->fused_ln_max_groups = 2;
+  m->ffn_down_split = 1;
   m->fused_ln_max_rows = 0;
   m->last_lengths = nullptr;
   m->d_weights = m->d_workspace = nullptr;
@@ -1059,6 +1109,12 @@ int mt_set_option(mt_model* m, const char* key, int64_t value) {
   if (strcmp(key, "fused_ln_max_rows") == 0) {
     if (value < 0) return fail(m, MT_ERR_INVALID_ARG, "fused_ln_max_rows must be >= 0");
     m->fused_ln_max_rows = static_cast<int32_t>(value);
+    m->plans.clear();
+    return MT_OK;
+  }
+  if (strcmp(key, "ffn_down_split") == 0) {
+    if (value != 0 && value != 1) return fail(m, MT_ERR_INVALID_ARG, "ffn_down_split must be 0 or 1");
+    m->ffn_down_split = static_cast<int32_t>(value);
     m->plans.clear();
     return MT_OK;
   }
@@ -1387,7 +1443,8 @@ int mt_forward_tokens(mt_model* m, const int32_t* d_token_ids, const int32_t* d_
                                               : launch_gemm_ln(t_->ffn_down_ln, stream),                              \
                "FFN down GEMM + LayerNorm");                                                                           \
     } else {                                                                                                           \
-      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t_->ffn_down, kEpiBiasResidual, m->sm_count, stream), "FFN down GEMM");  \
+      MT_TIMED(MT_CLASS_FFN_DOWN, launch_gemm(t_->ffn_down, t_->down_splits > 1 ? kEpiPartialF32 : kEpiBiasResidual,   \
+                                              m->sm_count, stream), "FFN down GEMM");                                  \
       MT_TIMED(MT_CLASS_LN2, launch_layernorm(t_->ln2, stream), "LayerNorm 2");                                        \
     }                                                                                                                  \
   } while (0)
@@ -1589,6 +1646,27 @@ int mt_kernel_linear(const void* d_x, const void* d_w, const void* d_bias, const
   return launch_gemm(p, epilogue, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
+int mt_kernel_linear_partial(const void* d_x, const void* d_w, void* d_part, int32_t M, int32_t N, int32_t K,
+                             int32_t k_splits, int32_t split_pitch, uint32_t* d_status, void* stream) {
+  if (d_x == nullptr || d_w == nullptr || d_part == nullptr || M < 1 || N < 128 || N % 128 != 0 || K < 64 ||
+      K % 64 != 0 || k_splits < 1 || (K / 64) % k_splits != 0 || split_pitch < M || split_pitch % 128 != 0)
+    return MT_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MT_ERR_CUDA;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_groups = 1; p.M = M; p.N = N; p.K = K; p.status = d_status;
+  p.k_splits = k_splits; p.split_pitch = split_pitch;
+  p.block_n = gemm_block_n(N, kEpiPartialF32, M, k_splits, false, sms);
+  if (g_force_block_n == 64 || g_force_block_n == 128) p.block_n = g_force_block_n;
+  if (set_gemm_group(&p, 0, kEpiPartialF32, d_x, d_w, nullptr, nullptr, d_part) != cudaSuccess) return MT_ERR_CUDA;
+  if (make_tmap(&p.tmap_out[0], d_part, static_cast<int64_t>(k_splits) * split_pitch, N, 32, 32, true) != cudaSuccess)
+    return MT_ERR_CUDA;
+  return launch_gemm(p, kEpiPartialF32, sms, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
 int mt_kernel_quantize_rows(const void* d_x, void* d_q, float* d_scale, int32_t rows, int32_t cols, void* stream) {
   if (d_x == nullptr || d_q == nullptr || d_scale == nullptr || rows < 1 || cols < 256 || cols % 256 != 0)
     return MT_ERR_INVALID_ARG;
@@ -1689,6 +1767,23 @@ int mt_kernel_layernorm(const void* d_x, const void* d_gamma, const void* d_beta
   p.x[0] = static_cast<const float*>(d_x); p.gamma[0] = static_cast<const bf16*>(d_gamma);
   p.beta[0] = static_cast<const bf16*>(d_beta); p.y[0] = static_cast<bf16*>(d_y);
   p.y32[0] = static_cast<float*>(d_y_f32);
+  p.n_groups = 1; p.rows = rows; p.hidden = hidden; p.eps = eps;
+  return launch_layernorm(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
+int mt_kernel_layernorm_partial(const float* d_part, int32_t n_parts, int32_t part_pitch, const float* d_residual,
+                                const void* d_bias, const void* d_gamma, const void* d_beta, void* d_y, void* d_y_f32,
+                                int32_t rows, int32_t hidden, float eps, void* stream) {
+  if (d_part == nullptr || d_residual == nullptr || d_bias == nullptr || d_gamma == nullptr || d_beta == nullptr ||
+      d_y == nullptr || rows < 1 || n_parts < 1 || n_parts > 4 || part_pitch < rows)
+    return MT_ERR_INVALID_ARG;
+  if (hidden != 768 && hidden != 1024) return MT_ERR_UNSUPPORTED;
+  LayerNormParams p;
+  memset(&p, 0, sizeof(p));
+  p.part[0] = d_part; p.residual[0] = d_residual; p.bias[0] = static_cast<const bf16*>(d_bias);
+  p.n_parts = n_parts; p.part_pitch = part_pitch;
+  p.gamma[0] = static_cast<const bf16*>(d_gamma); p.beta[0] = static_cast<const bf16*>(d_beta);
+  p.y[0] = static_cast<bf16*>(d_y); p.y32[0] = static_cast<float*>(d_y_f32);
   p.n_groups = 1; p.rows = rows; p.hidden = hidden; p.eps = eps;
   return launch_layernorm(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }

@@ -87,12 +87,18 @@ cudaError_t launch_kernel(void (*kernel)(Param), dim3 grid, dim3 block, size_t s
 }
 #endif
 
-enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2, kEpiBiasTanhF32 = 3 };
+enum GemmEpilogue { kEpiBias = 0, kEpiBiasGelu = 1, kEpiBiasResidual = 2, kEpiBiasTanhF32 = 3, kEpiPartialF32 = 4 };
 
 // One problem of a grouped GEMM: Y_g[M,N] = epi(X_g[M,K] . W_g[N,K]^T + bias_g (+ residual_g)).
 // All groups of a launch share M, N, K and the epilogue.  kEpiBias and kEpiBiasGelu write bf16;
 // kEpiBiasResidual adds an fp32 residual and writes fp32 (the pre-LayerNorm sum is never rounded);
 // kEpiBiasTanhF32 writes tanh(.) in fp32 (the pooler; single CTAs on 128-wide tiles only).
+// kEpiPartialF32 writes the bare fp32 accumulator (no bias): the launch may then split K into k_splits equal
+// ranges, one tile per (row block, group, column block, range); range s of group g writes rows
+// [s * split_pitch, s * split_pitch + M) of that group's output, and whoever reads the partial sums adds them
+// in the order s = 0, 1, ... (the LayerNorm kernel does, with the bias and the residual).  For launches of so
+// few rows that most SMs would have no tile while each tile walks a long K by itself (64- and 128-wide
+// tiles, single CTAs, bf16 operands only).
 // The output and the residual are reached through the tensor maps of GemmParams.
 struct GemmGroup {
   const bf16* bias;
@@ -111,6 +117,8 @@ struct alignas(64) GemmParams {
   const int32_t* m_valid;  // device scalar: rows actually in use (<= M); null = all M rows
   int32_t pair;            // 1: run as pairs of CTAs on 256-row tiles (the W maps then fetch half a tile's rows)
   int32_t block_n;         // tile width along N: 128, 192 or 256 (gemm_block_n); N % block_n == 0
+  int32_t k_splits;        // ranges K is split into (kEpiPartialF32 only; otherwise 1): (K / 64) % k_splits == 0
+  int32_t split_pitch;     // rows between the outputs of consecutive ranges (a multiple of 128, >= M)
   int32_t fp8;             // 1: X and W are E4M3 bytes (maps of uint8, boxes of 128 bytes of K) with row scales;
                            // single CTAs, block_n 256 (128 for the residual epilogue), K % 128 == 0
   uint32_t* status;        // sticky device status word (may be null)
@@ -164,8 +172,15 @@ cudaError_t launch_cls_attention(const ClsAttnParams& p, cudaStream_t stream);
 
 // y = LN(x): x fp32; y is written as bf16 (the next GEMM's operand) and, if y32 is not null, also
 // as fp32 (the residual of the next sub-layer, so the residual stream is never rounded to bf16).
+// y = LayerNorm(x) row by row.  With n_parts > 0 the row is first put together from the partial sums of a GEMM
+// whose K was split (kEpiPartialF32): x = residual + ((part_0 + part_1 + ... in this order) + bias), the
+// arithmetic of the residual epilogue with the sum over K taken range by range; `x` is then not read.
 struct LayerNormParams {
   const float* x[kMaxGroups];
+  const float* part[kMaxGroups];      // [n_parts][part_pitch rows][hidden] fp32
+  const float* residual[kMaxGroups];  // [rows][hidden] fp32
+  const bf16* bias[kMaxGroups];       // [hidden]
+  int32_t n_parts, part_pitch;
   const bf16* gamma[kMaxGroups];
   const bf16* beta[kMaxGroups];
   bf16* y[kMaxGroups];

@@ -10,8 +10,11 @@ namespace mt {
 namespace {
 
 constexpr int kRowThreads = 256;  // 8 rows per CTA
+constexpr int kMaxParts = 4;       // ranges of K a row can be put together from (LayerNormParams::n_parts)
 
-template <int V>
+// PARTS: the row is put together from the partial sums of a split projection (LayerNormParams::n_parts > 0); a
+// separate instantiation, so that the plain kernel keeps its registers and occupancy.
+template <int V, bool PARTS>
 __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormParams p) {
   constexpr int H = V * 256;
   const int lane = threadIdx.x & 31;
@@ -23,14 +26,56 @@ __global__ void __launch_bounds__(kRowThreads) layernorm_kernel(const LayerNormP
   grid_dependency_wait();
   grid_launch_dependents();
   if (row >= rows_in_use) return;
-  const float* xin = p.x[g] + static_cast<size_t>(row) * H;
   float x[V][8];
+  if (PARTS) {
+    // the row from the partial sums of a GEMM whose K was split: the ranges in order, then the bias, then
+    // the residual - residual + ((part_0 + part_1 + ...) + bias)
+    const float* part = p.part[g] + static_cast<size_t>(row) * H;
+    const float* res = p.residual[g] + static_cast<size_t>(row) * H;
+    const size_t pitch = static_cast<size_t>(p.part_pitch) * H;
+    const int n_parts = p.n_parts;   // at most kMaxParts (checked by the launcher)
+    // every load of the row is issued before the first addition: one round trip to L2, not one per range
+    float4 pa[V][kMaxParts], pb[V][kMaxParts], ra[V], rb[V];
+    uint4 bias8[V];
 #pragma unroll
-  for (int v = 0; v < V; ++v) {
-    const float4 a = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8);
-    const float4 b = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8 + 4);
-    x[v][0] = a.x; x[v][1] = a.y; x[v][2] = a.z; x[v][3] = a.w;
-    x[v][4] = b.x; x[v][5] = b.y; x[v][6] = b.z; x[v][7] = b.w;
+    for (int v = 0; v < V; ++v) {
+      const int col = (v * 32 + lane) * 8;
+#pragma unroll
+      for (int s = 0; s < kMaxParts; ++s) {
+        if (s < n_parts) {
+          pa[v][s] = *reinterpret_cast<const float4*>(part + s * pitch + col);
+          pb[v][s] = *reinterpret_cast<const float4*>(part + s * pitch + col + 4);
+        }
+      }
+      ra[v] = *reinterpret_cast<const float4*>(res + col);
+      rb[v] = *reinterpret_cast<const float4*>(res + col + 4);
+      bias8[v] = __ldg(reinterpret_cast<const uint4*>(p.bias[g] + col));
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      float acc[8] = {pa[v][0].x, pa[v][0].y, pa[v][0].z, pa[v][0].w, pb[v][0].x, pb[v][0].y, pb[v][0].z, pb[v][0].w};
+#pragma unroll
+      for (int s = 1; s < kMaxParts; ++s) {
+        if (s < n_parts) {
+          acc[0] += pa[v][s].x; acc[1] += pa[v][s].y; acc[2] += pa[v][s].z; acc[3] += pa[v][s].w;
+          acc[4] += pb[v][s].x; acc[5] += pb[v][s].y; acc[6] += pb[v][s].z; acc[7] += pb[v][s].w;
+        }
+      }
+      float bias[8];
+      unpack8(bias8[v], bias);
+      const float r[8] = {ra[v].x, ra[v].y, ra[v].z, ra[v].w, rb[v].x, rb[v].y, rb[v].z, rb[v].w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[v][i] = r[i] + (acc[i] + bias[i]);
+    }
+  } else {
+    const float* xin = p.x[g] + static_cast<size_t>(row) * H;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const float4 a = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8);
+      const float4 b = *reinterpret_cast<const float4*>(xin + (v * 32 + lane) * 8 + 4);
+      x[v][0] = a.x; x[v][1] = a.y; x[v][2] = a.z; x[v][3] = a.w;
+      x[v][4] = b.x; x[v][5] = b.y; x[v][6] = b.z; x[v][7] = b.w;
+    }
   }
   float* y32 = p.y32[g] != nullptr ? p.y32[g] + static_cast<size_t>(row) * H : nullptr;
   normalise_store<V>(x, p.gamma[g], p.beta[g], p.y[g] + static_cast<size_t>(row) * H, y32, lane, p.eps);
@@ -347,10 +392,15 @@ cudaError_t launch_token_heads(const TokenHeadParams& p, cudaStream_t stream) {
 }
 
 cudaError_t launch_layernorm(const LayerNormParams& p, cudaStream_t stream) {
-  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1) return cudaErrorInvalidValue;
+  if (p.n_groups < 1 || p.n_groups > kMaxGroups || p.rows < 1 || p.n_parts < 0 || p.n_parts > kMaxParts) return cudaErrorInvalidValue;
   dim3 grid((p.rows + kRowThreads / 32 - 1) / (kRowThreads / 32), p.n_groups);
-  if (p.hidden == 768) return launch_kernel(layernorm_kernel<3>, grid, dim3(kRowThreads), 0, stream, p);
-  if (p.hidden == 1024) return launch_kernel(layernorm_kernel<4>, grid, dim3(kRowThreads), 0, stream, p);
+  if (p.n_parts > 0) {
+    if (p.hidden == 768) return launch_kernel(layernorm_kernel<3, true>, grid, dim3(kRowThreads), 0, stream, p);
+    if (p.hidden == 1024) return launch_kernel(layernorm_kernel<4, true>, grid, dim3(kRowThreads), 0, stream, p);
+    return cudaErrorInvalidValue;
+  }
+  if (p.hidden == 768) return launch_kernel(layernorm_kernel<3, false>, grid, dim3(kRowThreads), 0, stream, p);
+  if (p.hidden == 1024) return launch_kernel(layernorm_kernel<4, false>, grid, dim3(kRowThreads), 0, stream, p);
   return cudaErrorInvalidValue;
 }
 

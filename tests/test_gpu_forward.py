@@ -157,6 +157,37 @@ def test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches():
     check_against_oracle(big, wf8, b8, m8, again, rows=[0, 13, 31], check_hidden=False)
 
 
+def test_small_launches_split_the_ffn_down_projection():
+    """Launches of at most 512 rows per layer (small batches; the first-token rows of the last branch layers) run
+    the FFN-down projection as partial sums over four ranges of K (option "ffn_down_split", the default): parity
+    with the oracle at every hidden state with and without it, the two within rounding of each other, and the
+    same bits whatever option "fused_ln" says (the split projection keeps its LayerNorm as its own launch)."""
+    cfg = synth.TreeConfig(trunk_layers=3, tasks=(synth.TaskSpec(0, 1, 1), synth.TaskSpec(2, 2, 3),
+                                                  synth.TaskSpec(3, 0, 2), synth.TaskSpec(1, 1, 2)))
+    w, blob, wf = cached_weights(cfg, 5, random_affine=True)
+    for B, S in ((1, 128), (4, 100), (2, 37)):
+        batch = synth.make_batch(cfg, B, S, 1, S, seed=8 + B)
+        results = {}
+        for split in (1, 0):
+            model = mt.MTModel(cfg, B, S, debug_capture=True)
+            model.set_option("ffn_down_split", split)
+            model.load_weights(blob)
+            tok, seg, lens = dev_batch(batch)
+            logits = torch.full((B, cfg.total_classes), float("nan"), dtype=torch.float32, device="cuda")
+            model.forward(tok, seg, lens, logits)
+            torch.cuda.synchronize()
+            assert model.poll_status() == 0
+            check_against_oracle(cfg, wf, batch, model, logits, rows=range(B))
+            results[split] = logits
+        assert float((results[1] - results[0]).abs().max()) <= 2e-3
+        assert not torch.equal(results[1], results[0]) or B * S > 512, "the option changed nothing: is the split path taken?"
+        for fused in (0, 1, 3):
+            _, other = run_model(cfg, blob, batch, fused_ln=fused)
+            assert torch.equal(other, results[1]), (B, S, fused)
+    # the big batch: only the first-token tails are split; the same bits for every setting of fused_ln is checked
+    # in test_gemm_with_cluster_layernorm_matches_oracle_and_separate_launches
+
+
 def test_cta_pair_gemms_match_oracle_and_single_cta_bits():
     """GEMMs run as pairs of CTAs on 256-row tiles (tcgen05 cta_group::2): parity with the oracle on
     every hidden state; every output element is still one fixed-order sum over K, so the logits are

@@ -182,6 +182,74 @@ def test_layernorm_matches_oracle(rows, H):
     assert torch.equal(y_only, y)
 
 
+@pytest.mark.parametrize("M,N,K,splits", [
+    (1, 768, 3072, 4),       # a first-token tail of a single sequence
+    (32, 768, 3072, 4),      # the first-token tail of the 32 x 128 batch
+    (100, 768, 3072, 4),     # ragged
+    (128, 768, 3072, 4),     # batch 1
+    (512, 768, 3072, 4),     # batch 4: four row blocks
+    (300, 1024, 4096, 4),    # BERT-large width
+    (77, 768, 768, 2),
+])
+@pytest.mark.parametrize("block_n", [0, 64, 128])
+def test_split_k_projection_and_its_layernorm(M, N, K, splits, block_n):
+    """The FFN-down projection of launches of few rows: partial sums over ranges of K, then one kernel that adds the
+    ranges in order, the bias and the residual and normalises the row."""
+    xb, x = rand_bf16(71, f"x{M}.{N}.{K}", (M, K), 1.0)
+    wb, w = rand_bf16(72, f"w{M}.{N}.{K}", (N, K), 0.05)
+    bb, b = rand_bf16(73, f"b{M}.{N}.{K}", (N,), 0.5)
+    gb, g = rand_bf16(74, f"g{N}", (N,), 0.2, mean=1.0)
+    eb, e = rand_bf16(75, f"e{N}", (N,), 0.2)
+    r32 = (synth.standard_normal(76, f"r{M}.{N}.{K}", M * N).astype(np.float32)).reshape(M, N)
+    pitch = (M + 127) // 128 * 128
+    part = torch.full((splits * pitch + 8, N), float("nan"), dtype=torch.float32, device="cuda")   # 8 guard rows
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lib = mt.lib()
+    lib.mt_kernel_linear_force_block_n(block_n)
+    try:
+        mt.mt_kernel_linear_partial(to_dev_bf16(xb), to_dev_bf16(wb), part, splits, pitch, status=status)
+        torch.cuda.synchronize()
+    finally:
+        lib.mt_kernel_linear_force_block_n(0)
+    assert int(status.item()) == 0
+    assert torch.isnan(part[splits * pitch:]).all(), "rows beyond the last range were written"
+    got = part.cpu().numpy()
+    ks = K // splits
+    for s in range(splits):
+        want_s = x[:, s * ks:(s + 1) * ks] @ w[:, s * ks:(s + 1) * ks].T          # this range of K alone, fp64
+        got_s = got[s * pitch:s * pitch + M].astype(np.float64)
+        assert np.all(np.isfinite(got_s))
+        assert rel_l2(got_s, want_s) <= 1e-5, s
+    # the rows put together and normalised, against the oracle's residual sub-layer
+    y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    y32 = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    r_dev = torch.from_numpy(r32).cuda()
+    mt.mt_kernel_layernorm_partial(part, splits, pitch, r_dev, to_dev_bf16(bb), to_dev_bf16(gb), to_dev_bf16(eb), y, 1e-12,
+                                   y_f32=y32)
+    torch.cuda.synchronize()
+    want = orc.layer_norm(r32.astype(np.float64) + orc.linear(x, w, b), g, e, 1e-12)
+    assert rel_l2(dev_bf16_to_f64(y), want) <= OUT_REL_L2
+    assert rel_l2(y32.cpu().numpy().astype(np.float64), want) <= 2e-5
+    # the order of the additions is part of the definition: residual + ((p0 + p1 + ...) + bias) in fp32, formed on
+    # the host from the kernel's own partial sums, must normalise to the same bits
+    acc = got[0:M].copy()
+    for s in range(1, splits):
+        acc = acc + got[s * pitch:s * pitch + M]
+    x_host = r32 + (acc + b.astype(np.float32))
+    y_ref = torch.empty_like(y)
+    mt.mt_kernel_layernorm(torch.from_numpy(x_host.astype(np.float32)).cuda(), to_dev_bf16(gb), to_dev_bf16(eb), y_ref,
+                           1e-12)
+    torch.cuda.synchronize()
+    assert torch.equal(y_ref, y)
+    # and the unsplit kernels give the same result to fp32 rounding of the sum over K
+    u = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    mt.mt_kernel_linear(to_dev_bf16(xb), to_dev_bf16(wb), to_dev_bf16(bb), r_dev, u, 2, status=status)
+    y_plain = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    mt.mt_kernel_layernorm(u, to_dev_bf16(gb), to_dev_bf16(eb), torch.empty_like(y), 1e-12, y_f32=y_plain)
+    torch.cuda.synchronize()
+    assert rel_l2(y32.cpu().numpy().astype(np.float64), y_plain.cpu().numpy().astype(np.float64)) <= 2e-5
+
+
 @pytest.mark.parametrize("H", [768, 1024])
 def test_embed_matches_oracle_and_flags_bad_ids(H):
     B, S, V = 3, 40, 500

@@ -83,16 +83,20 @@ def test_scheduler_masks_and_wavefront_of_the_8_task_tree(lib):
     with pytest.raises(binding.MTError):
         m.plan_summary(0)
     # fused_ln = 1: each residual GEMM carries the LayerNorm after it, so a layer on all tokens is 5 launches
-    # (projection, attention, output + LN, FFN up, FFN down + LN), a first-token tail 3
+    # (projection, attention, output + LN, FFN up, FFN down + LN), a first-token tail 4: its 32 rows per layer are
+    # few enough for the FFN-down projection to be split over K, which keeps its LayerNorm as a launch of its own
     m.set_option("fused_ln", 1)
+    assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 4 + 2
+    m.set_option("ffn_down_split", 0)
     assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 3 + 2
+    m.set_option("ffn_down_split", 1)
     # default (2): where at most two layers are on all tokens: waves 1-5 and wave 9
     m.set_option("fused_ln", 2)
     assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 5 + 2
     m.set_option("fused_ln_max_rows", 128)   # also the first-token tail (32 rows per layer)
-    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 3 + 2
+    assert m.plan_launches(0xFF) == 2 + 5 * 4 + 5 + 7 + 8 + 8 + 6 + 2 + 4 + 2
     m.set_option("fused_ln", 3)
-    assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 3 + 2
+    assert m.plan_launches(0xFF) == 2 + 5 * 6 + 6 * 3 + 2 + 4 + 2
     m.set_option("fused_ln", 0)
     # waves 7, 8, 9 mix layers on all tokens (7 launches) with last branch layers, which only add the
     # first-token attention there; wave 10 holds a last layer alone (projection + first-token attention);
