@@ -334,6 +334,18 @@ int mt_kernel_linear_fp8(const void* d_xq, const float* d_scale_x, const void* d
                          const void* d_bias, const void* d_residual, void* d_y, int32_t M, int32_t N, int32_t K,
                          int32_t epilogue, uint32_t* d_status, void* stream);
 
+/* What a kernel of the path does when one of its pipeline waits never ends.  Every mbarrier wait of the tensor-core
+ * kernels is bounded: after its limit (4 s in the kernels) the waiting role raises its CTA's abort flag, the other
+ * roles see the flag at their next look and leave too, and MT_FLAG_WAIT_TIMEOUT is set in the status word.  This
+ * call runs that same wait in a two-warp kernel with a limit of the caller's choosing (1 us .. 15 ms): warp 0 waits
+ * on a barrier with limit_ns, warp 1 on another with 64 * limit_ns.  arrive == 0: nothing ever completes the
+ * barriers - warp 0's wait runs out, warp 1 leaves through the abort flag, d_status (device, may be NULL) gets
+ * MT_FLAG_WAIT_TIMEOUT; arrive != 0: both barriers are complete, the waits succeed at once.  d_waited_ns[2] and
+ * d_ok[2] (device) receive per warp the nanoseconds waited and 1 / 0 for success.  Nothing faults and the
+ * context stays usable. */
+int mt_debug_wait_probe(uint64_t limit_ns, int32_t arrive, uint32_t* d_status, uint64_t* d_waited_ns, int32_t* d_ok,
+                        void* stream);
+
 /* Partial sums of X[M,K] . W[N,K]^T with K split into k_splits equal ranges (a launch of few rows then has
  * k_splits times as many tiles, each walking a k_splits-th of K): range s writes its fp32 sum, without bias, to rows
  * [s * split_pitch, s * split_pitch + M) of d_part (fp32 [k_splits * split_pitch, N], device).  X, W bf16;

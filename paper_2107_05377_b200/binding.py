@@ -67,6 +67,7 @@ SIGNATURES = {
     "mt_kernel_attention": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _P, _P]),
     "mt_kernel_layernorm": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_linear_partial": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, _I32, _I32, _P, _P]),
+    "mt_debug_wait_probe": (C.c_int, [C.c_uint64, _I32, _P, _P, _P, _P]),
     "mt_kernel_layernorm_partial": (C.c_int, [_P, _I32, _I32, _P, _P, _P, _P, _P, _P, _I32, _I32, C.c_float, _P]),
     "mt_kernel_embed": (C.c_int, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _I32, _I32, C.c_float, _P,
                                   _P]),
@@ -161,6 +162,12 @@ def mt_kernel_layernorm(x, gamma, beta, y, eps: float, y_f32=None, stream=None) 
     rows, hidden = x.shape
     _check(lib().mt_kernel_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), _ptr(y_f32), rows, hidden, eps,
                                      _stream(stream)), "mt_kernel_layernorm")
+
+
+def mt_debug_wait_probe(limit_ns: int, arrive: bool, status, waited_ns, ok, stream=None) -> None:
+    """The kernels' bounded mbarrier wait on a barrier that nothing completes (arrive False) or that is complete."""
+    _check(lib().mt_debug_wait_probe(int(limit_ns), 1 if arrive else 0, _ptr(status), _ptr(waited_ns), _ptr(ok),
+                                     _stream(stream)), "mt_debug_wait_probe")
 
 
 def mt_kernel_linear_partial(x, w, part, k_splits: int, split_pitch: int, status=None, stream=None) -> None:

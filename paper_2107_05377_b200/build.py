@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmt_bert.so")
-SOURCES = ["mt_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "gemm_ln_tcgen05.cu", "gemm_ln_wide_tcgen05.cu", "rowwise.cu", "noalloc.cu"]
+SOURCES = ["mt_api.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "gemm_ln_tcgen05.cu", "gemm_ln_wide_tcgen05.cu", "rowwise.cu", "noalloc.cu", "wait_probe.cu"]
 
 
 def sources():

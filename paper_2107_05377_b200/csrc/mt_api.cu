@@ -1788,6 +1788,14 @@ int mt_kernel_layernorm_partial(const float* d_part, int32_t n_parts, int32_t pa
   return launch_layernorm(p, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
 }
 
+int mt_debug_wait_probe(uint64_t limit_ns, int32_t arrive, uint32_t* d_status, uint64_t* d_waited_ns, int32_t* d_ok,
+                        void* stream) {
+  // (at most a second: the second warp's own limit is 64 times the first's)
+  if (limit_ns < 1000 || limit_ns > 15000000ull || d_waited_ns == nullptr || d_ok == nullptr) return MT_ERR_INVALID_ARG;
+  return launch_wait_probe(limit_ns, arrive != 0 ? 1 : 0, d_status, reinterpret_cast<unsigned long long*>(d_waited_ns),
+                           d_ok, as_stream(stream)) == cudaSuccess ? MT_OK : MT_ERR_CUDA;
+}
+
 int mt_kernel_embed(const int32_t* d_token_ids, const int32_t* d_segment_ids, const int32_t* d_lengths,
                     const void* d_word, const void* d_pos, const void* d_type, const void* d_gamma, const void* d_beta,
                     void* d_h0, void* d_h0_f32, int32_t batch, int32_t seq, int32_t hidden, int32_t vocab,

@@ -275,6 +275,12 @@ struct QuantParams {
 };
 cudaError_t launch_quantize_rows(const QuantParams& p, cudaStream_t stream);
 
+// The kernels' bounded mbarrier wait run on a barrier that nothing completes (arrive == 0) or that is complete
+// (arrive != 0), with a limit of the caller's choosing: waited_ns[2] and ok_out[2] (device) receive, per warp, how
+// long the wait took and whether it succeeded; status gets kFlagWaitTimeout when a wait ran out (wait_probe.cu).
+cudaError_t launch_wait_probe(unsigned long long limit_ns, int arrive, uint32_t* status, unsigned long long* waited_ns,
+                              int* ok_out, cudaStream_t stream);
+
 // row_start[b] for b = 0..batch and *rows_valid = row_start[batch]: b * seq (padded) or the running sum
 // of the lengths clamped to [1, seq] (packed).
 cudaError_t launch_row_starts(const int32_t* lengths, int32_t batch, int32_t seq, int32_t packed, int32_t* row_start,
