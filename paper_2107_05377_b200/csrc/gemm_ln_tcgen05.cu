@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_acc_full + 8 * a, 1);
       mbar_init(bar_acc_empty + 8 * a, kLnEpilogueWarps);
-      mbar_init(bar_stats + 8 * a, static_cast<uint32_t>(cluster_size * kLnEpilogueWarps));
+      mbar_init(bar_stats + 8 * a, 1);   // armed per tile by one thread with the bytes of all statistics
     }
     for (int i = 0; i < 2 * kLnEpilogueWarps; ++i) mbar_init(bar_res + 8 * i, 1);
     *abort_flag = 0;
@@ -204,6 +204,8 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
       const int col0 = n0 + half * 64;
       // the residual of this warp's 32 x 64 block, while the MMAs run
       if (lane == 0) {
+        // (one thread of the CTA) this tile's statistics: 8 bytes from every epilogue thread of the cluster
+        if (e == 0) mbar_expect_tx(bar_stats + 8 * parity, static_cast<uint32_t>(cluster_size * kLnEpilogueWarps * 32 * 8));
         tma_store_wait_read<0>();   // the previous tile's stores have read the staging buffers
         mbar_expect_tx(my_res_bar, kLnStagingBytes);
         tma_load_2d(my_stage, &p.tmap_res[g], col0, row0, my_res_bar);
@@ -275,15 +277,12 @@ __global__ void __launch_bounds__(kLnThreads, 1) gemm_ln_tcgen05(const __grid_co
         for (int j = 0; j < 8; ++j) sub[j] = sumsq8_in_order(*reinterpret_cast<const float(*)[8]>(v + 8 * j), mean_l);
         m2_l = ((sub[0] + sub[1]) + (sub[2] + sub[3])) + ((sub[4] + sub[5]) + (sub[6] + sub[7]));
       }
-      // into slot [parity][rank][half][row] of every CTA of the cluster, then one arrival per warp and CTA
+      // into slot [parity][rank][half][row] of every CTA of the cluster
       const uint32_t slot = sStats + static_cast<uint32_t>((((parity * kLnMaxCluster + rank) * 2 + half) * kGemmBlockM + row_in_tile) * 8);
-      for (int peer = 0; peer < cluster_size; ++peer) st_cluster_f2(map_to_cta(slot, static_cast<uint32_t>(peer)), mean_l, m2_l);
-      __syncwarp();
-      if (lane == 0) {
-        fence_acq_rel_cluster();
-        for (int peer = 0; peer < cluster_size; ++peer)
-          mbar_arrive_cluster_relaxed(map_to_cta(bar_stats + 8 * parity, static_cast<uint32_t>(peer)));
-      }
+      // (asynchronous stores that count their bytes on the receiver's barrier: its wait is all the synchronisation)
+      for (int peer = 0; peer < cluster_size; ++peer)
+        st_async_f2(map_to_cta(slot, static_cast<uint32_t>(peer)), mean_l, m2_l,
+                    map_to_cta(bar_stats + 8 * parity, static_cast<uint32_t>(peer)));
       if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_stats + 8 * parity, stats_phase[parity], abort_flag))) break;
       stats_phase[parity] ^= 1u;
       // merge the 2 * cluster_size segment statistics of this row, in column order
